@@ -1,0 +1,195 @@
+/*
+ * tts_gpt.h — C ABI of the B200 (sm_100a) decode step of IndexTTS-2's Text-to-Semantic GPT.
+ *
+ * The paper ("Faster IndexTTS-2") accelerates a decoder-only autoregressive GPT that emits
+ * semantic codec tokens one per step (Section II-A), fed by a conditioning prefix of embeddings
+ * followed by tokens (Section II-C), batched over concurrent utterances (Sections II-B, II-D),
+ * optionally with W8A16 / W4A16 weight-only quantization (Table I caption, Section III-B), and
+ * returning at every step the token id, the logits and the hidden state of the last layer
+ * (Section II-C).  This library is that engine for one GPU: a paged KV cache of 64-token pages,
+ * dequantizing linears, split-KV decode attention, fused LayerNorm / GELU / residual and greedy or
+ * top-k sampling, all in hand-written CUDA kernels.
+ *
+ * General rules
+ *  - Every function returns an int32 status: TTS_GPT_OK (0) or a negative TTS_GPT_E_* code.
+ *    Nothing throws, aborts or traps the device.  tts_gpt_last_error() describes the last failure.
+ *  - Memory: the caller owns every buffer, including the workspace given to tts_gpt_create.  The
+ *    library never allocates device memory.  "device" below means a pointer valid on the current
+ *    CUDA device, "host" a plain host pointer.  bf16 tensors are 16-bit brain floats, row-major.
+ *  - Asynchrony: prefill / decode_step / release_stream validate on the host, enqueue work on the
+ *    CUDA stream given at create, and return without waiting.  A host-detectable error is
+ *    returned immediately and leaves all state untouched.  Output buffers must stay alive until
+ *    the next tts_gpt_sync (or the caller's own synchronisation of that stream).
+ *  - A handle is not thread-safe; use one handle per thread / per GPU.
+ */
+#ifndef TTS_GPT_H_
+#define TTS_GPT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tts_gpt tts_gpt_t; /* opaque */
+
+/* Storage format of the four block linears (QKV, attention out, FC1, FC2).  Embeddings,
+ * LayerNorm parameters, biases and the LM head are bf16 in every format. */
+enum {
+  TTS_GPT_W_BF16 = 0,      /* bf16 [N,K] */
+  TTS_GPT_W_INT8_PC = 1,   /* int8 [N,K], symmetric, one bf16 scale per output row: W = s[n]*q */
+  TTS_GPT_W_INT4_G128 = 2  /* int32 words [N,K/8]; nibble j (bits 4j..4j+3) of word w holds column
+                              k = 8w+j as u = q+8; bf16 scales [N,K/128]: W = s[n,k/128]*(u-8) */
+};
+
+enum {
+  TTS_GPT_OK = 0,
+  TTS_GPT_E_ARG = -1,          /* invalid argument or configuration */
+  TTS_GPT_E_NO_PAGES = -2,     /* KV page pool exhausted */
+  TTS_GPT_E_STREAM = -3,       /* unknown, released or duplicate stream id; no free stream slot */
+  TTS_GPT_E_CTX_OVERFLOW = -4, /* a stream would exceed max_context */
+  TTS_GPT_E_CUDA = -5,         /* a CUDA runtime call failed */
+  TTS_GPT_E_TIMEOUT = -6,      /* a bounded device-side wait expired */
+  TTS_GPT_E_WORKSPACE = -7,    /* workspace too small or misaligned */
+  TTS_GPT_E_UNSUPPORTED = -8
+};
+
+typedef struct {
+  int32_t n_layer, d_model, n_head, head_dim, d_ff, vocab; /* head_dim must be 64, n_head*64 = d_model */
+  int32_t wfmt;          /* TTS_GPT_W_* of the block linears */
+  int32_t max_streams;   /* concurrent utterances, 1..128 */
+  int32_t max_context;   /* tokens per stream, multiple of page_tokens, <= 2048 */
+  int32_t page_tokens;   /* must be 64 */
+  int32_t n_pages;       /* pages in the KV pool (each holds 64 tokens of every layer) */
+  int32_t max_pos;       /* rows of pos_emb */
+  int32_t gelu_tanh;     /* 1: tanh-form GELU (GPT-2), 0: erf form */
+  int32_t stop_token;    /* -1: none */
+  float ln_eps;          /* LayerNorm epsilon (inside the square root) */
+} tts_gpt_config_t;
+
+/* All DEVICE pointers, read only during tts_gpt_create (the library keeps its own re-laid-out
+ * copy in the workspace; the caller may free these afterwards).  Per-layer entries are HOST arrays
+ * of n_layer device pointers.  Shapes: tok_emb [vocab,d]; pos_emb [max_pos,d]; ln*_g/_b [d];
+ * head_w [vocab,d]; head_b [vocab] or NULL; qkv_w [3d,d] with rows ordered Q,K,V and head h owning
+ * columns 64h..64h+63 of each; o_w [d,d]; fc1_w [d_ff,d]; fc2_w [d,d_ff]; *_b bf16 [N];
+ * *_s bf16 scales (NULL array or NULL entries for bf16 weights). */
+typedef struct {
+  const void *tok_emb, *pos_emb, *lnf_g, *lnf_b, *head_w, *head_b;
+  const void *const *ln1_g, *const *ln1_b, *const *ln2_g, *const *ln2_b;
+  const void *const *qkv_w, *const *qkv_s, *const *qkv_b;
+  const void *const *o_w, *const *o_s, *const *o_b;
+  const void *const *fc1_w, *const *fc1_s, *const *fc1_b;
+  const void *const *fc2_w, *const *fc2_s, *const *fc2_b;
+} tts_gpt_weights_t;
+
+/* Bytes of device workspace tts_gpt_create needs for this configuration (weights in streaming
+ * layout + KV pool + page tables + activations + scratch).  No CUDA call is made. */
+int32_t tts_gpt_query_workspace(const tts_gpt_config_t *cfg, size_t *bytes);
+
+/* Build an engine inside `workspace` (device, 256-byte aligned, >= query_workspace bytes).
+ * `cuda_stream` is a cudaStream_t (NULL = default stream) on which every later call enqueues.
+ * Re-lays the weights out for streaming, clears the page allocator and synchronises the stream
+ * once before returning.  The handle itself is a small host object freed by tts_gpt_destroy. */
+int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *weights,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream, tts_gpt_t **out);
+
+/* Context phase (Section II-C: conditioning embeddings, then text, precede the semantic tokens).
+ * Opens n new streams.  prefix_emb: HOST array of n DEVICE pointers to bf16 [prefix_len[i], d]
+ * embeddings that are used as given (the caller has already added, or for the conditioning rows
+ * not added, positional embeddings).  pos0[i] (HOST, may be NULL = 0) is the index into pos_emb of
+ * the stream's first generated token.  Fills the KV cache for positions 0..P_i-1, computes the
+ * logits of the last prefix row and samples y_0 from them with (top_k, temperature, uniforms).
+ * out_stream_ids: HOST [n], written before return.  out_tokens: DEVICE int32 [n].
+ * out_logits: DEVICE fp32 [n,vocab] or NULL.  out_hidden: DEVICE bf16 [n,d] or NULL (final
+ * LayerNorm output).  uniforms: DEVICE fp32 [n] in [0,1), needed only when top_k > 1.
+ * Errors: E_ARG (n < 1, a prefix_len < 1), E_STREAM (fewer than n free slots), E_CTX_OVERFLOW
+ * (prefix_len > max_context), E_NO_PAGES.  All-or-nothing. */
+int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb,
+                        const int32_t *prefix_len, const int32_t *pos0, int32_t top_k,
+                        float temperature, const float *uniforms, int32_t *out_stream_ids,
+                        int32_t *out_tokens, float *out_logits, void *out_hidden);
+
+/* One incremental decode step (Sections I, II-C) for n distinct open streams (stream_ids: HOST).
+ * Stream i consumes one input token — in_tokens[i] (DEVICE int32 [n]) or, if in_tokens is NULL,
+ * the token it sampled last — embedded as tok_emb[token] + pos_emb[pos0 + k - 1] on its k-th
+ * step, appends that token's K/V at position ctx_i, attends over ctx_i + 1 keys, and returns the
+ * logits of the next token, the sampled next token and optionally the final-LayerNorm hidden row.
+ * top_k 0 or 1 = greedy (lowest index on ties); top_k in 2..64 = softmax over the top_k logits
+ * at `temperature`, inverse CDF with uniforms[i].  Afterwards ctx_i += 1.
+ * Errors: E_ARG, E_STREAM (unknown / duplicate id), E_CTX_OVERFLOW (ctx_i + 1 > max_context),
+ * E_NO_PAGES.  All-or-nothing; nothing is enqueued on error. */
+int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
+                            const int32_t *in_tokens, int32_t top_k, float temperature,
+                            const float *uniforms, int32_t *out_tokens, float *out_logits,
+                            void *out_hidden);
+
+/* Close a stream and return its pages to the pool.  E_STREAM if the id is not open. */
+int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t stream_id);
+
+/* Wait for the engine's CUDA stream; returns a deferred device-side error if one was recorded. */
+int32_t tts_gpt_sync(tts_gpt_t *h);
+
+/* Free the host handle (after synchronising).  The workspace stays the caller's. */
+int32_t tts_gpt_destroy(tts_gpt_t *h);
+
+/* Human-readable description of the last error on this handle (NULL handle: of the last failed
+ * create / query on this thread).  The string is owned by the library. */
+const char *tts_gpt_last_error(const tts_gpt_t *h);
+
+/* Introspection used by tests and the bench (HOST outputs, any may be NULL): open streams, free
+ * pages, and the context length of one stream (-1 if not open). */
+int32_t tts_gpt_stats(const tts_gpt_t *h, int32_t *open_streams, int32_t *free_pages);
+int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t stream_id);
+
+/* Test aid: permute the free-page list with a seeded shuffle (between calls, any time no stream
+ * is open).  Results must not depend on which physical pages a stream receives. */
+int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed);
+
+/* ---------------------------------------------------------------------------------------------
+ * Single-kernel entry points: the building blocks of the step, callable on their own (unit parity
+ * tests, micro-benchmarks).  All pointers DEVICE unless marked HOST; `cuda_stream` as above; each
+ * call enqueues and returns.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Bytes of the streaming layout of one [N,K] linear in format wfmt (weights + scales). */
+int32_t tts_gpt_op_linear_packed_bytes(int32_t wfmt, int32_t N, int32_t K, size_t *bytes);
+
+/* Re-lay a canonical [N,K] matrix (formats above) into `packed` (device, 256-byte aligned,
+ * >= packed_bytes).  K must be a multiple of 128. */
+int32_t tts_gpt_op_linear_pack(int32_t wfmt, int32_t N, int32_t K, const void *w, const void *s,
+                               void *packed, void *cuda_stream);
+
+/* out[b,n] = sum_k W[n,k] * act[b,k] + bias[n]  (the weight-only dequantizing linear: Table I
+ * caption).  act bf16 [B,K], bias bf16 [N] or NULL, out fp32 [B,N], 1 <= B <= 128. */
+int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed, const void *bias,
+                          int32_t B, const void *act, float *out, void *cuda_stream);
+
+/* Bytes of scratch tts_gpt_op_attention needs for R rows of n_head heads. */
+int32_t tts_gpt_op_attention_scratch_bytes(int32_t R, int32_t n_head, size_t *bytes);
+
+/* Decode attention over a paged KV cache (Section I: attention kernels + KV-cache management of
+ * the decode engine).  Row r belongs to stream row_stream[r] and attends over keys 0..row_pos[r]
+ * of that stream: o = softmax(q.K^T / 8) V per head.  q fp32 [R, n_head*64]; kv_layer: one
+ * layer's slice of the pool, bf16 [n_pages][2 (K,V)][n_head][64 tokens][64]; page_table int32
+ * [*, pages_per_stream]; out bf16 [R, n_head*64].  `scratch` (>= scratch_bytes, 256-byte aligned)
+ * must be zero on first use; the kernel leaves it zeroed where that matters. */
+int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                             const int32_t *page_table, int32_t pages_per_stream,
+                             const int32_t *row_stream, const int32_t *row_pos, void *out,
+                             void *scratch, void *cuda_stream);
+
+/* LayerNorm over rows: x fp32 [R,d], g/b bf16 [d] -> out bf16 [R,d]. */
+int32_t tts_gpt_op_layernorm(int32_t R, int32_t d, const float *x, const void *g, const void *b,
+                             float eps, void *out, void *cuda_stream);
+
+/* Sampling (Section I: sampling strategies of the decode engine): logits fp32 [R,V]; top_k <= 1
+ * greedy, else top-k softmax at `temperature` with inverse CDF on uniforms[r]; tokens int32 [R]. */
+int32_t tts_gpt_op_sample(int32_t R, int32_t V, const float *logits, int32_t top_k,
+                          float temperature, const float *uniforms, int32_t *tokens,
+                          void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TTS_GPT_H_ */

@@ -1,0 +1,273 @@
+// Embedding lookup, LayerNorm and sampling kernels, plus the per-step I/O block they read.
+#pragma once
+#include "common.cuh"
+
+namespace ttsgpt {
+
+// Per-call I/O pointers and sampling settings, kept in device memory so that a captured CUDA graph
+// of the step can be replayed while the caller changes buffers from step to step.
+struct StepIO {
+  const int *in_tokens;
+  const float *uniforms;
+  int *out_tokens;
+  float *out_logits;
+  uint16_t *out_hidden;
+  int top_k;
+  float temperature;
+  int n_out;
+};
+
+// Per-pass row table (device arrays of kMaxRows entries).  A row is one (stream, position) pair.
+struct RowTable {
+  int *row_stream;            // stream slot of the row
+  int *row_pos;               // position in the stream's context the row occupies (its K/V slot)
+  int *row_token;             // >= 0: token id to embed; -1: take row_emb
+  int *row_posidx;            // index into pos_emb for token rows
+  const uint16_t **row_emb;   // bf16 [d] embedding of a prefix row
+  int *out_rows;              // rows whose logits are wanted, compacted
+  int *out_slot;              // position of that row's results in the caller's output arrays
+};
+
+// x[r,:] = tok_emb[token] + pos_emb[posidx]   (generated tokens take a positional embedding from
+// their own range of the position table; prefix embeddings are used as given: Section II-C)
+__global__ void embed_kernel(RowTable rt, const uint16_t *__restrict__ tok_emb, const uint16_t *__restrict__ pos_emb,
+                             int d, int vocab, int max_pos, float *__restrict__ x) {
+  const int r = blockIdx.x;
+  int tok = rt.row_token[r];
+  float *xr = x + (size_t)r * d;
+  if (tok >= 0) {
+    tok = min(tok, vocab - 1);
+    const int p = min(max(rt.row_posidx[r], 0), max_pos - 1);
+    const uint16_t *te = tok_emb + (size_t)tok * d, *pe = pos_emb + (size_t)p * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) xr[i] = bf16_bits_to_float(te[i]) + bf16_bits_to_float(pe[i]);
+  } else {
+    const uint16_t *e = rt.row_emb[r];
+    for (int i = threadIdx.x; i < d; i += blockDim.x) xr[i] = bf16_bits_to_float(e[i]);
+  }
+}
+
+__device__ __forceinline__ float block_sum(float v, float *sm) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) sm[warp] = v;
+  __syncthreads();
+  float t = 0.f;
+  for (int w = 0; w < nw; ++w) t += sm[w];
+  return t;
+}
+
+// LayerNorm of fp32 rows (biased variance, eps inside the square root), bf16 out.  With `gather`
+// row j of the output is row gather[j] of x; `io` (optional) also receives the rows at out_slot.
+constexpr int kLnThreads = 256;
+constexpr int kLnMaxPerThread = 8;  // d <= 2048
+__global__ void __launch_bounds__(kLnThreads) layernorm_kernel(const float *__restrict__ x, int d,
+                                                               const uint16_t *__restrict__ g,
+                                                               const uint16_t *__restrict__ b, float eps,
+                                                               uint16_t *__restrict__ out, const int *gather,
+                                                               const int *out_slot, const StepIO *io) {
+  __shared__ float sm[kLnThreads / 32];
+  const int j = blockIdx.x;
+  const int r = gather ? gather[j] : j;
+  const float *xr = x + (size_t)r * d;
+  float v[kLnMaxPerThread];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    v[i] = c < d ? xr[c] : 0.f;
+    s += v[i];
+  }
+  const float mu = block_sum(s, sm) / d;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    const float t = c < d ? v[i] - mu : 0.f;
+    q += t * t;
+  }
+  const float rstd = rsqrtf(block_sum(q, sm) / d + eps);
+  uint16_t *hid = (io && io->out_hidden) ? io->out_hidden + (size_t)(out_slot ? out_slot[j] : j) * d : nullptr;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    if (c < d) {
+      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * bf16_bits_to_float(g[c]) + bf16_bits_to_float(b[c]));
+      out[(size_t)j * d + c] = y;
+      if (hid) hid[c] = y;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// sampling
+// ------------------------------------------------------------------------------------------
+constexpr int kSampleThreads = 1024;
+constexpr int kSampleMaxPer = 9;   // vocab <= 9216
+constexpr int kMaxTopK = 64;
+
+__device__ __forceinline__ uint32_t float_to_ordered(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+struct SampleArgs {
+  const float *logits;   // [n][V], compact
+  int V;
+  const StepIO *io;      // if non-null: settings and pointers come from here
+  int top_k; float temperature; const float *uniforms; int *out_tokens;  // used when io == null
+  const int *out_slot, *out_rows, *row_stream;  // optional
+  int *last_token;       // optional, indexed by stream
+  int *stop_flag; int stop_token;
+};
+
+// One CTA per row.  Greedy: arg max, lowest index on ties.  Top-k: the k largest by (logit
+// descending, index ascending) found by a 4-pass radix select on the order-preserving integer
+// image of the float, then w_r = exp((l_r - l_0)/T), inverse CDF on the caller's uniform.
+__global__ void __launch_bounds__(kSampleThreads) sample_kernel(const SampleArgs a) {
+  extern __shared__ float lg[];  // V floats
+  __shared__ unsigned int hist[256];
+  __shared__ unsigned int sh_prefix, sh_remaining, sh_count;
+  __shared__ float wv[32]; __shared__ int wi[32];
+  __shared__ unsigned int tie_warp[32];
+  __shared__ float sel_v[kMaxTopK]; __shared__ int sel_i[kMaxTopK];
+  __shared__ float srt_v[kMaxTopK]; __shared__ int srt_i[kMaxTopK];
+
+  const int j = blockIdx.x;
+  const int slot = a.out_slot ? a.out_slot[j] : j;
+  const int V = a.V;
+  const float *src = a.logits + (size_t)j * V;
+  int top_k = a.top_k; float temperature = a.temperature;
+  const float *uniforms = a.uniforms; int *out_tokens = a.out_tokens; float *out_logits = nullptr;
+  if (a.io) {
+    top_k = a.io->top_k; temperature = a.io->temperature; uniforms = a.io->uniforms;
+    out_tokens = a.io->out_tokens; out_logits = a.io->out_logits;
+  }
+  for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    const float v = src[i];
+    lg[i] = v;
+    if (out_logits) out_logits[(size_t)slot * V + i] = v;
+  }
+  __syncthreads();
+  // blocked ownership: thread t owns indices [t*per, t*per+per)
+  const int per = (V + blockDim.x - 1) / blockDim.x;
+  const int i0 = threadIdx.x * per;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int token;
+
+  if (top_k <= 1) {
+    float bv = -INFINITY; int bi = 0x7FFFFFFF;
+    for (int q = 0; q < per; ++q) {
+      const int i = i0 + q;
+      if (i < V) { const float v = lg[i]; if (v > bv) { bv = v; bi = i; } }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+      const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+      if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+    }
+    if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w)
+      if (wv[w] > bv || (wv[w] == bv && wi[w] < bi)) { bv = wv[w]; bi = wi[w]; }
+    token = bi;
+  } else {
+    if (top_k > kMaxTopK) top_k = kMaxTopK;
+    if (top_k > V) top_k = V;
+    uint32_t ok[kSampleMaxPer];
+#pragma unroll
+    for (int q = 0; q < kSampleMaxPer; ++q) {
+      const int i = i0 + q;
+      ok[q] = (q < per && i < V) ? float_to_ordered(lg[i]) : 0u;
+    }
+    if (threadIdx.x == 0) { sh_prefix = 0u; sh_remaining = (unsigned)top_k; sh_count = 0u; }
+    uint32_t mask = 0u;
+    for (int pass = 3; pass >= 0; --pass) {
+      const int shift = 8 * pass;
+      if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
+      __syncthreads();
+      const uint32_t prefix = sh_prefix;
+#pragma unroll
+      for (int q = 0; q < kSampleMaxPer; ++q) {
+        const int i = i0 + q;
+        if (q < per && i < V && (ok[q] & mask) == prefix) atomicAdd(&hist[(ok[q] >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        unsigned int rem = sh_remaining, cum = 0u;
+        int bin = 255;
+        for (; bin > 0; --bin) {
+          if (cum + hist[bin] >= rem) break;
+          cum += hist[bin];
+        }
+        sh_remaining = rem - cum;
+        sh_prefix = prefix | ((uint32_t)bin << shift);
+      }
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+    const uint32_t thr = sh_prefix;           // ordered image of the k-th largest logit
+    const unsigned int need_ties = sh_remaining;  // how many entries equal to it belong to the top k
+    // rank ties by index: blocked ownership makes (thread, local order) the index order
+    unsigned int my_ties = 0u;
+#pragma unroll
+    for (int q = 0; q < kSampleMaxPer; ++q) {
+      const int i = i0 + q;
+      if (q < per && i < V && ok[q] == thr) ++my_ties;
+    }
+    unsigned int incl = my_ties;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) tie_warp[warp] = incl;
+    __syncthreads();
+    unsigned int base = incl - my_ties;
+    for (int w = 0; w < warp; ++w) base += tie_warp[w];
+#pragma unroll
+    for (int q = 0; q < kSampleMaxPer; ++q) {
+      const int i = i0 + q;
+      if (q < per && i < V) {
+        bool take = ok[q] > thr;
+        if (ok[q] == thr) { take = base < need_ties; ++base; }
+        if (take) {
+          const unsigned int p = atomicAdd(&sh_count, 1u);
+          if (p < (unsigned)kMaxTopK) { sel_v[p] = lg[i]; sel_i[p] = i; }
+        }
+      }
+    }
+    __syncthreads();
+    const int k = min((int)sh_count, top_k);
+    if ((int)threadIdx.x < k) {
+      const float v = sel_v[threadIdx.x]; const int id = sel_i[threadIdx.x];
+      int rank = 0;
+      for (int q = 0; q < k; ++q) rank += (sel_v[q] > v) || (sel_v[q] == v && sel_i[q] < id);
+      srt_v[rank] = v; srt_i[rank] = id;
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    const float inv_t = 1.0f / temperature;
+    float w[kMaxTopK];
+    float total = 0.f;
+    for (int r = 0; r < k; ++r) { w[r] = expf((srt_v[r] - srt_v[0]) * inv_t); total += w[r]; }
+    const float u = uniforms ? uniforms[slot] : 0.f;
+    float cum = 0.f;
+    token = srt_i[k - 1];
+    for (int r = 0; r < k; ++r) {
+      cum += w[r];
+      if (u < cum / total) { token = srt_i[r]; break; }
+    }
+  }
+  // thread 0 only
+  out_tokens[slot] = token;
+  if (a.last_token) {
+    const int s = a.row_stream[a.out_rows ? a.out_rows[j] : j];
+    a.last_token[s] = token;
+    if (a.stop_flag && token == a.stop_token) a.stop_flag[s] = 1;
+  }
+}
+
+}  // namespace ttsgpt

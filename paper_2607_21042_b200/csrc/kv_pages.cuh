@@ -1,0 +1,141 @@
+// KV page allocator and per-call set-up kernels (Section I: KV-cache management of the decode
+// engine).  The allocator state lives in device memory: a stack of free page ids, one page table
+// row and one context length per stream.  Set-up kernels receive the call's small host arrays BY
+// VALUE as kernel parameters, so no host staging buffer has to outlive the call and no step waits
+// for the host.  The host keeps only counters (free pages, context lengths), which evolve
+// deterministically, to reject calls that cannot succeed before anything is enqueued.
+#pragma once
+#include "common.cuh"
+#include "elementwise.cuh"
+
+namespace ttsgpt {
+
+struct PageState {
+  int *ctx_len;     // [max_streams]
+  int *page_table;  // [max_streams][pps]
+  int *free_list;   // [n_pages] stack; free_top entries valid
+  int *free_top;    // [1]
+  int *last_token;  // [max_streams]
+  int *pos_next;    // [max_streams] pos_emb index of the next generated token
+  int *stop_flag;   // [max_streams]
+  const uint16_t **stream_emb;  // [max_streams] prefix base pointer during prefill
+  int pps, n_pages, max_streams;
+};
+
+__global__ void init_pages_kernel(PageState ps) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < ps.n_pages) ps.free_list[i] = ps.n_pages - 1 - i;  // page 0 is popped first
+  if (i < ps.max_streams) { ps.ctx_len[i] = 0; ps.last_token[i] = 0; ps.pos_next[i] = 0; ps.stop_flag[i] = 0; }
+  if (i < ps.max_streams * ps.pps) ps.page_table[i] = 0;
+  if (i == 0) *ps.free_top = ps.n_pages;
+}
+
+// exclusive prefix sum of one int per thread over a block of kMaxRows threads
+__device__ __forceinline__ int block_exclusive_scan_128(int v, int *total) {
+  __shared__ int warp_tot[kMaxRows / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += n;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int base = 0, tot = 0;
+  for (int w = 0; w < kMaxRows / 32; ++w) { if (w < warp) base += warp_tot[w]; tot += warp_tot[w]; }
+  *total = tot;
+  return base + incl - v;
+}
+
+struct StepParams {
+  int n;
+  int stream_ids[kMaxRows];
+  StepIO io;
+};
+
+// One decode step: each stream whose context length sits on a page boundary pops a page (streams
+// in call order take pages in stack order), then the row table is written and ctx_len advances.
+__global__ void __launch_bounds__(kMaxRows) step_setup_kernel(const StepParams p, PageState ps, RowTable rt, StepIO *io) {
+  const int i = threadIdx.x;
+  int s = 0, t = 0, need = 0;
+  if (i < p.n) { s = p.stream_ids[i]; t = ps.ctx_len[s]; need = (t % kPageTokens) == 0; }
+  int total;
+  const int rank = block_exclusive_scan_128(need, &total);
+  const int top = *ps.free_top;
+  if (i < p.n) {
+    if (need) ps.page_table[(size_t)s * ps.pps + t / kPageTokens] = ps.free_list[top - 1 - rank];
+    rt.row_stream[i] = s;
+    rt.row_pos[i] = t;
+    rt.row_token[i] = p.io.in_tokens ? max(p.io.in_tokens[i], 0) : ps.last_token[s];
+    rt.row_posidx[i] = ps.pos_next[s];
+    rt.out_rows[i] = i;
+    rt.out_slot[i] = i;
+    ps.ctx_len[s] = t + 1;
+    ps.pos_next[s] += 1;
+  }
+  __syncthreads();
+  if (i == 0) { *ps.free_top = top - total; *io = p.io; }
+}
+
+struct PrefillParams {
+  int n;
+  int stream_ids[kMaxRows];
+  int prefix_len[kMaxRows];
+  int pos0[kMaxRows];
+  const uint16_t *emb[kMaxRows];
+};
+
+// Opens the streams of a prefill call: reserves ceil(P/64) pages each, sets ctx_len = P.
+__global__ void __launch_bounds__(kMaxRows) prefill_open_kernel(const PrefillParams p, PageState ps) {
+  const int i = threadIdx.x;
+  int need = 0;
+  if (i < p.n) need = (p.prefix_len[i] + kPageTokens - 1) / kPageTokens;
+  int total;
+  const int base = block_exclusive_scan_128(need, &total);
+  const int top = *ps.free_top;
+  if (i < p.n) {
+    const int s = p.stream_ids[i];
+    for (int j = 0; j < need; ++j) ps.page_table[(size_t)s * ps.pps + j] = ps.free_list[top - 1 - (base + j)];
+    ps.ctx_len[s] = p.prefix_len[i];
+    ps.pos_next[s] = p.pos0[i];
+    ps.stop_flag[s] = 0;
+    ps.stream_emb[s] = p.emb[i];
+  }
+  __syncthreads();
+  if (i == 0) *ps.free_top = top - total;
+}
+
+struct PassParams {
+  int n_rows, n_out;
+  short row_stream[kMaxRows], row_pos[kMaxRows], out_rows[kMaxRows], out_slot[kMaxRows];
+  StepIO io;
+};
+
+// Row table of one prefill pass: up to 128 (stream, position) rows taken from the prefixes.
+__global__ void __launch_bounds__(kMaxRows) prefill_pass_kernel(const PassParams p, PageState ps, RowTable rt, StepIO *io, int d) {
+  const int i = threadIdx.x;
+  if (i < p.n_rows) {
+    const int s = p.row_stream[i], t = p.row_pos[i];
+    rt.row_stream[i] = s;
+    rt.row_pos[i] = t;
+    rt.row_token[i] = -1;
+    rt.row_posidx[i] = 0;
+    rt.row_emb[i] = ps.stream_emb[s] + (size_t)t * d;
+  }
+  if (i < p.n_out) { rt.out_rows[i] = p.out_rows[i]; rt.out_slot[i] = p.out_slot[i]; }
+  if (i == 0) *io = p.io;
+}
+
+// Returns a stream's pages to the stack (last page first, so that the next stream to open pops
+// them in the order this one received them).
+__global__ void release_kernel(PageState ps, int s) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const int n = (ps.ctx_len[s] + kPageTokens - 1) / kPageTokens;
+  int top = *ps.free_top;
+  for (int j = n - 1; j >= 0; --j) ps.free_list[top++] = ps.page_table[(size_t)s * ps.pps + j];
+  *ps.free_top = top;
+  ps.ctx_len[s] = 0;
+}
+
+}  // namespace ttsgpt

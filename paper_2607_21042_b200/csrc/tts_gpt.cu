@@ -1,0 +1,616 @@
+// C ABI of the decode engine: host-side validation, workspace carving, the step schedule.
+// All arithmetic of the step happens in the kernels of the headers included below.
+#include "../../include/tts_gpt.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstdarg>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "linear.cuh"
+#include "attention.cuh"
+#include "elementwise.cuh"
+#include "kv_pages.cuh"
+
+using namespace ttsgpt;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+struct PackedLinear {
+  void *w = nullptr;
+  uint16_t *s = nullptr;
+  uint16_t *bias = nullptr;
+  int N = 0, K = 0;
+};
+
+struct LayerW {
+  uint16_t *ln1_g, *ln1_b, *ln2_g, *ln2_b;
+  PackedLinear qkv, o, fc1, fc2;
+};
+
+}  // namespace
+
+struct tts_gpt {
+  tts_gpt_config_t cfg;
+  cudaStream_t stream;
+  int pps;  // pages per stream
+  std::string err;
+  // weights (workspace)
+  uint16_t *tok_emb, *pos_emb, *lnf_g, *lnf_b;
+  PackedLinear head;
+  std::vector<LayerW> layers;
+  // KV pool
+  uint16_t *kv;
+  size_t kv_layer_elems;
+  // state
+  PageState ps;
+  RowTable rt;
+  StepIO *io;
+  // activations
+  float *x, *q, *logits;
+  uint16_t *a, *o, *hbuf, *hf;
+  // attention scratch
+  float *attn_partials;
+  unsigned int *attn_tickets;
+  // host mirrors
+  std::vector<char> open;
+  std::vector<int> ctx, pos_next;
+  int n_free;
+  // step graphs by row count
+  std::map<int, cudaGraphExec_t> graphs;
+  bool use_graph;
+};
+
+namespace {
+
+int fail(tts_gpt *h, int code, const char *fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (h) h->err = buf;
+  g_last_error = buf;
+  return code;
+}
+
+#define CUDA_TRY(h, expr)                                                                      \
+  do {                                                                                         \
+    cudaError_t e_ = (expr);                                                                   \
+    if (e_ != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+  } while (0)
+
+int check_config(const tts_gpt_config_t *c) {
+  if (!c) return fail(nullptr, TTS_GPT_E_ARG, "null config");
+  if (c->head_dim != 64 || c->page_tokens != 64) return fail(nullptr, TTS_GPT_E_UNSUPPORTED, "head_dim and page_tokens must be 64");
+  if (c->n_layer < 1 || c->n_head < 1 || c->d_model != c->n_head * 64) return fail(nullptr, TTS_GPT_E_ARG, "d_model must equal n_head*64");
+  if (c->d_model % 128 || c->d_ff % 128 || c->d_ff < 128) return fail(nullptr, TTS_GPT_E_ARG, "d_model and d_ff must be multiples of 128");
+  if (c->d_model > kLnThreads * kLnMaxPerThread) return fail(nullptr, TTS_GPT_E_UNSUPPORTED, "d_model too large");
+  if (c->vocab < 2 || c->vocab > kSampleThreads * kSampleMaxPer) return fail(nullptr, TTS_GPT_E_UNSUPPORTED, "vocab out of range");
+  if (c->wfmt < 0 || c->wfmt > 2) return fail(nullptr, TTS_GPT_E_ARG, "unknown weight format");
+  if (c->max_streams < 1 || c->max_streams > kMaxRows) return fail(nullptr, TTS_GPT_E_ARG, "max_streams must be 1..128");
+  if (c->max_context < 64 || c->max_context % 64 || c->max_context > kAttnMaxChunks * kAttnWarps * 64)
+    return fail(nullptr, TTS_GPT_E_ARG, "max_context must be a multiple of 64 in 64..2048");
+  if (c->n_pages < 1 || c->max_pos < 1) return fail(nullptr, TTS_GPT_E_ARG, "n_pages and max_pos must be positive");
+  if (!(c->ln_eps > 0.f)) return fail(nullptr, TTS_GPT_E_ARG, "ln_eps must be positive");
+  return TTS_GPT_OK;
+}
+
+// Walks the workspace; with base == nullptr only measures.
+struct Carver {
+  char *base;
+  size_t off = 0;
+  explicit Carver(void *b) : base((char *)b) {}
+  template <typename T>
+  T *take(size_t count) {
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += align256(count * sizeof(T));
+    return p;
+  }
+};
+
+void carve_linear(Carver &cv, PackedLinear &pl, int wf, int N, int K) {
+  pl.N = N; pl.K = K;
+  pl.w = cv.take<char>(packed_weight_bytes(wf, N, K));
+  size_t sb = packed_scale_bytes(wf, N, K);
+  pl.s = sb ? cv.take<uint16_t>(sb / 2) : nullptr;
+  pl.bias = cv.take<uint16_t>(N);
+}
+
+size_t carve(tts_gpt *h, void *base) {
+  const tts_gpt_config_t &c = h->cfg;
+  const int d = c.d_model, F = c.d_ff, V = c.vocab, S = c.max_streams;
+  h->pps = c.max_context / 64;
+  Carver cv(base);
+  h->tok_emb = cv.take<uint16_t>((size_t)V * d);
+  h->pos_emb = cv.take<uint16_t>((size_t)c.max_pos * d);
+  h->lnf_g = cv.take<uint16_t>(d);
+  h->lnf_b = cv.take<uint16_t>(d);
+  carve_linear(cv, h->head, WF_BF16, V, d);
+  h->layers.resize(c.n_layer);
+  for (auto &L : h->layers) {
+    L.ln1_g = cv.take<uint16_t>(d); L.ln1_b = cv.take<uint16_t>(d);
+    L.ln2_g = cv.take<uint16_t>(d); L.ln2_b = cv.take<uint16_t>(d);
+    carve_linear(cv, L.qkv, c.wfmt, 3 * d, d);
+    carve_linear(cv, L.o, c.wfmt, d, d);
+    carve_linear(cv, L.fc1, c.wfmt, F, d);
+    carve_linear(cv, L.fc2, c.wfmt, d, F);
+  }
+  h->kv_layer_elems = (size_t)c.n_pages * 2 * c.n_head * kPageElems;
+  h->kv = cv.take<uint16_t>(h->kv_layer_elems * c.n_layer);
+  PageState &ps = h->ps;
+  ps.pps = h->pps; ps.n_pages = c.n_pages; ps.max_streams = S;
+  ps.ctx_len = cv.take<int>(S);
+  ps.page_table = cv.take<int>((size_t)S * h->pps);
+  ps.free_list = cv.take<int>(c.n_pages);
+  ps.free_top = cv.take<int>(1);
+  ps.last_token = cv.take<int>(S);
+  ps.pos_next = cv.take<int>(S);
+  ps.stop_flag = cv.take<int>(S);
+  ps.stream_emb = cv.take<const uint16_t *>(S);
+  RowTable &rt = h->rt;
+  rt.row_stream = cv.take<int>(kMaxRows);
+  rt.row_pos = cv.take<int>(kMaxRows);
+  rt.row_token = cv.take<int>(kMaxRows);
+  rt.row_posidx = cv.take<int>(kMaxRows);
+  rt.row_emb = cv.take<const uint16_t *>(kMaxRows);
+  rt.out_rows = cv.take<int>(kMaxRows);
+  rt.out_slot = cv.take<int>(kMaxRows);
+  h->io = cv.take<StepIO>(1);
+  h->x = cv.take<float>((size_t)kMaxRows * d);
+  h->q = cv.take<float>((size_t)kMaxRows * d);
+  h->logits = cv.take<float>((size_t)kMaxRows * V);
+  h->a = cv.take<uint16_t>((size_t)kMaxRows * d);
+  h->o = cv.take<uint16_t>((size_t)kMaxRows * d);
+  h->hbuf = cv.take<uint16_t>((size_t)kMaxRows * F);
+  h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
+  h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
+  h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
+  return cv.off;
+}
+
+int copy_bf16(tts_gpt *h, uint16_t *dst, const void *src, size_t n, const char *what) {
+  if (!src) return fail(h, TTS_GPT_E_ARG, "weights: %s is null", what);
+  CUDA_TRY(h, cudaMemcpyAsync(dst, src, n * 2, cudaMemcpyDeviceToDevice, h->stream));
+  return TTS_GPT_OK;
+}
+
+int load_linear(tts_gpt *h, PackedLinear &pl, int wf, const void *w, const void *s, const void *b, const char *what) {
+  if (!w || !b || (wf != WF_BF16 && !s)) return fail(h, TTS_GPT_E_ARG, "weights: %s has a null tensor", what);
+  CUDA_TRY(h, launch_pack(wf, pl.N, pl.K, w, s, pl.w, pl.s, h->stream));
+  CUDA_TRY(h, cudaMemcpyAsync(pl.bias, b, (size_t)pl.N * 2, cudaMemcpyDeviceToDevice, h->stream));
+  return TTS_GPT_OK;
+}
+
+LinearArgs linear_args(const PackedLinear &pl, const uint16_t *act, int B, int mode) {
+  LinearArgs a;
+  memset(&a, 0, sizeof a);
+  a.w = pl.w; a.scales = pl.s; a.bias = pl.bias; a.act = act;
+  a.N = pl.N; a.K = pl.K; a.B = B; a.mode = mode;
+  return a;
+}
+
+// The transformer blocks for R rows already described by the row table, x holding the input rows.
+int run_layers(tts_gpt *h, int R) {
+  const tts_gpt_config_t &c = h->cfg;
+  const int d = c.d_model;
+  cudaStream_t st = h->stream;
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW &L = h->layers[l];
+    uint16_t *kvl = h->kv + h->kv_layer_elems * l;
+    layernorm_kernel<<<R, kLnThreads, 0, st>>>(h->x, d, L.ln1_g, L.ln1_b, c.ln_eps, h->a, nullptr, nullptr, nullptr);
+    LinearArgs qa = linear_args(L.qkv, h->a, R, EPI_QKV);
+    qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
+    qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+    CUDA_TRY(h, launch_linear(c.wfmt, qa, st));
+    AttnArgs aa;
+    aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
+    aa.row_pos = h->rt.row_pos; aa.out = h->o; aa.partials = h->attn_partials; aa.tickets = h->attn_tickets;
+    aa.H = c.n_head; aa.pps = h->pps;
+    CUDA_TRY(h, launch_attention(aa, R, c.max_context, st));
+    LinearArgs oa = linear_args(L.o, h->o, R, EPI_RESID);
+    oa.out_f32 = h->x; oa.out_stride = d;
+    CUDA_TRY(h, launch_linear(c.wfmt, oa, st));
+    layernorm_kernel<<<R, kLnThreads, 0, st>>>(h->x, d, L.ln2_g, L.ln2_b, c.ln_eps, h->a, nullptr, nullptr, nullptr);
+    LinearArgs f1 = linear_args(L.fc1, h->a, R, EPI_GELU);
+    f1.out_bf16 = h->hbuf; f1.gelu_tanh = c.gelu_tanh;
+    CUDA_TRY(h, launch_linear(c.wfmt, f1, st));
+    LinearArgs f2 = linear_args(L.fc2, h->hbuf, R, EPI_RESID);
+    f2.out_f32 = h->x; f2.out_stride = d;
+    CUDA_TRY(h, launch_linear(c.wfmt, f2, st));
+  }
+  CUDA_TRY(h, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
+// Final LayerNorm (gathered to the wanted rows), LM head, sampling.
+int run_head(tts_gpt *h, int n_out) {
+  const tts_gpt_config_t &c = h->cfg;
+  cudaStream_t st = h->stream;
+  layernorm_kernel<<<n_out, kLnThreads, 0, st>>>(h->x, c.d_model, h->lnf_g, h->lnf_b, c.ln_eps, h->hf,
+                                                 h->rt.out_rows, h->rt.out_slot, h->io);
+  LinearArgs ha = linear_args(h->head, h->hf, n_out, EPI_F32);
+  ha.out_f32 = h->logits; ha.out_stride = c.vocab;
+  CUDA_TRY(h, launch_linear(WF_BF16, ha, st));
+  SampleArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.logits = h->logits; sa.V = c.vocab; sa.io = h->io; sa.out_slot = h->rt.out_slot; sa.out_rows = h->rt.out_rows;
+  sa.row_stream = h->rt.row_stream; sa.last_token = h->ps.last_token; sa.stop_flag = h->ps.stop_flag;
+  sa.stop_token = c.stop_token;
+  sample_kernel<<<n_out, kSampleThreads, (size_t)c.vocab * sizeof(float), st>>>(sa);
+  CUDA_TRY(h, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
+int run_embed(tts_gpt *h, int R) {
+  const tts_gpt_config_t &c = h->cfg;
+  embed_kernel<<<R, 256, 0, h->stream>>>(h->rt, h->tok_emb, h->pos_emb, c.d_model, c.vocab, c.max_pos, h->x);
+  CUDA_TRY(h, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
+int check_top_k(tts_gpt *h, int top_k, float temperature, const float *uniforms) {
+  if (top_k < 0 || top_k > kMaxTopK) return fail(h, TTS_GPT_E_ARG, "top_k must be in 0..%d", kMaxTopK);
+  if (top_k > 1 && !(temperature > 0.f)) return fail(h, TTS_GPT_E_ARG, "temperature must be positive");
+  if (top_k > 1 && !uniforms) return fail(h, TTS_GPT_E_ARG, "top-k sampling needs uniforms");
+  return TTS_GPT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t tts_gpt_query_workspace(const tts_gpt_config_t *cfg, size_t *bytes) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!bytes) return fail(nullptr, TTS_GPT_E_ARG, "null bytes");
+  tts_gpt tmp;
+  tmp.cfg = *cfg;
+  *bytes = carve(&tmp, nullptr);
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream, tts_gpt_t **out) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!w || !workspace || !out) return fail(nullptr, TTS_GPT_E_ARG, "null argument");
+  if ((uintptr_t)workspace % 256) return fail(nullptr, TTS_GPT_E_WORKSPACE, "workspace must be 256-byte aligned");
+  tts_gpt *h = new (std::nothrow) tts_gpt();
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "out of host memory");
+  h->cfg = *cfg;
+  h->stream = (cudaStream_t)cuda_stream;
+  const size_t need = carve(h, workspace);
+  if (need > workspace_bytes) {
+    delete h;
+    return fail(nullptr, TTS_GPT_E_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+  }
+  const tts_gpt_config_t &c = h->cfg;
+  const int d = c.d_model;
+#define TRY_(expr) do { rc = (expr); if (rc) { g_last_error = h->err; delete h; return rc; } } while (0)
+  TRY_(copy_bf16(h, h->tok_emb, w->tok_emb, (size_t)c.vocab * d, "tok_emb"));
+  TRY_(copy_bf16(h, h->pos_emb, w->pos_emb, (size_t)c.max_pos * d, "pos_emb"));
+  TRY_(copy_bf16(h, h->lnf_g, w->lnf_g, d, "lnf_g"));
+  TRY_(copy_bf16(h, h->lnf_b, w->lnf_b, d, "lnf_b"));
+  if (!w->head_w) { delete h; return fail(nullptr, TTS_GPT_E_ARG, "weights: head_w is null"); }
+  {
+    cudaError_t e = launch_pack(WF_BF16, h->head.N, h->head.K, w->head_w, nullptr, h->head.w, nullptr, h->stream);
+    if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "pack head: %s", cudaGetErrorString(e)); }
+    if (w->head_b) {
+      TRY_(copy_bf16(h, h->head.bias, w->head_b, c.vocab, "head_b"));
+    } else {
+      h->head.bias = nullptr;
+    }
+  }
+  const void *const *per_layer[] = {w->ln1_g, w->ln1_b, w->ln2_g, w->ln2_b, w->qkv_w, w->qkv_b, w->o_w, w->o_b,
+                                    w->fc1_w, w->fc1_b, w->fc2_w, w->fc2_b};
+  for (auto p : per_layer)
+    if (!p) { delete h; return fail(nullptr, TTS_GPT_E_ARG, "weights: a per-layer pointer array is null"); }
+  if (c.wfmt != WF_BF16 && (!w->qkv_s || !w->o_s || !w->fc1_s || !w->fc2_s)) {
+    delete h;
+    return fail(nullptr, TTS_GPT_E_ARG, "weights: scale arrays are required for quantized formats");
+  }
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW &L = h->layers[l];
+    TRY_(copy_bf16(h, L.ln1_g, w->ln1_g[l], d, "ln1_g"));
+    TRY_(copy_bf16(h, L.ln1_b, w->ln1_b[l], d, "ln1_b"));
+    TRY_(copy_bf16(h, L.ln2_g, w->ln2_g[l], d, "ln2_g"));
+    TRY_(copy_bf16(h, L.ln2_b, w->ln2_b[l], d, "ln2_b"));
+    const bool qz = c.wfmt != WF_BF16;
+    TRY_(load_linear(h, L.qkv, c.wfmt, w->qkv_w[l], qz ? w->qkv_s[l] : nullptr, w->qkv_b[l], "qkv"));
+    TRY_(load_linear(h, L.o, c.wfmt, w->o_w[l], qz ? w->o_s[l] : nullptr, w->o_b[l], "o"));
+    TRY_(load_linear(h, L.fc1, c.wfmt, w->fc1_w[l], qz ? w->fc1_s[l] : nullptr, w->fc1_b[l], "fc1"));
+    TRY_(load_linear(h, L.fc2, c.wfmt, w->fc2_w[l], qz ? w->fc2_s[l] : nullptr, w->fc2_b[l], "fc2"));
+  }
+#undef TRY_
+  const int init_n = std::max(std::max(c.n_pages, c.max_streams * h->pps), c.max_streams);
+  init_pages_kernel<<<(init_n + 255) / 256, 256, 0, h->stream>>>(h->ps);
+  cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)kMaxRows * c.n_head * sizeof(unsigned int), h->stream);
+  if (e == cudaSuccess) e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+  if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(e)); }
+  h->open.assign(c.max_streams, 0);
+  h->ctx.assign(c.max_streams, 0);
+  h->pos_next.assign(c.max_streams, 0);
+  h->n_free = c.n_pages;
+  const char *ng = getenv("TTS_GPT_NO_GRAPH");
+  // the legacy default stream cannot be captured
+  h->use_graph = !(ng && ng[0] == '1') && h->stream != nullptr && h->stream != cudaStreamLegacy;
+  *out = h;
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, const int32_t *prefix_len,
+                        const int32_t *pos0, int32_t top_k, float temperature, const float *uniforms,
+                        int32_t *out_stream_ids, int32_t *out_tokens, float *out_logits, void *out_hidden) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  const tts_gpt_config_t &c = h->cfg;
+  if (n < 1 || n > c.max_streams || !prefix_emb || !prefix_len || !out_stream_ids || !out_tokens)
+    return fail(h, TTS_GPT_E_ARG, "prefill: bad n or null argument");
+  int rc = check_top_k(h, top_k, temperature, uniforms);
+  if (rc) return rc;
+  int pages = 0;
+  for (int i = 0; i < n; ++i) {
+    if (prefix_len[i] < 1 || !prefix_emb[i]) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has an empty prefix", i);
+    if (prefix_len[i] > c.max_context) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "prefill: prefix %d exceeds max_context %d", prefix_len[i], c.max_context);
+    if (pos0 && (pos0[i] < 0 || pos0[i] >= c.max_pos)) return fail(h, TTS_GPT_E_ARG, "prefill: pos0 out of range");
+    pages += (prefix_len[i] + 63) / 64;
+  }
+  PrefillParams pp;
+  memset(&pp, 0, sizeof pp);
+  pp.n = n;
+  int found = 0;
+  for (int s = 0; s < c.max_streams && found < n; ++s)
+    if (!h->open[s]) pp.stream_ids[found++] = s;
+  if (found < n) return fail(h, TTS_GPT_E_STREAM, "prefill: %d free stream slots, %d needed", found, n);
+  if (pages > h->n_free) return fail(h, TTS_GPT_E_NO_PAGES, "prefill: %d pages needed, %d free", pages, h->n_free);
+  for (int i = 0; i < n; ++i) {
+    pp.prefix_len[i] = prefix_len[i];
+    pp.pos0[i] = pos0 ? pos0[i] : 0;
+    pp.emb[i] = (const uint16_t *)prefix_emb[i];
+  }
+  prefill_open_kernel<<<1, kMaxRows, 0, h->stream>>>(pp, h->ps);
+  CUDA_TRY(h, cudaGetLastError());
+  for (int i = 0; i < n; ++i) {
+    const int s = pp.stream_ids[i];
+    h->open[s] = 1; h->ctx[s] = prefix_len[i]; h->pos_next[s] = pp.pos0[i];
+    out_stream_ids[i] = s;
+  }
+  h->n_free -= pages;
+
+  StepIO io;
+  io.in_tokens = nullptr; io.uniforms = uniforms; io.out_tokens = out_tokens; io.out_logits = out_logits;
+  io.out_hidden = (uint16_t *)out_hidden; io.top_k = top_k; io.temperature = temperature; io.n_out = 0;
+  // rows in stream-major order, 128 per pass
+  PassParams ps;
+  memset(&ps, 0, sizeof ps);
+  ps.io = io;
+  auto flush = [&]() -> int {
+    if (ps.n_rows == 0) return TTS_GPT_OK;
+    ps.io.n_out = ps.n_out;
+    prefill_pass_kernel<<<1, kMaxRows, 0, h->stream>>>(ps, h->ps, h->rt, h->io, c.d_model);
+    CUDA_TRY(h, cudaGetLastError());
+    int r = run_embed(h, ps.n_rows);
+    if (r) return r;
+    r = run_layers(h, ps.n_rows);
+    if (r) return r;
+    if (ps.n_out > 0) r = run_head(h, ps.n_out);
+    ps.n_rows = 0; ps.n_out = 0;
+    return r;
+  };
+  for (int i = 0; i < n; ++i) {
+    for (int t = 0; t < prefix_len[i]; ++t) {
+      const int r = ps.n_rows++;
+      ps.row_stream[r] = (short)pp.stream_ids[i];
+      ps.row_pos[r] = (short)t;
+      if (t == prefix_len[i] - 1) {
+        ps.out_rows[ps.n_out] = (short)r;
+        ps.out_slot[ps.n_out] = (short)i;
+        ++ps.n_out;
+      }
+      if (ps.n_rows == kMaxRows) { rc = flush(); if (rc) return rc; }
+    }
+  }
+  return flush();
+}
+
+int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, const int32_t *in_tokens,
+                            int32_t top_k, float temperature, const float *uniforms, int32_t *out_tokens,
+                            float *out_logits, void *out_hidden) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  const tts_gpt_config_t &c = h->cfg;
+  if (n < 1 || n > c.max_streams || !stream_ids || !out_tokens) return fail(h, TTS_GPT_E_ARG, "decode_step: bad n or null argument");
+  int rc = check_top_k(h, top_k, temperature, uniforms);
+  if (rc) return rc;
+  int pages = 0;
+  char seen[kMaxRows];
+  memset(seen, 0, sizeof seen);
+  for (int i = 0; i < n; ++i) {
+    const int s = stream_ids[i];
+    if (s < 0 || s >= c.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "decode_step: stream %d is not open", s);
+    if (seen[s]) return fail(h, TTS_GPT_E_STREAM, "decode_step: stream %d listed twice", s);
+    seen[s] = 1;
+    if (h->ctx[s] + 1 > c.max_context) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "decode_step: stream %d is at max_context %d", s, c.max_context);
+    if (h->pos_next[s] >= c.max_pos) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "decode_step: stream %d ran past max_pos %d", s, c.max_pos);
+    if (h->ctx[s] % 64 == 0) ++pages;
+  }
+  if (pages > h->n_free) return fail(h, TTS_GPT_E_NO_PAGES, "decode_step: %d pages needed, %d free", pages, h->n_free);
+
+  StepParams sp;
+  sp.n = n;
+  memcpy(sp.stream_ids, stream_ids, (size_t)n * sizeof(int));
+  sp.io.in_tokens = in_tokens; sp.io.uniforms = uniforms; sp.io.out_tokens = out_tokens; sp.io.out_logits = out_logits;
+  sp.io.out_hidden = (uint16_t *)out_hidden; sp.io.top_k = top_k; sp.io.temperature = temperature; sp.io.n_out = n;
+  step_setup_kernel<<<1, kMaxRows, 0, h->stream>>>(sp, h->ps, h->rt, h->io);
+  CUDA_TRY(h, cudaGetLastError());
+  for (int i = 0; i < n; ++i) { h->ctx[stream_ids[i]] += 1; h->pos_next[stream_ids[i]] += 1; }
+  h->n_free -= pages;
+
+  if (h->use_graph) {
+    auto it = h->graphs.find(n);
+    if (it == h->graphs.end()) {
+      cudaGraph_t g = nullptr;
+      CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      rc = run_embed(h, n);
+      if (!rc) rc = run_layers(h, n);
+      if (!rc) rc = run_head(h, n);
+      cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+      if (rc) { if (g) cudaGraphDestroy(g); return rc; }
+      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph capture: %s", cudaGetErrorString(e));
+      cudaGraphExec_t ge = nullptr;
+      e = cudaGraphInstantiate(&ge, g, 0);
+      cudaGraphDestroy(g);
+      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
+      it = h->graphs.emplace(n, ge).first;
+    }
+    CUDA_TRY(h, cudaGraphLaunch(it->second, h->stream));
+    return TTS_GPT_OK;
+  }
+  rc = run_embed(h, n);
+  if (!rc) rc = run_layers(h, n);
+  if (!rc) rc = run_head(h, n);
+  return rc;
+}
+
+int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  if (s < 0 || s >= h->cfg.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "release_stream: stream %d is not open", s);
+  release_kernel<<<1, 32, 0, h->stream>>>(h->ps, s);
+  CUDA_TRY(h, cudaGetLastError());
+  h->n_free += (h->ctx[s] + 63) / 64;
+  h->open[s] = 0; h->ctx[s] = 0;
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_sync(tts_gpt_t *h) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_destroy(tts_gpt_t *h) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  cudaStreamSynchronize(h->stream);
+  for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second);
+  delete h;
+  return TTS_GPT_OK;
+}
+
+const char *tts_gpt_last_error(const tts_gpt_t *h) { return h ? h->err.c_str() : g_last_error.c_str(); }
+
+int32_t tts_gpt_stats(const tts_gpt_t *h, int32_t *open_streams, int32_t *free_pages) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  if (open_streams) { int n = 0; for (char o : h->open) n += o; *open_streams = n; }
+  if (free_pages) *free_pages = h->n_free;
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t s) {
+  if (!h || s < 0 || s >= h->cfg.max_streams || !h->open[s]) return -1;
+  return h->ctx[s];
+}
+
+int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  for (char o : h->open) if (o) return fail(h, TTS_GPT_E_STREAM, "shuffle: streams are open");
+  std::vector<int> perm(h->cfg.n_pages);
+  for (int i = 0; i < h->cfg.n_pages; ++i) perm[i] = i;
+  uint64_t x = 0x9E3779B97F4A7C15ull ^ seed;
+  for (int i = h->cfg.n_pages - 1; i > 0; --i) {
+    x = x * 6364136223846793005ull + 1442695040888963407ull;
+    const int j = (int)((x >> 33) % (uint64_t)(i + 1));
+    std::swap(perm[i], perm[j]);
+  }
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  CUDA_TRY(h, cudaMemcpy(h->ps.free_list, perm.data(), perm.size() * sizeof(int), cudaMemcpyHostToDevice));
+  return TTS_GPT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// single-kernel entry points
+// ---------------------------------------------------------------------------------------------
+int32_t tts_gpt_op_linear_packed_bytes(int32_t wfmt, int32_t N, int32_t K, size_t *bytes) {
+  if (wfmt < 0 || wfmt > 2 || N < 1 || K < 128 || K % 128 || !bytes) return fail(nullptr, TTS_GPT_E_ARG, "op_linear: bad shape");
+  *bytes = align256(packed_weight_bytes(wfmt, N, K)) + align256(packed_scale_bytes(wfmt, N, K));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_linear_pack(int32_t wfmt, int32_t N, int32_t K, const void *w, const void *s, void *packed,
+                               void *cuda_stream) {
+  size_t bytes;
+  int rc = tts_gpt_op_linear_packed_bytes(wfmt, N, K, &bytes);
+  if (rc) return rc;
+  if (!w || !packed || (wfmt != WF_BF16 && !s) || (uintptr_t)packed % 256) return fail(nullptr, TTS_GPT_E_ARG, "op_linear_pack: null or misaligned");
+  char *ps = (char *)packed + align256(packed_weight_bytes(wfmt, N, K));
+  CUDA_TRY(nullptr, launch_pack(wfmt, N, K, w, s, packed, ps, (cudaStream_t)cuda_stream));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed, const void *bias, int32_t B,
+                          const void *act, float *out, void *cuda_stream) {
+  size_t bytes;
+  int rc = tts_gpt_op_linear_packed_bytes(wfmt, N, K, &bytes);
+  if (rc) return rc;
+  if (!packed || !act || !out || B < 1 || B > kMaxRows) return fail(nullptr, TTS_GPT_E_ARG, "op_linear: bad argument");
+  PackedLinear pl;
+  pl.N = N; pl.K = K; pl.w = (void *)packed;
+  pl.s = (uint16_t *)((char *)packed + align256(packed_weight_bytes(wfmt, N, K)));
+  pl.bias = (uint16_t *)bias;
+  LinearArgs a = linear_args(pl, (const uint16_t *)act, B, EPI_F32);
+  a.out_f32 = out; a.out_stride = N;
+  CUDA_TRY(nullptr, launch_linear(wfmt, a, (cudaStream_t)cuda_stream));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_attention_scratch_bytes(int32_t R, int32_t n_head, size_t *bytes) {
+  if (R < 1 || n_head < 1 || !bytes) return fail(nullptr, TTS_GPT_E_ARG, "op_attention: bad shape");
+  *bytes = attention_scratch_bytes(R, n_head);
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                             const int32_t *page_table, int32_t pages_per_stream, const int32_t *row_stream,
+                             const int32_t *row_pos, void *out, void *scratch, void *cuda_stream) {
+  if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out || !scratch ||
+      pages_per_stream < 1 || pages_per_stream > kAttnMaxChunks * kAttnWarps || (uintptr_t)scratch % 256)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention: bad argument");
+  AttnArgs a;
+  a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
+  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  a.partials = (float *)scratch;
+  a.tickets = (unsigned int *)((char *)scratch + align256((size_t)R * n_head * kAttnMaxChunks * kAttnPartialFloats * sizeof(float)));
+  CUDA_TRY(nullptr, launch_attention(a, R, pages_per_stream * kPageTokens, (cudaStream_t)cuda_stream));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_layernorm(int32_t R, int32_t d, const float *x, const void *g, const void *b, float eps,
+                             void *out, void *cuda_stream) {
+  if (R < 1 || d < 1 || d > kLnThreads * kLnMaxPerThread || !x || !g || !b || !out) return fail(nullptr, TTS_GPT_E_ARG, "op_layernorm: bad argument");
+  layernorm_kernel<<<R, kLnThreads, 0, (cudaStream_t)cuda_stream>>>(x, d, (const uint16_t *)g, (const uint16_t *)b, eps,
+                                                                    (uint16_t *)out, nullptr, nullptr, nullptr);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_sample(int32_t R, int32_t V, const float *logits, int32_t top_k, float temperature,
+                          const float *uniforms, int32_t *tokens, void *cuda_stream) {
+  if (R < 1 || V < 2 || V > kSampleThreads * kSampleMaxPer || !logits || !tokens || top_k < 0 || top_k > kMaxTopK ||
+      (top_k > 1 && (!uniforms || !(temperature > 0.f))))
+    return fail(nullptr, TTS_GPT_E_ARG, "op_sample: bad argument");
+  SampleArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.logits = logits; sa.V = V; sa.top_k = top_k; sa.temperature = temperature; sa.uniforms = uniforms; sa.out_tokens = tokens;
+  sample_kernel<<<R, kSampleThreads, (size_t)V * sizeof(float), (cudaStream_t)cuda_stream>>>(sa);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,244 @@
+"""End-to-end parity of prefill + decode_step through the C ABI on the tiny workload (and small
+variants): per-step comparison with the fp64 oracle on identical history (replay and teacher-forced),
+all three weight formats, top-k, batching invariants, paging edge cases and error behaviour."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gpt_oracle as O
+from paper_2607_21042_b200 import binding as B
+from paper_2607_21042_b200 import cases as C
+from helpers import (assert_logits_close, bits_dev, check_tokens, gpu_run_stream)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _tiny(wfmt=C.W_BF16, **kw):
+    base = dict(wfmt=wfmt, max_streams=4, n_pages=4 * 32)
+    base.update(kw)
+    return C.tiny_config(**base)
+
+
+@pytest.fixture(scope="module")
+def tiny_models():
+    out = {}
+    for wfmt in (C.W_BF16, C.W_INT8_PC, C.W_INT4_G128):
+        cfg = _tiny(wfmt)
+        w = C.make_weights(cfg, seed=0)
+        out[wfmt] = (cfg, w, O.OracleModel(cfg, w))
+    return out
+
+
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
+def test_workload1_replay_and_teacher_forced(tiny_models, wfmt):
+    cfg, w, model = tiny_models[wfmt]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [64], seed=0)[0]
+    n = 32
+    # replay: the GPU runs free, the oracle is fed the GPU's tokens
+    toks, logits, hidden, sid = gpu_run_stream(eng, bits_dev(prefix), n, want_hidden=True)
+    ref_logits, ref_hidden = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref_logits, "replay")
+    check_tokens(toks, ref_logits, 0, 1.0, None, "replay")
+    hid = O.bf16_to_f64(hidden)
+    assert np.max(np.abs(hid - ref_hidden)) <= 2e-2 * max(1.0, np.abs(ref_hidden).max())
+    assert eng.stream_context(sid) == 64 + n
+    eng.release_stream(sid)
+    # teacher-forced: the oracle runs free, the GPU is fed the oracle's tokens
+    run = O.run_stream(model, O.bf16_to_f64(prefix), n)
+    forced = torch.from_numpy(run["tokens"][:-1].astype(np.int32)).to(DEV)
+    toks2, logits2, _, sid2 = gpu_run_stream(eng, bits_dev(prefix), n, forced_tokens=forced)
+    assert_logits_close(logits2, run["logits"], "teacher-forced")
+    check_tokens(toks2, run["logits"], 0, 1.0, None, "teacher-forced")
+    # first free-running divergence, if any, falls on an excused step
+    diff = np.nonzero(toks != run["tokens"])[0]
+    if len(diff):
+        assert O.top2_gap(run["logits"][diff[0]]) < 3e-2
+    eng.destroy()
+
+
+def test_topk_sampling_replay(tiny_models):
+    cfg, w, model = tiny_models[C.W_INT8_PC]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [40], seed=3)[0]
+    n = 48
+    u = C.make_uniforms(n + 1, 1, seed=3)[:, 0]
+    toks, logits, _, sid = gpu_run_stream(eng, bits_dev(prefix), n, top_k=30, temperature=1.0,
+                                          uniforms_dev=torch.from_numpy(u).to(DEV))
+    ref_logits, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref_logits, "top-k replay")
+    check_tokens(toks, ref_logits, 30, 1.0, u, "top-k replay")
+    assert len(set(toks.tolist())) > 5         # it does sample, not arg-max
+    eng.destroy()
+
+
+def _run_batch(eng, prefixes, n_steps, shuffle_seed=None):
+    """Prefill all prefixes in one call, decode n_steps with the whole batch; returns per-stream
+    logits [S, n_steps+1, V] and tokens."""
+    S = len(prefixes)
+    V = eng.cfg.vocab
+    if shuffle_seed is not None:
+        eng.debug_shuffle_free_pages(shuffle_seed)
+    toks = torch.zeros((n_steps + 1, S), dtype=torch.int32, device=DEV)
+    logits = torch.zeros((n_steps + 1, S, V), dtype=torch.float32, device=DEV)
+    ids, _ = eng.prefill([bits_dev(p) for p in prefixes], out_tokens=toks[0], out_logits=logits[0])
+    for k in range(1, n_steps + 1):
+        eng.decode_step(ids, toks[k], out_logits=logits[k])
+    eng.sync()
+    for s in ids:
+        eng.release_stream(s)
+    return logits.cpu().numpy().transpose(1, 0, 2), toks.cpu().numpy().T
+
+
+def test_batch_invariance_page_permutation_and_reuse(tiny_models):
+    cfg, w, model = tiny_models[C.W_BF16]
+    eng = B.TtsGpt(cfg, w, DEV)
+    lens = [63, 64, 65, 130]          # around the page edge; decode crosses more edges
+    prefixes = C.make_prefixes(cfg, lens, seed=5)
+    n = 70
+    lg_batch, tk_batch = _run_batch(eng, prefixes, n)
+    assert eng.stats() == {"open_streams": 0, "free_pages": cfg.n_pages}
+    # each stream alone gives the same numbers as inside the batch
+    for s in range(4):
+        lg_one, tk_one = _run_batch(eng, [prefixes[s]], n)
+        assert np.array_equal(tk_one[0], tk_batch[s])
+        assert np.array_equal(lg_one[0], lg_batch[s]), "batch of 4 vs alone, stream %d" % s
+    # physical page placement does not matter: bit-identical after shuffling the free list
+    lg_shuf, tk_shuf = _run_batch(eng, prefixes, n, shuffle_seed=123)
+    assert np.array_equal(lg_shuf, lg_batch) and np.array_equal(tk_shuf, tk_batch)
+    # release + re-prefill (done above, repeatedly) reproduces the first run
+    lg_again, _ = _run_batch(eng, prefixes, n)
+    assert np.array_equal(lg_again, lg_batch)
+    # and the batch agrees with the oracle (replay), stream by stream
+    for s in range(4):
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk_batch[s][:-1])
+        assert_logits_close(lg_batch[s], ref, "batch stream %d" % s)
+        check_tokens(tk_batch[s], ref, 0, 1.0, None, "batch stream %d" % s)
+    eng.destroy()
+
+
+def test_prefix_of_one_row_and_pos0(tiny_models):
+    cfg, w, model = tiny_models[C.W_INT4_G128]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [1], seed=8)[0]
+    toks, logits, _, sid = gpu_run_stream(eng, bits_dev(prefix), 5, pos0=7)
+    ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1], pos0=7)
+    assert_logits_close(logits, ref, "P=1, pos0=7")
+    ref0, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1], pos0=0)
+    assert np.max(np.abs(ref0[1:] - ref[1:])) > 1e-3          # the position offset does matter
+    eng.destroy()
+
+
+def test_ragged_batch_with_streams_leaving(tiny_models):
+    """Streams of different lengths decode together; one leaves mid-way, a new one joins."""
+    cfg, w, model = tiny_models[C.W_INT8_PC]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefixes = C.make_prefixes(cfg, [10, 100, 33, 70], seed=9)
+    V = cfg.vocab
+    steps = 12
+    toks = torch.zeros((steps + 1, 4), dtype=torch.int32, device=DEV)
+    logits = torch.zeros((steps + 1, 4, V), dtype=torch.float32, device=DEV)
+    ids, _ = eng.prefill([bits_dev(p) for p in prefixes[:3]], out_tokens=toks[0, :3], out_logits=logits[0, :3])
+    active = list(ids)
+    col = {s: i for i, s in enumerate(ids)}
+    hist = {s: [] for s in ids}
+    late_id = None
+    for k in range(1, steps + 1):
+        if k == 5:
+            eng.release_stream(active.pop(1))              # the 100-row stream leaves
+            (late_id,), _ = eng.prefill([bits_dev(prefixes[3])], out_tokens=toks[k - 1, 3:4],
+                                        out_logits=logits[k - 1, 3:4])
+            active.append(late_id); col[late_id] = 3; hist[late_id] = []
+        cols = [col[s] for s in active]
+        ot = torch.zeros(len(active), dtype=torch.int32, device=DEV)
+        ol = torch.zeros((len(active), V), dtype=torch.float32, device=DEV)
+        eng.wait_for_caller()
+        eng.decode_step(active, ot, out_logits=ol)
+        eng.sync()
+        for j, s in enumerate(active):
+            hist[s].append((int(ot[j]), ol[j].cpu().numpy()))
+    eng.sync()
+    first = {ids[0]: (0, 0), ids[1]: (0, 1), ids[2]: (0, 2), late_id: (4, 3)}
+    for s, (k0, c) in first.items():
+        y0 = int(toks[k0, c]); l0 = logits[k0, c].cpu().numpy()
+        seq = [y0] + [t for t, _ in hist[s]]
+        lg = np.stack([l0] + [l for _, l in hist[s]])
+        p = prefixes[c]
+        ref, _ = O.replay_full(model, O.bf16_to_f64(p), seq[:-1])
+        assert_logits_close(lg, ref, "ragged stream col %d" % c)
+        check_tokens(seq, ref, 0, 1.0, None, "ragged stream col %d" % c)
+    eng.destroy()
+
+
+def test_error_behaviour_leaves_state_untouched(tiny_models):
+    cfg0, w, _ = tiny_models[C.W_BF16]
+    cfg = _tiny(C.W_BF16, max_streams=2, max_context=128, n_pages=3)
+    eng = B.TtsGpt(cfg, w, DEV)
+    p = C.make_prefixes(cfg, [127, 70, 129, 1], seed=1)
+    out = torch.zeros(2, dtype=torch.int32, device=DEV)
+    torch.cuda.synchronize()
+
+    def code(fn):
+        with pytest.raises(B.TtsGptError) as e:
+            fn()
+        return e.value.code
+
+    assert code(lambda: eng.prefill([bits_dev(p[2])])) == B.E_CTX_OVERFLOW          # 129 > 128
+    assert code(lambda: eng.prefill([bits_dev(p[0]), bits_dev(p[1])])) == B.E_NO_PAGES   # 2 + 2 > 3
+    assert eng.stats() == {"open_streams": 0, "free_pages": 3}
+    (a,), _ = eng.prefill([bits_dev(p[0])])                                          # 2 pages
+    assert eng.stats() == {"open_streams": 1, "free_pages": 1}
+    assert code(lambda: eng.decode_step([a, a], out)) == B.E_STREAM                  # duplicate
+    assert code(lambda: eng.decode_step([1 - a], out)) == B.E_STREAM                 # not open
+    assert code(lambda: eng.decode_step([], out)) == B.E_ARG
+    assert code(lambda: eng.decode_step([a], out, top_k=30)) == B.E_ARG              # no uniforms
+    eng.decode_step([a], out)                                                        # ctx 127 -> 128: allowed
+    assert eng.stream_context(a) == 128
+    assert code(lambda: eng.decode_step([a], out)) == B.E_CTX_OVERFLOW               # 129
+    assert eng.stream_context(a) == 128
+    (b,), _ = eng.prefill([bits_dev(p[3])])                                          # last page
+    assert eng.stats() == {"open_streams": 2, "free_pages": 0}
+    assert code(lambda: eng.prefill([bits_dev(p[3])])) == B.E_STREAM                 # no slot
+    eng.release_stream(a)
+    assert code(lambda: eng.release_stream(a)) == B.E_STREAM                         # double release
+    assert eng.stats() == {"open_streams": 1, "free_pages": 2}
+    for _ in range(63):
+        eng.decode_step([b], out)                                                    # fills page 0 of b
+    (c,), _ = eng.prefill([bits_dev(p[1])])                                          # takes the 2 free pages
+    assert code(lambda: eng.decode_step([b], out)) == B.E_NO_PAGES                   # b needs a new page
+    assert eng.stream_context(b) == 64
+    eng.release_stream(c)
+    eng.decode_step([b], out)
+    eng.sync()
+    assert "pages" in eng.last_error() or eng.last_error() != ""
+    eng.destroy()
+
+
+def test_context_exactly_max_and_oracle_agreement():
+    cfg = _tiny(C.W_BF16, max_streams=1, max_context=256, n_pages=4, max_pos=256)
+    w = C.make_weights(cfg, seed=2)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [200], seed=2)[0]
+    toks, logits, _, sid = gpu_run_stream(eng, bits_dev(prefix), 56)          # 200 + 56 = 256
+    assert eng.stream_context(sid) == 256
+    ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref, "full context")
+    with pytest.raises(B.TtsGptError):
+        eng.decode_step([sid], torch.zeros(1, dtype=torch.int32, device=DEV))
+    eng.destroy()
+
+
+def test_erf_gelu_variant():
+    cfg = _tiny(C.W_BF16, gelu_tanh=0, max_streams=1, n_pages=8)
+    w = C.make_weights(cfg, seed=4)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [20], seed=4)[0]
+    toks, logits, _, _ = gpu_run_stream(eng, bits_dev(prefix), 8)
+    ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref, "erf gelu")
+    eng.destroy()

@@ -1,0 +1,212 @@
+"""Single-kernel parity through the C ABI: dequantizing linear, paged decode attention, LayerNorm,
+sampling — each against the fp64 oracle on seeded inputs spanning several tiles and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gpt_oracle as O
+from paper_2607_21042_b200 import binding as B
+from paper_2607_21042_b200 import cases as C
+from helpers import bits_dev, bits_to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _rand_bf16(rng, shape, std):
+    return C.f32_to_bf16_bits((rng.standard_normal(size=shape) * std).astype(np.float32))
+
+
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
+@pytest.mark.parametrize("N,K,Bn", [(48, 256, 1), (50, 384, 3), (1280, 1280, 8), (130, 1024, 16),
+                                    (64, 5120, 9), (258, 256, 37), (8194, 1280, 2), (96, 128, 128)])
+def test_linear_matches_oracle(wfmt, N, K, Bn):
+    rng = np.random.default_rng(N * 7 + K + Bn + wfmt)
+    wb = _rand_bf16(rng, (N, K), 0.02)
+    if wfmt == C.W_BF16:
+        w, s = wb, None
+    elif wfmt == C.W_INT8_PC:
+        w, s = C.quantize_int8_per_channel(wb)
+    else:
+        w, s = C.quantize_int4_group128(wb)
+    bias = _rand_bf16(rng, (N,), 0.02)
+    act = _rand_bf16(rng, (Bn, K), 1.0)
+    ref = O.bf16_to_f64(act) @ O.dequant(wfmt, w, s).T + O.bf16_to_f64(bias)
+    packed, n_, k_ = B.op_linear_pack(wfmt, bits_dev(w), None if s is None else bits_dev(s))
+    assert (n_, k_) == (N, K)
+    out = B.op_linear(wfmt, packed, N, K, bits_dev(act), bits_dev(bias))
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    # exact products, fp32 accumulation: error ~ sqrt(K) * 2^-24 * |terms|; allow 2e-5 of the scale
+    scale = np.abs(ref).max()
+    assert np.max(np.abs(got - ref)) <= 2e-5 * scale + 1e-6
+    # no bias
+    out = B.op_linear(wfmt, packed, N, K, bits_dev(act), None)
+    got = out.cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(got - (ref - O.bf16_to_f64(bias)))) <= 2e-5 * scale + 1e-6
+
+
+def test_linear_int4_extreme_codes_and_group_scales():
+    # every nibble value at every position of a word, groups with different scales
+    N, K = 16, 256
+    u = np.zeros((N, K), dtype=np.int64)
+    for n in range(N):
+        u[n] = (np.arange(K) * (n + 1) + n) % 16
+    words = C.pack_int4_words(u)
+    sc = C.f32_to_bf16_bits(np.array([[0.5, 2.0]] * N, np.float32) * (1 + np.arange(N))[:, None].astype(np.float32))
+    act = C.f32_to_bf16_bits(np.eye(8, K, dtype=np.float32) * 1.0 + np.eye(8, K, k=128, dtype=np.float32) * 3.0)
+    ref = O.bf16_to_f64(act) @ O.dequant_int4_g128(words, sc).T
+    packed, _, _ = B.op_linear_pack(C.W_INT4_G128, bits_dev(words), bits_dev(sc))
+    got = B.op_linear(C.W_INT4_G128, packed, N, K, bits_dev(act)).cpu().numpy()
+    assert np.array_equal(got.astype(np.float64), ref)       # small integers times powers of two: exact
+
+
+def test_linear_int8_extreme_codes_exact():
+    N, K = 32, 128
+    q = np.zeros((N, K), dtype=np.int8)
+    vals = np.array([-127, 127, -1, 0, 1, 64, -64, 100], dtype=np.int8)
+    for n in range(N):
+        q[n] = np.roll(np.tile(vals, K // 8), n)
+    s = C.f32_to_bf16_bits(np.full(N, 0.25, np.float32))
+    act = C.f32_to_bf16_bits(np.eye(5, K, dtype=np.float32))
+    ref = O.bf16_to_f64(act) @ O.dequant_int8_pc(q, s).T
+    packed, _, _ = B.op_linear_pack(C.W_INT8_PC, bits_dev(q), bits_dev(s))
+    got = B.op_linear(C.W_INT8_PC, packed, N, K, bits_dev(act)).cpu().numpy()
+    assert np.array_equal(got.astype(np.float64), ref)
+
+
+def _attention_case(rng, H, ctxs, n_pages, pps, shuffle=True):
+    """Random paged KV for streams with ctxs[i] tokens (the row attends over all of them)."""
+    S = len(ctxs)
+    kv = np.zeros((n_pages, 2, H, 64, 64), dtype=np.uint16)
+    perm = rng.permutation(n_pages) if shuffle else np.arange(n_pages)
+    page_table = np.zeros((S, pps), dtype=np.int32)
+    Ks, Vs = [], []
+    nxt = 0
+    for s, n in enumerate(ctxs):
+        Kb = _rand_bf16(rng, (n, H, 64), 1.0)
+        Vb = _rand_bf16(rng, (n, H, 64), 1.0)
+        Ks.append(Kb); Vs.append(Vb)
+        for p in range((n + 63) // 64):
+            phys = perm[nxt]; nxt += 1
+            page_table[s, p] = phys
+            m = min(64, n - 64 * p)
+            kv[phys, 0, :, :m, :] = Kb[64 * p:64 * p + m].transpose(1, 0, 2)
+            kv[phys, 1, :, :m, :] = Vb[64 * p:64 * p + m].transpose(1, 0, 2)
+            # poison the unused tail of the page: must never be read into the result
+            kv[phys, :, :, m:, :] = 0x7FC0
+    return kv, page_table, Ks, Vs
+
+
+def _attention_ref(q, K, V, H):
+    o = np.empty(H * 64)
+    Kf, Vf = O.bf16_to_f64(K), O.bf16_to_f64(V)
+    for h in range(H):
+        s = Kf[:, h, :] @ q[h * 64:(h + 1) * 64] / 8.0
+        o[h * 64:(h + 1) * 64] = O.softmax(s) @ Vf[:, h, :]
+    return o
+
+
+@pytest.mark.parametrize("H,ctxs", [(4, [1]), (4, [63, 64, 65]), (2, [256, 257, 1000]), (20, [900]),
+                                    (3, [2048, 1, 511, 513, 1025])])
+def test_attention_matches_oracle(H, ctxs):
+    rng = np.random.default_rng(sum(ctxs) + H)
+    pps = 32
+    n_pages = sum((c + 63) // 64 for c in ctxs) + 3
+    kv, pt, Ks, Vs = _attention_case(rng, H, ctxs, n_pages, pps)
+    R = len(ctxs)
+    q = (rng.standard_normal(size=(R, H * 64)) * 2.0).astype(np.float32)
+    row_stream = np.arange(R, dtype=np.int32)
+    row_pos = np.array([c - 1 for c in ctxs], dtype=np.int32)
+    scratch = B.op_attention_scratch(R, H, DEV)
+    for rep in range(2):          # second call reuses the scratch the first one left behind
+        out = B.op_attention(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                             torch.from_numpy(row_stream).to(DEV), torch.from_numpy(row_pos).to(DEV), scratch)
+        torch.cuda.synchronize()
+        got = bits_to_f64(out)
+        for r in range(R):
+            ref = _attention_ref(q[r].astype(np.float64), Ks[r], Vs[r], H)
+            # bf16 output: half an ulp is 2^-9 relative; fp32 softmax adds ~1e-6
+            assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (r, rep)
+
+
+def test_attention_rows_of_one_stream_share_pages():
+    # several rows of the same stream at different positions (a prefill pass)
+    rng = np.random.default_rng(77)
+    H, n = 4, 200
+    kv, pt, Ks, Vs = _attention_case(rng, H, [n], 6, 32)
+    pos = np.array([0, 1, 63, 64, 130, 199], dtype=np.int32)
+    R = len(pos)
+    q = rng.standard_normal(size=(R, H * 64)).astype(np.float32)
+    out = B.op_attention(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                         torch.zeros(R, dtype=torch.int32, device=DEV), torch.from_numpy(pos).to(DEV))
+    got = bits_to_f64(out)
+    for r in range(R):
+        ref = _attention_ref(q[r].astype(np.float64), Ks[0][:pos[r] + 1], Vs[0][:pos[r] + 1], H)
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5
+
+
+@pytest.mark.parametrize("R,d", [(1, 256), (5, 1280), (128, 1280), (3, 2048), (2, 128)])
+def test_layernorm_matches_oracle(R, d):
+    rng = np.random.default_rng(R + d)
+    x = (rng.standard_normal(size=(R, d)) * 3 + 0.5).astype(np.float32)
+    g = _rand_bf16(rng, (d,), 0.1) ; b = _rand_bf16(rng, (d,), 0.1)
+    g = C.f32_to_bf16_bits(C.bf16_bits_to_f32(g) + 1)
+    out = B.op_layernorm(torch.from_numpy(x).to(DEV), bits_dev(g), bits_dev(b), 1e-5)
+    ref = O.layer_norm(x.astype(np.float64), O.bf16_to_f64(g), O.bf16_to_f64(b), 1e-5)
+    got = bits_to_f64(out)
+    assert np.max(np.abs(got - ref)) <= 2.0 ** -8 * np.abs(ref).max()
+
+
+def test_sampling_greedy_and_ties():
+    rng = np.random.default_rng(5)
+    R, V = 7, 8194
+    lg = rng.standard_normal(size=(R, V)).astype(np.float32)
+    lg[1, [17, 4000, 8193]] = 9.0          # three-way tie: lowest index wins
+    lg[2, 8193] = 10.0                     # last element (ragged tail of the vocabulary)
+    lg[3, 0] = 10.0
+    got = B.op_sample(torch.from_numpy(lg).to(DEV)).cpu().numpy()
+    want = [O.sample_greedy(lg[r].astype(np.float64)) for r in range(R)]
+    assert list(got) == want
+    assert got[1] == 17 and got[2] == 8193 and got[3] == 0
+
+
+@pytest.mark.parametrize("V,k,T", [(8194, 30, 1.0), (1024, 30, 0.7), (8194, 64, 1.3), (100, 2, 1.0), (50, 50, 1.0)])
+def test_sampling_topk_matches_oracle(V, k, T):
+    rng = np.random.default_rng(V + k)
+    R = 64
+    lg = (rng.standard_normal(size=(R, V)) * 2).astype(np.float32)
+    # ties inside the top-k and across its boundary
+    lg[0, [3, 9, 40]] = lg[0].max() + 1.0
+    order = np.argsort(-lg[1])
+    lg[1, order[k - 2:k + 3]] = lg[1, order[k - 1]]
+    u = rng.random(size=R).astype(np.float32)
+    u[2] = 0.0
+    u[3] = np.nextafter(np.float32(1.0), np.float32(0.0))
+    got = B.op_sample(torch.from_numpy(lg).to(DEV), k, T, torch.from_numpy(u).to(DEV)).cpu().numpy()
+    for r in range(R):
+        l64 = lg[r].astype(np.float64)
+        want = O.sample_topk(l64, k, T, float(u[r]))
+        if got[r] != want:
+            # fp32 vs fp64 CDF: only allowed when u sits on a CDF boundary within rounding
+            I, c = O.topk_cdf(l64, k, T)
+            assert np.min(np.abs(c - u[r])) < 1e-5, (r, got[r], want)
+            assert got[r] in I
+    # the selected set itself is exact: with u -> 1 the last rank comes out
+    assert got[3] == O.topk_order(lg[3].astype(np.float64), k)[-1]
+    assert got[2] == O.topk_order(lg[2].astype(np.float64), k)[0]
+
+
+def test_sampling_topk_frequencies():
+    V, k = 1024, 8
+    rng = np.random.default_rng(11)
+    lg = rng.standard_normal(size=V).astype(np.float32) * 2
+    R = 4096
+    u = C.make_uniforms(R, 1, seed=21)[:, 0]
+    got = B.op_sample(torch.from_numpy(np.tile(lg, (R, 1))).to(DEV), k, 1.0, torch.from_numpy(u).to(DEV)).cpu().numpy()
+    I, c = O.topk_cdf(lg.astype(np.float64), k, 1.0)
+    p = np.diff(np.concatenate([[0.0], c]))
+    counts = np.array([(got == i).sum() for i in I])
+    assert counts.sum() == R
+    chi2 = ((counts - p * R) ** 2 / (p * R)).sum()
+    assert chi2 < 24.32       # 99.9 % quantile, 7 degrees of freedom
