@@ -142,6 +142,10 @@ const char *tts_gpt_last_error(const tts_gpt_t *h);
 int32_t tts_gpt_stats(const tts_gpt_t *h, int32_t *open_streams, int32_t *free_pages);
 int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t stream_id);
 
+/* Number of this library's kernels enqueued on the handle's stream so far (a replayed CUDA graph
+ * counts its kernel nodes on every replay).  HOST output. */
+int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n);
+
 /* Test aid: permute the free-page list with a seeded shuffle (between calls, any time no stream
  * is open).  Results must not depend on which physical pages a stream receives. */
 int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed);

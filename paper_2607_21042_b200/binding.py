@@ -24,6 +24,7 @@ EXPORTS = [
     "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_decode_step",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
+    "tts_gpt_debug_kernel_launches",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
     "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_layernorm",
     "tts_gpt_op_sample",
@@ -218,6 +219,11 @@ class TtsGpt:
 
     def stream_context(self, stream_id):
         return int(self.lib.tts_gpt_stream_context(self.handle, C.c_int32(stream_id)))
+
+    def kernel_launches(self):
+        n = C.c_uint64(0)
+        _check(self.lib.tts_gpt_debug_kernel_launches(self.handle, C.byref(n)), self.handle)
+        return n.value
 
     def debug_shuffle_free_pages(self, seed):
         return _check(self.lib.tts_gpt_debug_shuffle_free_pages(self.handle, C.c_uint32(seed)), self.handle)

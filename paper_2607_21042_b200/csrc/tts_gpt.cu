@@ -66,7 +66,9 @@ struct tts_gpt {
   int n_free;
   // step graphs by row count
   std::map<int, cudaGraphExec_t> graphs;
+  std::map<int, int> graph_nodes;
   bool use_graph;
+  unsigned long long launches = 0;  // kernels enqueued so far (graph nodes counted per replay)
 };
 
 namespace {
@@ -228,6 +230,7 @@ int run_layers(tts_gpt *h, int R) {
     CUDA_TRY(h, launch_linear(c.wfmt, f2, st));
   }
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 7ull * c.n_layer;
   return TTS_GPT_OK;
 }
 
@@ -247,6 +250,7 @@ int run_head(tts_gpt *h, int n_out) {
   sa.stop_token = c.stop_token;
   sample_kernel<<<n_out, kSampleThreads, (size_t)c.vocab * sizeof(float), st>>>(sa);
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 3;
   return TTS_GPT_OK;
 }
 
@@ -254,6 +258,7 @@ int run_embed(tts_gpt *h, int R) {
   const tts_gpt_config_t &c = h->cfg;
   embed_kernel<<<R, 256, 0, h->stream>>>(h->rt, h->tok_emb, h->pos_emb, c.d_model, c.vocab, c.max_pos, h->x);
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 1;
   return TTS_GPT_OK;
 }
 
@@ -379,6 +384,7 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
   }
   prefill_open_kernel<<<1, kMaxRows, 0, h->stream>>>(pp, h->ps);
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 1;
   for (int i = 0; i < n; ++i) {
     const int s = pp.stream_ids[i];
     h->open[s] = 1; h->ctx[s] = prefix_len[i]; h->pos_next[s] = pp.pos0[i];
@@ -398,6 +404,7 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     ps.io.n_out = ps.n_out;
     prefill_pass_kernel<<<1, kMaxRows, 0, h->stream>>>(ps, h->ps, h->rt, h->io, c.d_model);
     CUDA_TRY(h, cudaGetLastError());
+    h->launches += 1;
     int r = run_embed(h, ps.n_rows);
     if (r) return r;
     r = run_layers(h, ps.n_rows);
@@ -451,6 +458,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   sp.io.out_hidden = (uint16_t *)out_hidden; sp.io.top_k = top_k; sp.io.temperature = temperature; sp.io.n_out = n;
   step_setup_kernel<<<1, kMaxRows, 0, h->stream>>>(sp, h->ps, h->rt, h->io);
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 1;
   for (int i = 0; i < n; ++i) { h->ctx[stream_ids[i]] += 1; h->pos_next[stream_ids[i]] += 1; }
   h->n_free -= pages;
 
@@ -458,6 +466,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
     auto it = h->graphs.find(n);
     if (it == h->graphs.end()) {
       cudaGraph_t g = nullptr;
+      const unsigned long long before = h->launches;
       CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
       rc = run_embed(h, n);
       if (!rc) rc = run_layers(h, n);
@@ -470,8 +479,11 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
       cudaGraphDestroy(g);
       if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
       it = h->graphs.emplace(n, ge).first;
+      h->graph_nodes[n] = (int)(h->launches - before);
+      h->launches = before;  // captured, not run
     }
     CUDA_TRY(h, cudaGraphLaunch(it->second, h->stream));
+    h->launches += h->graph_nodes[n];
     return TTS_GPT_OK;
   }
   rc = run_embed(h, n);
@@ -485,6 +497,7 @@ int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
   if (s < 0 || s >= h->cfg.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "release_stream: stream %d is not open", s);
   release_kernel<<<1, 32, 0, h->stream>>>(h->ps, s);
   CUDA_TRY(h, cudaGetLastError());
+  h->launches += 1;
   h->n_free += (h->ctx[s] + 63) / 64;
   h->open[s] = 0; h->ctx[s] = 0;
   return TTS_GPT_OK;
@@ -510,6 +523,12 @@ int32_t tts_gpt_stats(const tts_gpt_t *h, int32_t *open_streams, int32_t *free_p
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   if (open_streams) { int n = 0; for (char o : h->open) n += o; *open_streams = n; }
   if (free_pages) *free_pages = h->n_free;
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n) {
+  if (!h || !n) return fail(nullptr, TTS_GPT_E_ARG, "null argument");
+  *n = h->launches;
   return TTS_GPT_OK;
 }
 

@@ -1,0 +1,167 @@
+"""Parity at the full model size (24 layers, d=1280, vocab 8194) in the launch configuration the
+bench times: workloads 2-5, judged per step on identical history against the fp64 oracle's
+no-cache forward (replay mode), plus batch invariance for the streams the oracle does not replay."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gpt_oracle as O
+from paper_2607_21042_b200 import binding as B
+from paper_2607_21042_b200 import cases as C
+from helpers import assert_logits_close, bits_dev, check_tokens, gpu_run_stream
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+_cache = {}
+
+
+def _model(wfmt):
+    """Weights of the full model in one format (drawn once per session) and its oracle."""
+    if wfmt not in _cache:
+        _cache.clear()              # one fp64 model (3.9 GB) at a time
+        cfg = C.full_config(wfmt=wfmt)
+        w = C.make_weights(cfg, seed=0)
+        _cache[wfmt] = (w, O.OracleModel(cfg, w))
+    return _cache[wfmt]
+
+
+def _batch_run(eng, wl, prefixes, n_steps, decode_lens=None):
+    """All streams prefilled together; n_steps batched steps; streams leave after decode_lens[i]
+    steps.  Returns per-stream lists of (token, logits row)."""
+    S = len(prefixes)
+    V = wl.cfg.vocab
+    t0 = torch.zeros(S, dtype=torch.int32, device=DEV)
+    l0 = torch.zeros((S, V), dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    ids, _ = eng.prefill([bits_dev(p) for p in prefixes], out_tokens=t0, out_logits=l0)
+    toks = torch.zeros((n_steps, S), dtype=torch.int32, device=DEV)
+    logits = torch.zeros((n_steps, S, V), dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    alive = list(range(S))
+    rows = [[] for _ in range(S)]
+    for k in range(1, n_steps + 1):
+        if decode_lens is not None:
+            for i in list(alive):
+                if decode_lens[i] < k:
+                    eng.release_stream(ids[i]); alive.remove(i)
+        if not alive:
+            break
+        n = len(alive)
+        eng.decode_step([ids[i] for i in alive], toks[k - 1, :n], out_logits=logits[k - 1, :n])
+        for j, i in enumerate(alive):
+            rows[i].append((k - 1, j))
+    eng.sync()
+    for i in alive:
+        eng.release_stream(ids[i])
+    tk, lg = toks.cpu().numpy(), logits.cpu().numpy()
+    t0, l0 = t0.cpu().numpy(), l0.cpu().numpy()
+    out = []
+    for i in range(S):
+        seq = [int(t0[i])] + [int(tk[k, j]) for k, j in rows[i]]
+        lgs = np.stack([l0[i]] + [lg[k, j] for k, j in rows[i]])
+        out.append((np.array(seq), lgs))
+    return out
+
+def _workload5(wfmt):
+    wl = C.workload(5, wfmt=wfmt)
+    w, model = _model(wfmt)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    prefixes = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)
+    # shorten the drain so the test stays in minutes: every stream leaves after min(n_i, cap) steps
+    cap = 96
+    dl = [min(x, cap - (i % 32)) for i, x in enumerate(wl.decode_lens)]
+    res = _batch_run(eng, wl, prefixes, cap, decode_lens=dl)
+    assert eng.stats() == {"open_streams": 0, "free_pages": wl.cfg.n_pages}
+    total = [p + x for p, x in zip(wl.prefix_lens, dl)]
+    picks = sorted({int(np.argmax(total)), int(np.argmin(wl.prefix_lens)), 17, 100})
+    for i in picks:
+        seq, lg = res[i]
+        assert len(seq) == dl[i] + 1
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
+        ma, rl = assert_logits_close(lg, ref, "workload 5 stream %d" % i)
+        exc = check_tokens(seq, ref, 0, 1.0, None, "workload 5 stream %d" % i)
+        print("workload5[%s] stream %d (P=%d, n=%d): max-abs %.4g rel-L2 %.4g excused %d" % (
+            C.WFMT_NAMES[wfmt], i, wl.prefix_lens[i], dl[i], ma, rl, exc))
+    # batch invariance for two streams the oracle did not replay
+    for i in (5, 64):
+        if i in picks:
+            continue
+        alone = _batch_run(eng, wl, [prefixes[i]], 24)[0]
+        m = min(25, len(res[i][0]))
+        assert np.array_equal(alone[0][:m], res[i][0][:m])
+        assert_logits_close(alone[1][:m], res[i][1][:m].astype(np.float64), "batch invariance stream %d" % i)
+    eng.destroy()
+
+def test_workload2_bf16_batch1_replay():
+    wl = C.workload(2)
+    w, model = _model(C.W_BF16)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    prefix = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)[0]
+    n = wl.decode_lens[0]
+    toks, logits, hidden, sid = gpu_run_stream(eng, bits_dev(prefix), n, want_hidden=True)
+    ref, ref_h = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    ma, rl = assert_logits_close(logits, ref, "workload 2")
+    exc = check_tokens(toks, ref, 0, 1.0, None, "workload 2")
+    assert np.max(np.abs(O.bf16_to_f64(hidden) - ref_h)) <= 3e-2 * max(1.0, np.abs(ref_h).max())
+    print("workload2: max-abs %.4g rel-L2 %.4g excused %d/%d" % (ma, rl, exc, n + 1))
+    eng.destroy()
+
+def test_long_context_2048_full_model():
+    """One stream driven to the maximum context (2048 tokens = 32 pages = 8 chunks)."""
+    wl = C.workload(2)
+    w, model = _model(C.W_BF16)
+    cfg = C.full_config(wfmt=C.W_BF16, max_streams=1, n_pages=32, max_pos=1024)
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [1990], seed=6)[0]
+    toks, logits, _, sid = gpu_run_stream(eng, bits_dev(prefix), 58)
+    assert eng.stream_context(sid) == 2048
+    ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref, "context 2048")
+    check_tokens(toks, ref, 0, 1.0, None, "context 2048")
+    eng.destroy()
+
+def test_workload5_bf16_batch128_ragged_drain():
+    _workload5(C.W_BF16)
+
+def test_workload3_w8a16_topk_replay():
+    wl = C.workload(3)
+    w, model = _model(C.W_INT8_PC)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    prefix = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)[0]
+    n = wl.decode_lens[0]
+    u = C.make_uniforms(n + 1, 1, seed=0)[:, 0]
+    toks, logits, _, sid = gpu_run_stream(eng, bits_dev(prefix), n, top_k=30, temperature=1.0,
+                                          uniforms_dev=torch.from_numpy(u).to(DEV))
+    ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    ma, rl = assert_logits_close(logits, ref, "workload 3")
+    exc = check_tokens(toks, ref, 30, 1.0, u, "workload 3")
+    print("workload3: max-abs %.4g rel-L2 %.4g excused %d/%d" % (ma, rl, exc, n + 1))
+    eng.destroy()
+
+def test_workload4_w4a16_batch16_replay_and_batch_invariance():
+    wl = C.workload(4)
+    w, model = _model(C.W_INT4_G128)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    prefixes = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)
+    n = 120        # decode steps compared (the bench runs 500; every step is the same launch shape)
+    res = _batch_run(eng, wl, prefixes, n)
+    lens = list(wl.prefix_lens)
+    picks = sorted({int(np.argmin(lens)), int(np.argmax(lens)), 3, 11})
+    for i in picks:
+        seq, lg = res[i]
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
+        ma, rl = assert_logits_close(lg, ref, "workload 4 stream %d" % i)
+        exc = check_tokens(seq, ref, 0, 1.0, None, "workload 4 stream %d" % i)
+        print("workload4 stream %d (P=%d): max-abs %.4g rel-L2 %.4g excused %d/%d" % (i, lens[i], ma, rl, exc, n + 1))
+    # the other streams: same numbers inside the batch of 16 as when run alone
+    for i in (0, 7):
+        if i in picks:
+            continue
+        alone = _batch_run(eng, wl, [prefixes[i]], 40)[0]
+        assert np.array_equal(alone[0], res[i][0][:41])
+        assert_logits_close(alone[1], res[i][1][:41].astype(np.float64), "batch invariance stream %d" % i)
+    eng.destroy()
+
+def test_workload5_w4a16_batch128_ragged_drain():
+    _workload5(C.W_INT4_G128)
