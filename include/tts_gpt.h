@@ -183,6 +183,27 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
                              const int32_t *row_stream, const int32_t *row_pos, void *out,
                              void *scratch, void *cuda_stream);
 
+/* Same attention as tts_gpt_op_attention for callers that cannot hand over scratch memory because
+ * they cannot allocate any: code that runs where cudaMalloc is off limits — a per-request handler of
+ * a serving process whose whole device budget was carved up at start-up, a plug-in inside a host
+ * engine that owns all device memory, a latency-critical audio thread that must never hit the
+ * device-wide synchronisation an allocation implies.  (The paper has no counterpart of this call; it
+ * is a convenience of this library.)  The split-KV partial results and ticket counters go into an
+ * array built into the library image: about 2.7 MB that every GPU loading the library carries
+ * until the process exits.  Limit: R * n_head <= TTS_GPT_STATIC_ATTN_MAX_ROW_HEADS; larger calls
+ * return TTS_GPT_E_WORKSPACE and enqueue nothing.  The call allocates nothing and frees nothing.
+ * The first call on each device (with that device current) looks up the array's device address;
+ * make that first call before starting any stream capture.  All calls on a device share the one
+ * array: it still holds the previous call's partials (harmless, they are overwritten before use)
+ * and the call itself zeroes the tickets it needs on `cuda_stream`; two calls that can overlap on
+ * the GPU (different streams without ordering) race on it and must be serialised by the caller.
+ * Arguments and results otherwise exactly as tts_gpt_op_attention. */
+#define TTS_GPT_STATIC_ATTN_MAX_ROW_HEADS 1280
+int32_t tts_gpt_op_attention_static(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                                    const int32_t *page_table, int32_t pages_per_stream,
+                                    const int32_t *row_stream, const int32_t *row_pos, void *out,
+                                    void *cuda_stream);
+
 /* LayerNorm over rows: x fp32 [R,d], g/b bf16 [d] -> out bf16 [R,d]. */
 int32_t tts_gpt_op_layernorm(int32_t R, int32_t d, const float *x, const void *g, const void *b,
                              float eps, void *out, void *cuda_stream);

@@ -26,7 +26,8 @@ EXPORTS = [
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
     "tts_gpt_debug_kernel_launches",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
-    "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_layernorm",
+    "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static",
+    "tts_gpt_op_layernorm",
     "tts_gpt_op_sample",
 ]
 
@@ -284,6 +285,22 @@ def op_attention(q, kv_layer, page_table, row_stream, row_pos, scratch=None, str
     _check(load().tts_gpt_op_attention(C.c_int32(R), C.c_int32(H), _ptr(q), _ptr(kv_layer), _ptr(page_table),
                                        C.c_int32(page_table.shape[1]), _ptr(row_stream), _ptr(row_pos),
                                        _ptr(out), _ptr(scratch), _stream_ptr(stream)))
+    return out
+
+
+STATIC_ATTN_MAX_ROW_HEADS = 1280
+
+
+def op_attention_static(q, kv_layer, page_table, row_stream, row_pos, stream=None):
+    """Attention for callers that may not allocate: scratch is an array inside the library (at most
+    STATIC_ATTN_MAX_ROW_HEADS rows x heads).  Only the output tensor is created here, by torch; pass
+    your own through the C entry point to avoid even that.  Calls on one device must not overlap."""
+    R, dm = q.shape
+    H = dm // 64
+    out = torch.empty((R, dm), dtype=torch.int16, device=q.device)
+    _check(load().tts_gpt_op_attention_static(C.c_int32(R), C.c_int32(H), _ptr(q), _ptr(kv_layer),
+                                              _ptr(page_table), C.c_int32(page_table.shape[1]),
+                                              _ptr(row_stream), _ptr(row_pos), _ptr(out), _stream_ptr(stream)))
     return out
 
 

@@ -610,6 +610,62 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
   return TTS_GPT_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Attention without caller-provided scratch: the split-KV partials and tickets live in a fixed
+// array inside the library image.
+// ---------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+constexpr int kStaticAttnMaxRowHeads = TTS_GPT_STATIC_ATTN_MAX_ROW_HEADS;
+constexpr size_t kStaticAttnPartialBytes =
+    (size_t)kStaticAttnMaxRowHeads * kAttnMaxChunks * kAttnPartialFloats * sizeof(float);
+constexpr size_t kStaticAttnBytes = kStaticAttnPartialBytes + (size_t)kStaticAttnMaxRowHeads * sizeof(unsigned int);
+static_assert(kStaticAttnPartialBytes % 256 == 0, "tickets must start 256-byte aligned");
+// Lives in every GPU that loads the library, from load until process exit (about 2.7 MB).
+static __device__ __align__(256) unsigned char g_static_attn_scratch[kStaticAttnBytes];
+// The symbol above is only a host-side stand-in when named in host code: its device address has to
+// be asked for, once per device, with that device current.
+constexpr int kMaxDevices = 64;
+void *g_static_attn_ptr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" {
+
+int32_t tts_gpt_op_attention_static(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                                    const int32_t *page_table, int32_t pages_per_stream,
+                                    const int32_t *row_stream, const int32_t *row_pos, void *out,
+                                    void *cuda_stream) {
+  if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
+      pages_per_stream < 1 || pages_per_stream > kAttnMaxChunks * kAttnWarps)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_static: bad argument");
+  if ((long long)R * n_head > kStaticAttnMaxRowHeads)
+    return fail(nullptr, TTS_GPT_E_WORKSPACE,
+                "op_attention_static: R*n_head = %lld exceeds the built-in scratch limit of %d row-heads; "
+                "use tts_gpt_op_attention with caller scratch",
+                (long long)R * n_head, kStaticAttnMaxRowHeads);
+  int dev = -1;
+  CUDA_TRY(nullptr, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, TTS_GPT_E_UNSUPPORTED, "op_attention_static: device index %d", dev);
+  if (!g_static_attn_ptr[dev]) {  // first call on this device: resolve the array's device address
+    void *p = nullptr;
+    CUDA_TRY(nullptr, cudaGetSymbolAddress(&p, g_static_attn_scratch));
+    if (!p) return fail(nullptr, TTS_GPT_E_CUDA, "op_attention_static: no device address for the scratch array");
+    g_static_attn_ptr[dev] = p;
+  }
+  unsigned char *base = (unsigned char *)g_static_attn_ptr[dev];
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  AttnArgs a;
+  a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
+  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  a.partials = (float *)base;
+  a.tickets = (unsigned int *)(base + kStaticAttnPartialBytes);
+  // The array keeps whatever the previous call left; the tickets have to start at zero.
+  CUDA_TRY(nullptr, cudaMemsetAsync(a.tickets, 0, (size_t)R * n_head * sizeof(unsigned int), st));
+  CUDA_TRY(nullptr, launch_attention(a, R, pages_per_stream * kPageTokens, st));
+  return TTS_GPT_OK;
+}
+
 int32_t tts_gpt_op_layernorm(int32_t R, int32_t d, const float *x, const void *g, const void *b, float eps,
                              void *out, void *cuda_stream) {
   if (R < 1 || d < 1 || d > kLnThreads * kLnMaxPerThread || !x || !g || !b || !out) return fail(nullptr, TTS_GPT_E_ARG, "op_layernorm: bad argument");
