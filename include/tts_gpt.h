@@ -146,6 +146,13 @@ int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t stream_id);
  * counts its kernel nodes on every replay).  HOST output. */
 int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n);
 
+/* Timeline tracing (off by default).  `trace` is a DEVICE array of 8 * n_slots uint64, or NULL to
+ * switch tracing off; *n_slots (HOST, may be NULL) receives the number of traced kernels per step
+ * (5 per layer: QKV, attention, O-proj, FC1, FC2; then the LM head).  While set, CTA 0 of each
+ * traced kernel stores the GPU's global nanosecond timer at entry, after its dependency wait and
+ * at its end into trace[8*slot + 0..2] (3..5: inner points of the linear kernels).  Synchronises and drops captured graphs. */
+int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots);
+
 /* Test aid: permute the free-page list with a seeded shuffle (between calls, any time no stream
  * is open).  Results must not depend on which physical pages a stream receives. */
 int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed);
@@ -182,6 +189,14 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
                              const int32_t *page_table, int32_t pages_per_stream,
                              const int32_t *row_stream, const int32_t *row_pos, void *out,
                              void *scratch, void *cuda_stream);
+
+/* The engine's attention kernel: same result as tts_gpt_op_attention, but each (row, head) is split
+ * over a thread-block cluster of cluster_size (1, 2, 4 or 8) CTAs that merge their partial results
+ * through distributed shared memory; needs no scratch. */
+int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                                     const int32_t *page_table, int32_t pages_per_stream,
+                                     const int32_t *row_stream, const int32_t *row_pos, void *out,
+                                     int32_t cluster_size, void *cuda_stream);
 
 /* Same attention as tts_gpt_op_attention for callers that cannot hand over scratch memory because
  * they cannot allocate any: code that runs where cudaMalloc is off limits — a per-request handler of

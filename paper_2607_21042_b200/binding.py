@@ -24,9 +24,9 @@ EXPORTS = [
     "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_decode_step",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
-    "tts_gpt_debug_kernel_launches",
+    "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
-    "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static",
+    "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static", "tts_gpt_op_attention_cluster",
     "tts_gpt_op_layernorm",
     "tts_gpt_op_sample",
 ]
@@ -226,6 +226,13 @@ class TtsGpt:
         _check(self.lib.tts_gpt_debug_kernel_launches(self.handle, C.byref(n)), self.handle)
         return n.value
 
+    def set_trace(self, trace_tensor):
+        """trace_tensor: int64 device tensor with 8 * slots entries (or None to switch off).
+        Returns the number of traced kernels per step."""
+        n = C.c_int32(0)
+        _check(self.lib.tts_gpt_debug_set_trace(self.handle, _ptr(trace_tensor), C.byref(n)), self.handle)
+        return n.value
+
     def debug_shuffle_free_pages(self, seed):
         return _check(self.lib.tts_gpt_debug_shuffle_free_pages(self.handle, C.c_uint32(seed)), self.handle)
 
@@ -285,6 +292,17 @@ def op_attention(q, kv_layer, page_table, row_stream, row_pos, scratch=None, str
     _check(load().tts_gpt_op_attention(C.c_int32(R), C.c_int32(H), _ptr(q), _ptr(kv_layer), _ptr(page_table),
                                        C.c_int32(page_table.shape[1]), _ptr(row_stream), _ptr(row_pos),
                                        _ptr(out), _ptr(scratch), _stream_ptr(stream)))
+    return out
+
+
+def op_attention_cluster(q, kv_layer, page_table, row_stream, row_pos, cluster_size, stream=None):
+    R, dm = q.shape
+    H = dm // 64
+    out = torch.empty((R, dm), dtype=torch.int16, device=q.device)
+    _check(load().tts_gpt_op_attention_cluster(C.c_int32(R), C.c_int32(H), _ptr(q), _ptr(kv_layer),
+                                               _ptr(page_table), C.c_int32(page_table.shape[1]),
+                                               _ptr(row_stream), _ptr(row_pos), _ptr(out),
+                                               C.c_int32(cluster_size), _stream_ptr(stream)))
     return out
 
 

@@ -1,21 +1,35 @@
 // Split-KV decode attention over 64-token pages (Section I: the decode engine's attention kernels
-// and KV-cache management).  One warp owns one page of one (row, head): it streams the 8 KB K block
-// and the 8 KB V block with 128-bit loads, keeps scores, softmax statistics and the output in fp32
-// registers, and uses warp shuffles for the reductions.  Four warps (a 256-token chunk) meet in
-// shared memory; when a row needs several chunks the per-chunk (max, sum, output) triples go to
-// scratch and the CTA that arrives last at the row's ticket counter merges them in chunk order by
-// log-sum-exp (no spinning, no dependence on arrival order).
+// and KV-cache management).
 //
 // KV pool, per layer: bf16 [n_pages][2 (K|V)][n_head][64 tokens][64]; each (page, K|V, head) block
 // is 8 KB contiguous.
+//
+// Work split.  A (row, head) pair is handled by a thread-block cluster of S CTAs (S = 1, 2, 4 or 8,
+// picked per launch so that the grid fills the GPU: S = 8 at batch 1, S = 1 at batch 128).  The
+// row's pages are dealt round-robin: CTA c of the cluster takes pages c, c+S, c+2S, ...; inside a
+// CTA its 4 warps take those in turn.  One warp streams a page's 8 KB K block and 8 KB V block
+// with 16+16 independent 128-bit loads per lane, keeps scores, the running softmax statistics
+// (max, sum) and the running output in fp32 registers (online softmax across its pages), and uses
+// shuffles for the reductions.  The warps of a CTA meet in shared memory; the CTAs of a cluster
+// meet in distributed shared memory: rank 0 reads the other ranks' (max, sum, output) triples and
+// merges them by log-sum-exp in rank order.  No global scratch, no atomics, no spinning; the
+// result does not depend on timing.
+//
+// A second variant (`attention_ticket_kernel`) exchanges the partial results through global
+// scratch and lets the CTA that arrives last at a ticket counter do the merge.  It needs no
+// cluster launch and backs the stand-alone entry points.
 #pragma once
+#include <cooperative_groups.h>
 #include "common.cuh"
 
 namespace ttsgpt {
 
-constexpr int kAttnWarps = 4;             // pages per chunk
-constexpr int kAttnMaxChunks = 8;         // 2048 tokens / 256
+namespace cg = cooperative_groups;
+
+constexpr int kAttnWarps = 4;             // warps per CTA (pages in flight per CTA)
+constexpr int kAttnMaxChunks = 8;         // ticket variant: 2048 tokens / 256
 constexpr int kAttnPartialFloats = 66;    // m, l, o[64]
+constexpr int kAttnMaxCluster = 8;
 
 inline size_t attention_scratch_bytes(int R, int H) {
   return align256((size_t)R * H * kAttnMaxChunks * kAttnPartialFloats * sizeof(float)) +
@@ -28,19 +42,240 @@ struct AttnArgs {
   const int *page_table;     // [*, pps]
   const int *row_stream, *row_pos;
   uint16_t *out;             // bf16 [R][H*64]
-  float *partials;           // [R][H][kAttnMaxChunks][66]
-  unsigned int *tickets;     // [R][H], zero between launches
+  float *partials;           // ticket variant: [R][H][kAttnMaxChunks][66]
+  unsigned int *tickets;     // ticket variant: [R][H], zero between launches
   int H, pps;
+  unsigned long long *trace;  // optional timeline trace
+  int trace_slot;
+  int old_pages_final;       // 1: one row per stream (decode step), pages before a row's last are not written by this step
 };
 
+// ------------------------------------------------------------------------------------------
+// one page for one warp: scores, page-local softmax statistics, weighted values
+// ------------------------------------------------------------------------------------------
+struct PageLoad { uint4 kk[16], vv[16]; };
+
+__device__ __forceinline__ void load_page(PageLoad &pl, const uint16_t *K, const uint16_t *V, int tg, int sub) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) pl.kk[i] = ld_stream_u4(K + (size_t)(tg + 4 * i) * kHeadDim + 8 * sub);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) pl.vv[i] = ld_stream_u4(V + (size_t)(tg + 4 * i) * kHeadDim + 8 * sub);
+}
+
+// Folds one page into the warp's running (m, l, o).  Lane (tg, sub) = (lane/8, lane%8) sees tokens
+// tg, tg+4, ... and elements 8*sub..8*sub+7 of the head; m and l are warp-uniform, o[e] is the
+// lane's partial over its tokens (summed over tg at the very end).
+__device__ __forceinline__ void fold_page(PageLoad &pl, const float (&qv)[8], int n_here, int tg, float &m, float &l,
+                                          float (&o)[8]) {
+  float s[16];
+  float pm = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    float d = qv[0] * bf16_lo(pl.kk[i].x);
+    d = fmaf(qv[1], bf16_hi(pl.kk[i].x), d);
+    d = fmaf(qv[2], bf16_lo(pl.kk[i].y), d);
+    d = fmaf(qv[3], bf16_hi(pl.kk[i].y), d);
+    d = fmaf(qv[4], bf16_lo(pl.kk[i].z), d);
+    d = fmaf(qv[5], bf16_hi(pl.kk[i].z), d);
+    d = fmaf(qv[6], bf16_lo(pl.kk[i].w), d);
+    d = fmaf(qv[7], bf16_hi(pl.kk[i].w), d);
+    d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
+    d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
+    d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
+    const bool valid = tg + 4 * i < n_here;
+    s[i] = valid ? d : -INFINITY;
+    if (!valid) pl.vv[i] = make_uint4(0, 0, 0, 0);  // stale page contents may hold NaN: 0 * NaN must not reach o
+    pm = fmaxf(pm, s[i]);
+  }
+  pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 8));
+  pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 16));
+  const float m_new = fmaxf(m, pm);           // finite: every page has at least one valid token
+  const float rescale = exp2f(m - m_new);     // first page: exp2(-inf) = 0
+  float lp = 0.f;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) o[e] *= rescale;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const float p = exp2f(s[i] - m_new);  // masked tokens: exp2(-inf) = 0
+    lp += p;
+    o[0] = fmaf(p, bf16_lo(pl.vv[i].x), o[0]);
+    o[1] = fmaf(p, bf16_hi(pl.vv[i].x), o[1]);
+    o[2] = fmaf(p, bf16_lo(pl.vv[i].y), o[2]);
+    o[3] = fmaf(p, bf16_hi(pl.vv[i].y), o[3]);
+    o[4] = fmaf(p, bf16_lo(pl.vv[i].z), o[4]);
+    o[5] = fmaf(p, bf16_hi(pl.vv[i].z), o[5]);
+    o[6] = fmaf(p, bf16_lo(pl.vv[i].w), o[6]);
+    o[7] = fmaf(p, bf16_hi(pl.vv[i].w), o[7]);
+  }
+  lp += __shfl_xor_sync(0xFFFFFFFFu, lp, 8);
+  lp += __shfl_xor_sync(0xFFFFFFFFu, lp, 16);
+  l = l * rescale + lp;
+  m = m_new;
+}
+
+__device__ __forceinline__ void load_q(float (&qv)[8], const float *q) {
+  // scores come out in log2 units: 1/sqrt(64) * log2(e)
+  const float qs = 0.125f * 1.4426950408889634f;
+  const float4 q0 = *reinterpret_cast<const float4 *>(q);
+  const float4 q1 = *reinterpret_cast<const float4 *>(q + 4);
+  qv[0] = q0.x * qs; qv[1] = q0.y * qs; qv[2] = q0.z * qs; qv[3] = q0.w * qs;
+  qv[4] = q1.x * qs; qv[5] = q1.y * qs; qv[6] = q1.z * qs; qv[7] = q1.w * qs;
+}
+
+// warp result -> shared memory; then threads 0..63 merge the CTA's warps in warp order
+__device__ __forceinline__ void cta_merge(float m, float l, float (&o)[8], int warp, int tg, int sub,
+                                          float (&sm_m)[kAttnWarps], float (&sm_l)[kAttnWarps],
+                                          float (&sm_o)[kAttnWarps][kHeadDim], float &M, float &L, float &O) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 8);
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 16);
+  }
+  if (tg == 0) {
+    if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sm_o[warp][8 * sub + e] = o[e];
+  }
+  __syncthreads();
+  M = -INFINITY; L = 0.f; O = 0.f;
+  const int e = threadIdx.x;
+  if (e < kHeadDim) {
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sm_m[w]);
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) {
+      const float f = (sm_m[w] == -INFINITY) ? 0.f : exp2f(sm_m[w] - M);  // idle warp contributes nothing
+      L = fmaf(sm_l[w], f, L);
+      O = fmaf(sm_o[w][e], f, O);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// cluster variant (the engine's path)
+// ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnArgs a) {
+  const int S = gridDim.x, c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
+  trace_mark(a.trace, a.trace_slot, 0);
+  // The row table and page table were written before the first kernel of the step started, so
+  // they may be read ahead of the dependency wait.
+  const int n_tok = a.row_pos[r] + 1;
+  const int n_pages = (n_tok + kPageTokens - 1) / kPageTokens;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tg = lane >> 3, sub = lane & 7;
+  const int *pt = a.page_table + (size_t)a.row_stream[r] * a.pps;
+
+  __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
+  __shared__ float cl_part[kAttnPartialFloats];  // this CTA's (M, L, O[64]) for the cluster merge
+
+  // this warp's pages: c + S*(warp + kAttnWarps*it)
+  int page = c + S * warp;
+  PageLoad pl;
+  // In a decode step every page but the row's last one holds only tokens of earlier steps: the
+  // first page's loads do not depend on the QKV kernel in front and are issued before waiting for it.
+  const bool early = a.old_pages_final && page < n_pages - 1;
+  if (early) {
+    const int phys = pt[page];
+    load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
+              a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+
+  float m = -INFINITY, l = 0.f;
+  float o[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) o[e] = 0.f;
+  float qv[8];
+  load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+  bool loaded = early;
+  for (; page < n_pages; page += S * kAttnWarps) {
+    if (!loaded) {
+      const int phys = pt[page];
+      load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
+                a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
+    }
+    loaded = false;
+    fold_page(pl, qv, min(kPageTokens, n_tok - page * kPageTokens), tg, m, l, o);
+  }
+  trace_mark(a.trace, a.trace_slot, 3);
+  float M, L, O;
+  cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
+  trace_mark(a.trace, a.trace_slot, 4);
+  const int e = threadIdx.x;
+  uint16_t *out = a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim;
+  if (S == 1) {
+    if (e < kHeadDim) out[e] = float_to_bf16_bits(O / L);
+    trace_mark(a.trace, a.trace_slot, 2);
+    return;
+  }
+  cg::cluster_group cluster = cg::this_cluster();
+  if (e < kHeadDim) {
+    if (e == 0) { cl_part[0] = M; cl_part[1] = L; }
+    cl_part[2 + e] = O;
+  }
+  cluster.sync();
+  trace_mark(a.trace, a.trace_slot, 5);
+  if (c == 0 && e < kHeadDim) {
+    float MM = -INFINITY;
+    for (int rr = 0; rr < S; ++rr) MM = fmaxf(MM, cluster.map_shared_rank(cl_part, rr)[0]);
+    float LL = 0.f, OO = 0.f;
+    for (int rr = 0; rr < S; ++rr) {
+      const float *p = cluster.map_shared_rank(cl_part, rr);
+      const float pm = p[0];
+      const float f = (pm == -INFINITY) ? 0.f : exp2f(pm - MM);  // a rank without pages contributes nothing
+      LL = fmaf(p[1], f, LL);
+      OO = fmaf(p[2 + e], f, OO);
+    }
+    out[e] = float_to_bf16_bits(OO / LL);
+  }
+  cluster.sync();  // keep every rank's shared memory alive until rank 0 has read it
+  trace_mark(a.trace, a.trace_slot, 2);
+}
+
+// Cluster size for R rows of H heads on n_sm SMs: enough CTAs to cover the GPU about once.
+inline int attention_cluster_size(int R, int H, int n_sm) {
+  int s = 1;
+  while (s < kAttnMaxCluster && R * H * s < n_sm) s *= 2;
+  return s;
+}
+
+inline cudaError_t launch_attention(const AttnArgs &a, int R, int cluster, cudaStream_t st, bool pdl) {
+  cudaLaunchConfig_t cfg;
+  cfg.gridDim = dim3(cluster, a.H, R);
+  cfg.blockDim = dim3(kAttnWarps * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  int n = 0;
+  if (cluster > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = cluster; at[n].val.clusterDim.y = 1; at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  if (pdl) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, attention_kernel, a);
+}
+
+// ------------------------------------------------------------------------------------------
+// ticket variant: chunks of 4 pages per CTA, partial results through global scratch, merged by
+// the CTA that arrives last at the row's ticket counter (no spinning)
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kAttnWarps * 32) attention_ticket_kernel(const AttnArgs a) {
   const int c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
   const int n_tok = a.row_pos[r] + 1;
   const int n_pages = (n_tok + kPageTokens - 1) / kPageTokens;
   const int n_chunks = (n_pages + kAttnWarps - 1) / kAttnWarps;
   if (c >= n_chunks) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tg = lane >> 3, sub = lane & 7;  // token group (4 tokens per load), 8-element slice of the head
+  const int tg = lane >> 3, sub = lane & 7;
   const int page = c * kAttnWarps + warp;
 
   __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
@@ -50,88 +285,18 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   float o[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) o[e] = 0.f;
-
   if (page < n_pages) {
     const int phys = a.page_table[(size_t)a.row_stream[r] * a.pps + page];
-    const uint16_t *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
-    const uint16_t *V = a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems;
-    const int n_here = min(kPageTokens, n_tok - page * kPageTokens);
-    // scores come out in log2 units: 1/sqrt(64) * log2(e)
-    const float qs = 0.125f * 1.4426950408889634f;
+    PageLoad pl;
+    load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
+              a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
     float qv[8];
-    {
-      const float4 q0 = *reinterpret_cast<const float4 *>(a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
-      const float4 q1 = *reinterpret_cast<const float4 *>(a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub + 4);
-      qv[0] = q0.x * qs; qv[1] = q0.y * qs; qv[2] = q0.z * qs; qv[3] = q0.w * qs;
-      qv[4] = q1.x * qs; qv[5] = q1.y * qs; qv[6] = q1.z * qs; qv[7] = q1.w * qs;
-    }
-    uint4 kk[16], vv[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) kk[i] = ld_stream_u4(K + (size_t)(tg + 4 * i) * kHeadDim + 8 * sub);
-#pragma unroll
-    for (int i = 0; i < 16; ++i) vv[i] = ld_stream_u4(V + (size_t)(tg + 4 * i) * kHeadDim + 8 * sub);
-    float s[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      float d = qv[0] * bf16_lo(kk[i].x);
-      d = fmaf(qv[1], bf16_hi(kk[i].x), d);
-      d = fmaf(qv[2], bf16_lo(kk[i].y), d);
-      d = fmaf(qv[3], bf16_hi(kk[i].y), d);
-      d = fmaf(qv[4], bf16_lo(kk[i].z), d);
-      d = fmaf(qv[5], bf16_hi(kk[i].z), d);
-      d = fmaf(qv[6], bf16_lo(kk[i].w), d);
-      d = fmaf(qv[7], bf16_hi(kk[i].w), d);
-      d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
-      d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
-      d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
-      const bool valid = tg + 4 * i < n_here;
-      s[i] = valid ? d : -INFINITY;
-      if (!valid) vv[i] = make_uint4(0, 0, 0, 0);  // stale page contents may hold NaN: 0 * NaN must not reach o
-      m = fmaxf(m, s[i]);
-    }
-    m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 8));
-    m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, 16));
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const float p = exp2f(s[i] - m);  // masked tokens: exp2(-inf) = 0
-      l += p;
-      o[0] = fmaf(p, bf16_lo(vv[i].x), o[0]);
-      o[1] = fmaf(p, bf16_hi(vv[i].x), o[1]);
-      o[2] = fmaf(p, bf16_lo(vv[i].y), o[2]);
-      o[3] = fmaf(p, bf16_hi(vv[i].y), o[3]);
-      o[4] = fmaf(p, bf16_lo(vv[i].z), o[4]);
-      o[5] = fmaf(p, bf16_hi(vv[i].z), o[5]);
-      o[6] = fmaf(p, bf16_lo(vv[i].w), o[6]);
-      o[7] = fmaf(p, bf16_hi(vv[i].w), o[7]);
-    }
-    l += __shfl_xor_sync(0xFFFFFFFFu, l, 8);
-    l += __shfl_xor_sync(0xFFFFFFFFu, l, 16);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 8);
-      o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 16);
-    }
+    load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+    fold_page(pl, qv, min(kPageTokens, n_tok - page * kPageTokens), tg, m, l, o);
   }
-  if (tg == 0) {
-    if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) sm_o[warp][8 * sub + e] = o[e];
-  }
-  __syncthreads();
-
-  // merge the chunk's warps (in warp order)
-  float M = -INFINITY, L = 0.f, O = 0.f;
+  float M, L, O;
+  cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
   const int e = threadIdx.x;
-  if (e < kHeadDim) {
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sm_m[w]);
-#pragma unroll
-    for (int w = 0; w < kAttnWarps; ++w) {
-      const float f = exp2f(sm_m[w] - M);  // empty warp: m = -inf -> 0
-      L = fmaf(sm_l[w], f, L);
-      O = fmaf(sm_o[w][e], f, O);
-    }
-  }
   uint16_t *out = a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim;
   if (n_chunks == 1) {
     if (e < kHeadDim) out[e] = float_to_bf16_bits(O / L);
@@ -164,12 +329,11 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   if (threadIdx.x == 0) a.tickets[(size_t)r * a.H + h] = 0u;  // ready for the next launch
 }
 
-inline cudaError_t launch_attention(const AttnArgs &a, int R, int max_tokens, cudaStream_t st) {
+inline cudaError_t launch_attention_ticket(const AttnArgs &a, int R, int max_tokens, cudaStream_t st) {
   int chunks = (max_tokens + kAttnWarps * kPageTokens - 1) / (kAttnWarps * kPageTokens);
   if (chunks < 1) chunks = 1;
   if (chunks > kAttnMaxChunks) chunks = kAttnMaxChunks;
-  dim3 grid(chunks, a.H, R);
-  attention_kernel<<<grid, kAttnWarps * 32, 0, st>>>(a);
+  attention_ticket_kernel<<<dim3(chunks, a.H, R), kAttnWarps * 32, 0, st>>>(a);
   return cudaGetLastError();
 }
 

@@ -47,6 +47,41 @@ __device__ __forceinline__ uint4 ld_stream_u4(const void *p) {
   return r;
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute
+// may start while its predecessor on the stream is still running; `pdl_wait` blocks until every
+// predecessor has completed and its writes are visible, `pdl_launch_dependents` lets the successor
+// start early.  Before `pdl_wait` a kernel may only touch data that no kernel of the step writes
+// (weights, and state written before the first kernel of the chain started).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Optional timeline trace: thread 0 of CTA 0 of a traced kernel stores the global nanosecond timer
+// at entry, after the dependency wait, at its end (and at up to five inner points) into
+// trace[8*slot + 0..7].
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void trace_mark(unsigned long long *trace, int slot, int which) {
+  if (trace && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    trace[8 * slot + which] = global_timer_ns();
+}
+
+// Launches `kernel` with or without the programmatic-serialization attribute.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 bool pdl, Args... args) {
+  cudaLaunchConfig_t cfg;
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col).  Fragment layout (g = lane/4, t = lane%4):
 // a0=(row g, k 2t..2t+1) a1=(row g+8, same k) a2=(row g, k 2t+8..2t+9) a3=(row g+8, same);
 // b0=(k 2t..2t+1, col g) b1=(k 2t+8..2t+9, col g); c0,c1=(row g, cols 2t,2t+1) c2,c3=(row g+8).

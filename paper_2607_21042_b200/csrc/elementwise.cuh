@@ -67,6 +67,8 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_kernel(const float *__re
                                                                uint16_t *__restrict__ out, const int *gather,
                                                                const int *out_slot, const StepIO *io) {
   __shared__ float sm[kLnThreads / 32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int j = blockIdx.x;
   const int r = gather ? gather[j] : j;
   const float *xr = x + (size_t)r * d;
@@ -133,6 +135,8 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const SampleArgs
   __shared__ float sel_v[kMaxTopK]; __shared__ int sel_i[kMaxTopK];
   __shared__ float srt_v[kMaxTopK]; __shared__ int srt_i[kMaxTopK];
 
+  pdl_launch_dependents();
+  pdl_wait();
   const int j = blockIdx.x;
   const int slot = a.out_slot ? a.out_slot[j] : j;
   const int V = a.V;

@@ -1,50 +1,56 @@
 // Weight-only dequantizing linear (Table I caption: W8A16 / W4A16 applied to the GPT; bf16 is the
 // unquantized case): out[b,n] = sum_k W[n,k] act[b,k] (+ bias, + epilogue), bf16 activations,
-// fp32 accumulation.
+// fp32 accumulation, optional LayerNorm of the fp32 input fused in front.
 //
-// Streaming layout.  At engine creation every [N,K] matrix is re-laid into 1 KB tiles of 16 output
-// rows x KT columns (KT = 32 bf16 / 64 int8 / 128 int4, i.e. always 1 KB), stored tile after tile
-// as [row-tile nt][k-tile kb].  Inside a tile the bytes sit in the order the warp-level MMA wants
-// its A operand: first 512 B = for lane 0..31 the 16 bytes of row (lane/4) covering columns
-// KT/4*(lane%4) .. +KT/4-1 of the tile, second 512 B = the same for row (lane/4)+8.  A warp then
-// fetches a tile with two fully coalesced 128-bit loads per lane and feeds registers straight to
-// the tensor pipe; int8 / int4 codes are widened to bf16 integers in registers (exact) and the
-// bf16 scale multiplies the fp32 partial sums (per row for int8, per row and 128-column group for
-// int4).  A CTA owns one 16-row tile and splits K over its warps; partial sums meet in shared
-// memory in a fixed order, so results do not depend on timing.
+// Streaming layout.  At engine creation every [N,K] matrix is re-laid into 512-byte tiles of 8
+// output rows x KT columns (KT = 32 bf16 / 64 int8 / 128 int4), stored tile after tile as
+// [row-tile][k-tile].  Inside a tile lane (g,t) = (lane/4, lane%4) owns the 16 bytes of row g that
+// cover columns t*KT/4 .. +KT/4-1: one coalesced 128-bit load per lane fetches a tile in the order
+// the warp-level MMA wants its 8-wide operand.  The batch is the 16-wide M operand (rows 0..15 of
+// an m-tile), the 8 weight rows the N operand; int8 / int4 codes are widened to bf16 integers in
+// registers (exact) and the bf16 scale multiplies the fp32 partial sums (per row for int8, per row
+// and 128-column group for int4).
+//
+// A CTA owns one 8-row tile and splits K over its 10 warps.  Every lane loads ALL of its weights
+// into registers before anything else — weights do not depend on the previous kernel, so under
+// programmatic dependent launch these loads overlap the predecessor's tail — then waits for the
+// predecessor, builds the activation fragments, runs the MMAs, and the warps' partial sums meet in
+// shared memory in warp order (results do not depend on timing).  Batches above 16 loop over
+// m-tiles re-using the weight registers.
 #pragma once
 #include "common.cuh"
+#include "elementwise.cuh"
 
 namespace ttsgpt {
 
 enum { WF_BF16 = 0, WF_INT8 = 1, WF_INT4 = 2 };
 enum { EPI_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_GELU = 3 };
 
-constexpr int kLinearThreads = 320;  // 10 warps: divides the k-tile counts of K=1280 and K=5120
+constexpr int kLinearWarps = 10;  // divides the k-tile counts of K=1280 and K=5120 in every format
+constexpr int kLinearThreads = kLinearWarps * 32;
+constexpr int kLnFuseMaxRows = 16;  // LayerNorm is fused into the linear up to this batch
 
 __host__ __device__ inline int k_per_tile(int wf) { return wf == WF_BF16 ? 32 : (wf == WF_INT8 ? 64 : 128); }
-__host__ __device__ inline int row_tiles(int N) { return (N + 15) / 16; }
+__host__ __device__ inline int row_tiles(int N) { return (N + 7) / 8; }
 // bytes of the tiled weights / of the tiled scales
-inline size_t packed_weight_bytes(int wf, int N, int K) { return (size_t)row_tiles(N) * (K / k_per_tile(wf)) * 1024; }
+inline size_t packed_weight_bytes(int wf, int N, int K) { return (size_t)row_tiles(N) * (K / k_per_tile(wf)) * 512; }
 inline size_t packed_scale_bytes(int wf, int N, int K) {
-  if (wf == WF_INT8) return (size_t)row_tiles(N) * 16 * 2;
-  if (wf == WF_INT4) return (size_t)row_tiles(N) * (K / 128) * 16 * 2;
+  if (wf == WF_INT8) return (size_t)row_tiles(N) * 8 * 2;
+  if (wf == WF_INT4) return (size_t)row_tiles(N) * (K / 128) * 8 * 2;
   return 0;
 }
 
 // ------------------------------------------------------------------------------------------
-// canonical -> streaming re-layout (run once at creation)
+// canonical -> streaming re-layout (run once at creation).  One thread per 16-byte unit.
 // ------------------------------------------------------------------------------------------
-// One thread per 16-byte unit of the destination.
 __global__ void pack_bf16_kernel(const uint16_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
   const int KB = K / 32;
   size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t total = (size_t)row_tiles(N) * KB * 64;
-  if (unit >= total) return;
-  int lane = unit & 31, half = (unit >> 5) & 1;
-  size_t tile = unit >> 6;
-  int kb = tile % KB, nt = tile / KB;
-  int row = nt * 16 + (lane >> 2) + 8 * half, k = kb * 32 + 8 * (lane & 3);
+  if (unit >= (size_t)row_tiles(N) * KB * 32) return;
+  const int lane = unit & 31;
+  const size_t tile = unit >> 5;
+  const int kb = tile % KB, rt = tile / KB;
+  const int row = rt * 8 + (lane >> 2), k = kb * 32 + 8 * (lane & 3);
   uint4 v = make_uint4(0, 0, 0, 0);
   if (row < N) v = *reinterpret_cast<const uint4 *>(w + (size_t)row * K + k);
   dst[unit] = v;
@@ -55,12 +61,11 @@ __global__ void pack_bf16_kernel(const uint16_t *__restrict__ w, int N, int K, u
 __global__ void pack_int8_kernel(const int8_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
   const int KB = K / 64;
   size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t total = (size_t)row_tiles(N) * KB * 64;
-  if (unit >= total) return;
-  int lane = unit & 31, half = (unit >> 5) & 1;
-  size_t tile = unit >> 6;
-  int kb = tile % KB, nt = tile / KB;
-  int row = nt * 16 + (lane >> 2) + 8 * half, k = kb * 64 + 16 * (lane & 3);
+  if (unit >= (size_t)row_tiles(N) * KB * 32) return;
+  const int lane = unit & 31;
+  const size_t tile = unit >> 5;
+  const int kb = tile % KB, rt = tile / KB;
+  const int row = rt * 8 + (lane >> 2), k = kb * 64 + 16 * (lane & 3);
   uint4 v = make_uint4(0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u);
   if (row < N) {
     v = *reinterpret_cast<const uint4 *>(w + (size_t)row * K + k);
@@ -76,8 +81,8 @@ __device__ __forceinline__ uint32_t permute_nibbles(uint32_t c) {
   uint32_t r = 0;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    uint32_t nib = (c >> (4 * j)) & 15u;
-    int pos = (j >> 1) + 4 * (j & 1);
+    const uint32_t nib = (c >> (4 * j)) & 15u;
+    const int pos = (j >> 1) + 4 * (j & 1);
     r |= nib << (4 * pos);
   }
   return r;
@@ -85,28 +90,26 @@ __device__ __forceinline__ uint32_t permute_nibbles(uint32_t c) {
 __global__ void pack_int4_kernel(const uint32_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
   const int KB = K / 128;
   size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t total = (size_t)row_tiles(N) * KB * 64;
-  if (unit >= total) return;
-  int lane = unit & 31, half = (unit >> 5) & 1;
-  size_t tile = unit >> 6;
-  int kb = tile % KB, nt = tile / KB;
-  int row = nt * 16 + (lane >> 2) + 8 * half, k = kb * 128 + 32 * (lane & 3);
+  if (unit >= (size_t)row_tiles(N) * KB * 32) return;
+  const int lane = unit & 31;
+  const size_t tile = unit >> 5;
+  const int kb = tile % KB, rt = tile / KB;
+  const int row = rt * 8 + (lane >> 2), k = kb * 128 + 32 * (lane & 3);
   uint4 v = make_uint4(0x88888888u, 0x88888888u, 0x88888888u, 0x88888888u);
   if (row < N) {
-    uint4 c = *reinterpret_cast<const uint4 *>(w + (size_t)row * (K / 8) + k / 8);
+    const uint4 c = *reinterpret_cast<const uint4 *>(w + (size_t)row * (K / 8) + k / 8);
     v = make_uint4(permute_nibbles(c.x), permute_nibbles(c.y), permute_nibbles(c.z), permute_nibbles(c.w));
   }
   dst[unit] = v;
 }
-// scales: int8 [N] -> [nt][16]; int4 [N][K/128] -> [nt][kb][16]; padding rows get 0
+// scales: int8 [N] -> [rt][8]; int4 [N][K/128] -> [rt][kb][8]; padding rows get 0
 __global__ void pack_scales_kernel(const uint16_t *__restrict__ s, int N, int G, uint16_t *__restrict__ dst) {
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  size_t total = (size_t)row_tiles(N) * G * 16;
-  if (i >= total) return;
-  int r = i & 15;
-  size_t t = i >> 4;
-  int g = t % G, nt = t / G;
-  int row = nt * 16 + r;
+  if (i >= (size_t)row_tiles(N) * G * 8) return;
+  const int r = i & 7;
+  const size_t t = i >> 3;
+  const int g = t % G, rt = t / G;
+  const int row = rt * 8 + r;
   dst[i] = row < N ? s[(size_t)row * G + g] : (uint16_t)0;
 }
 
@@ -117,8 +120,15 @@ struct LinearArgs {
   const void *w;          // tiled weights
   const uint16_t *scales; // tiled scales (int8 / int4) or null
   const uint16_t *bias;   // bf16 [N] or null
-  const uint16_t *act;    // bf16 [B][K]
+  const uint16_t *act;    // bf16 [B][K]  (unused when ln_x is set)
   int N, K, B, mode;
+  // fused LayerNorm in front (B <= kLnFuseMaxRows, K <= kLnFuseMaxK): act = LN(ln_x[gather[b]])
+  const float *ln_x;      // fp32 [*][K] or null
+  const uint16_t *ln_g, *ln_b;
+  float ln_eps;
+  const int *ln_gather;   // optional row indices into ln_x
+  const int *ln_out_slot; // with ln_io: row of io->out_hidden that receives LN row b
+  const StepIO *ln_io;    // optional: CTA 0 also writes the LN rows to io->out_hidden
   float *out_f32;         // EPI_F32: out[b*out_stride+n] = v ; EPI_RESID: out[b*out_stride+n] += v ; EPI_QKV: q
   int out_stride;
   uint16_t *out_bf16;     // EPI_GELU: h[b*N+n] = bf16(gelu(v))
@@ -127,11 +137,13 @@ struct LinearArgs {
   uint16_t *kv_layer;
   const int *page_table, *row_stream, *row_pos;
   int pps, d, H;
+  unsigned long long *trace;  // optional timeline trace (see trace_mark)
+  int trace_slot;
 };
 
 // exact int8 (biased byte) -> float via the 2^23 magic number
 __device__ __forceinline__ float biased_byte_to_float(uint32_t word, int i) {
-  uint32_t m = __byte_perm(word, 0x4B000000u, 0x7540u | (uint32_t)i);
+  const uint32_t m = __byte_perm(word, 0x4B000000u, 0x7540u | (uint32_t)i);
   return __uint_as_float(m) - 8388736.0f;  // 2^23 + 128
 }
 // exact int4 pair (two nibbles in the low bits of each half-word) -> bf16x2 of (u - 8)
@@ -143,128 +155,304 @@ __device__ __forceinline__ uint32_t nib_pair_to_bf16x2(uint32_t masked) {
   return *reinterpret_cast<uint32_t *>(&v);
 }
 
-template <int WF, int NT>
-__global__ void __launch_bounds__(kLinearThreads) linear_kernel(const LinearArgs a) {
+// row stride (in bf16 elements) of the LayerNorm staging buffer; the odd multiple of 16 bytes keeps
+// the 8 batch rows of a fragment load on different banks
+__host__ __device__ inline int ln_stage_stride(int wf, int K) { return K + (wf == WF_BF16 ? 32 : 8); }
+
+// MODE: how the activation fragments are obtained
+//   ACT_DIRECT  bf16 activations read from global memory, a few k-tiles at a time (large B*K)
+//   ACT_STAGED  bf16 activations copied to shared memory first (one round trip for the whole CTA)
+//   ACT_LN      fp32 rows layer-normalised into shared memory first
+enum { ACT_DIRECT = 0, ACT_STAGED = 1, ACT_LN = 2 };
+constexpr int kStageMaxBytes = 44 * 1024;
+
+template <int WF, int KPW, int RT, int MODE>
+__global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearArgs a) {
+  constexpr bool LN = MODE == ACT_LN;
+  constexpr bool STAGED = MODE != ACT_DIRECT;
   constexpr int KT = WF == WF_BF16 ? 32 : (WF == WF_INT8 ? 64 : 128);
-  constexpr int AW = KT / 32;  // uint4 activation loads per lane, tile and batch row
-  extern __shared__ float red[];  // [nwarps][16][NT*8]
-  const int nt = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nwarps = blockDim.x >> 5;
+  constexpr int AW = KT / 32;  // uint4 activation loads per lane, k-tile and batch row
+  constexpr int C = 8 * RT;    // output columns (weight rows) of this CTA
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float *red = reinterpret_cast<float *>(smem_raw);                                       // [warps][16][C]
+  uint16_t *stage = reinterpret_cast<uint16_t *>(smem_raw + kLinearWarps * 16 * C * 4);   // LN rows
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int KB = a.K / KT;
-  const uint4 *wt = reinterpret_cast<const uint4 *>(a.w) + (size_t)nt * KB * 64;
-  const uint16_t *sc = a.scales;
+  const int tile0 = blockIdx.x * RT, n_rt = row_tiles(a.N);
+  trace_mark(a.trace, a.trace_slot, 0);
 
-  for (int b0 = 0; b0 < a.B; b0 += NT * 8) {
-    float acc[NT][4];
+  // ---- all weights of this lane into registers (independent of the previous kernel) ----
+  uint4 wr[RT][KPW];
+  uint32_t sc2[RT][KPW];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-
-#pragma unroll 4
-    for (int kb = warp; kb < KB; kb += nwarps) {
-      const uint4 wa = ld_stream_u4(wt + (size_t)kb * 64 + lane);
-      const uint4 wb = ld_stream_u4(wt + (size_t)kb * 64 + 32 + lane);
-      uint4 xa[NT][AW];
+  for (int j = 0; j < RT; ++j) {
+    const int rt = tile0 + j;
+    const uint4 *wt = reinterpret_cast<const uint4 *>(a.w) + (size_t)rt * KB * 32;
 #pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        const int b = b0 + 8 * j + g;
-#pragma unroll
-        for (int q = 0; q < AW; ++q) {
-          xa[j][q] = make_uint4(0, 0, 0, 0);
-          if (b < a.B)
-            xa[j][q] = *reinterpret_cast<const uint4 *>(a.act + (size_t)b * a.K + (size_t)kb * KT + t * (KT / 4) + 8 * q);
-        }
-      }
-      if (WF == WF_BF16) {
-#pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          mma_bf16_16816(acc[j], wa.x, wb.x, wa.y, wb.y, xa[j][0].x, xa[j][0].y);
-          mma_bf16_16816(acc[j], wa.z, wb.z, wa.w, wb.w, xa[j][0].z, xa[j][0].w);
-        }
-      } else if (WF == WF_INT8) {
-        const uint32_t wwa[4] = {wa.x, wa.y, wa.z, wa.w}, wwb[4] = {wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-        for (int s = 0; s < 4; ++s) {
-          const uint32_t a0 = pack_bf16x2(biased_byte_to_float(wwa[s], 0), biased_byte_to_float(wwa[s], 1));
-          const uint32_t a2 = pack_bf16x2(biased_byte_to_float(wwa[s], 2), biased_byte_to_float(wwa[s], 3));
-          const uint32_t a1 = pack_bf16x2(biased_byte_to_float(wwb[s], 0), biased_byte_to_float(wwb[s], 1));
-          const uint32_t a3 = pack_bf16x2(biased_byte_to_float(wwb[s], 2), biased_byte_to_float(wwb[s], 3));
-#pragma unroll
-          for (int j = 0; j < NT; ++j) {
-            const uint4 x = xa[j][s >> 1];
-            const uint32_t b0r = (s & 1) ? x.z : x.x, b1r = (s & 1) ? x.w : x.y;
-            mma_bf16_16816(acc[j], a0, a1, a2, a3, b0r, b1r);
-          }
-        }
-      } else {
-        float tmp[NT][4];
-#pragma unroll
-        for (int j = 0; j < NT; ++j) tmp[j][0] = tmp[j][1] = tmp[j][2] = tmp[j][3] = 0.f;
-        const uint32_t wwa[4] = {wa.x, wa.y, wa.z, wa.w}, wwb[4] = {wb.x, wb.y, wb.z, wb.w};
-#pragma unroll
-        for (int wd = 0; wd < 4; ++wd) {
-#pragma unroll
-          for (int hs = 0; hs < 2; ++hs) {  // the word's two MMA steps
-            const uint32_t ua = wwa[wd] >> (8 * hs), ub = wwb[wd] >> (8 * hs);
-            const uint32_t a0 = nib_pair_to_bf16x2(ua & 0x000F000Fu);
-            const uint32_t a2 = nib_pair_to_bf16x2((ua >> 4) & 0x000F000Fu);
-            const uint32_t a1 = nib_pair_to_bf16x2(ub & 0x000F000Fu);
-            const uint32_t a3 = nib_pair_to_bf16x2((ub >> 4) & 0x000F000Fu);
-#pragma unroll
-            for (int j = 0; j < NT; ++j) {
-              const uint4 x = xa[j][wd];
-              const uint32_t b0r = hs ? x.z : x.x, b1r = hs ? x.w : x.y;
-              mma_bf16_16816(tmp[j], a0, a1, a2, a3, b0r, b1r);
-            }
-          }
-        }
-        const float s_lo = bf16_bits_to_float(sc[((size_t)nt * KB + kb) * 16 + g]);
-        const float s_hi = bf16_bits_to_float(sc[((size_t)nt * KB + kb) * 16 + g + 8]);
-#pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          acc[j][0] = fmaf(s_lo, tmp[j][0], acc[j][0]);
-          acc[j][1] = fmaf(s_lo, tmp[j][1], acc[j][1]);
-          acc[j][2] = fmaf(s_hi, tmp[j][2], acc[j][2]);
-          acc[j][3] = fmaf(s_hi, tmp[j][3], acc[j][3]);
-        }
+    for (int i = 0; i < KPW; ++i) {
+      const int kb = warp + i * kLinearWarps;
+      wr[j][i] = make_uint4(0, 0, 0, 0);
+      sc2[j][i] = 0u;
+      if (rt < n_rt && kb < KB) {
+        wr[j][i] = ld_stream_u4(wt + (size_t)kb * 32 + lane);
+        if (WF == WF_INT4) sc2[j][i] = *reinterpret_cast<const uint32_t *>(a.scales + ((size_t)rt * KB + kb) * 8 + 2 * t);
       }
     }
-
-    // partial sums of the warps meet in shared memory and are added in warp order
-    constexpr int C = NT * 8;
+  }
+  // ---- everything else that no kernel of the step writes: LN gamma/beta, bias, scales, KV slots ----
+  const int ecol = threadIdx.x % C;             // this thread's output column in every epilogue round
+  const int en = tile0 * 8 + ecol;              // = output feature n
+  float e_bias = 0.f, e_scale = 1.f;
+  if (en < a.N) {
+    if (a.bias) e_bias = bf16_bits_to_float(a.bias[en]);
+    if (WF == WF_INT8) e_scale = bf16_bits_to_float(a.scales[en]);
+  }
+  // EPI_QKV: where this thread's K/V outputs go (row table and page table are final before the
+  // first kernel of the step starts); batches above 16 rows look the slot up in the epilogue
+  constexpr int ER = (16 * C + kLinearThreads - 1) / kLinearThreads;  // epilogue rounds
+  uint16_t *kv_dst[ER];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      float *r0 = red + ((size_t)warp * 16 + g) * C + 8 * j + 2 * t;
-      float *r1 = red + ((size_t)warp * 16 + g + 8) * C + 8 * j + 2 * t;
-      r0[0] = acc[j][0]; r0[1] = acc[j][1];
-      r1[0] = acc[j][2]; r1[1] = acc[j][3];
+  for (int e = 0; e < ER; ++e) {
+    kv_dst[e] = nullptr;
+    const int b = (threadIdx.x + e * kLinearThreads) / C;
+    if (a.mode == EPI_QKV && en >= a.d && en < a.N && b < a.B && b < 16) {
+      const int which = en >= 2 * a.d;  // 0 = K, 1 = V
+      const int col = en - (which ? 2 * a.d : a.d);
+      const int pos = a.row_pos[b];
+      const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
+      kv_dst[e] = a.kv_layer + (((size_t)page * 2 + which) * a.H + (col >> 6)) * kPageElems +
+                  (size_t)(pos & 63) * kHeadDim + (col & 63);
+    }
+  }
+  uint2 ln_gg = make_uint2(0, 0), ln_bb = make_uint2(0, 0);
+  const int lc = threadIdx.x * 4;               // fused LN: this thread's 4 columns (K <= 1280)
+  if (LN && lc < a.K) {
+    ln_gg = *reinterpret_cast<const uint2 *>(a.ln_g + lc);
+    ln_bb = *reinterpret_cast<const uint2 *>(a.ln_b + lc);
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+
+  // ---- optional fused LayerNorm: the CTA splits each row over all threads (4 columns each) and
+  //      handles up to 4 rows per round.  Each thread forms the mean and the centered sum of
+  //      squares of its 4 values; (mean, M2) pairs of equal weight are then merged pairwise
+  //      (mean = (ma+mb)/2, M2 = M2a + M2b + (mb-ma)^2 * n/2), first by shuffles, then across the
+  //      warps through shared memory: one block barrier, no cancellation.
+  const int stride = ln_stage_stride(WF, a.K);
+  if (LN) {
+    float2 *lnred = reinterpret_cast<float2 *>(red);  // [warps][4] (mean, M2), reused later for the partial sums
+    const int nw_used = (a.K / 4 + 31) / 32;           // warps that hold columns (K is a multiple of 128)
+    const float inv_nw = 1.0f / nw_used, inv_k = 1.0f / a.K;
+    for (int b0 = 0; b0 < a.B; b0 += 4) {
+      float4 xv[4];
+      float mean[4], m2[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        xv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int b = b0 + r;
+        if (b < a.B && lc < a.K) {
+          const int src = a.ln_gather ? a.ln_gather[b] : b;
+          xv[r] = *reinterpret_cast<const float4 *>(a.ln_x + (size_t)src * a.K + lc);
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        mean[r] = 0.f; m2[r] = 0.f;
+        if (b0 + r >= a.B) break;
+        mean[r] = 0.25f * ((xv[r].x + xv[r].y) + (xv[r].z + xv[r].w));
+        const float d0 = xv[r].x - mean[r], d1 = xv[r].y - mean[r], d2 = xv[r].z - mean[r], d3 = xv[r].w - mean[r];
+        m2[r] = (d0 * d0 + d1 * d1) + (d2 * d2 + d3 * d3);
+        float cnt = 4.f;  // values behind each side of a merge
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const float mb = __shfl_xor_sync(0xFFFFFFFFu, mean[r], o);
+          const float qb = __shfl_xor_sync(0xFFFFFFFFu, m2[r], o);
+          const float dl = mb - mean[r];
+          m2[r] = m2[r] + qb + dl * dl * (0.5f * cnt);
+          mean[r] = 0.5f * (mean[r] + mb);
+          cnt *= 2.f;
+        }
+      }
+      if (lane < 4) {
+        const float mm = lane == 0 ? mean[0] : (lane == 1 ? mean[1] : (lane == 2 ? mean[2] : mean[3]));
+        const float qq = lane == 0 ? m2[0] : (lane == 1 ? m2[1] : (lane == 2 ? m2[2] : m2[3]));
+        lnred[warp * 4 + lane] = make_float2(mm, qq);
+      }
+      __syncthreads();
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int b = b0 + r;
+        if (b >= a.B) break;
+        // merge of the warps' (mean, M2), each over 128 values: the grand mean is the mean of the
+        // warp means, M2 = sum M2_w + 128 * sum (mean_w - mean)^2
+        float msum = 0.f;
+        for (int w = 0; w < nw_used; ++w) msum += lnred[w * 4 + r].x;
+        float2 acc0;
+        acc0.x = msum * inv_nw;
+        acc0.y = 0.f;
+        for (int w = 0; w < nw_used; ++w) {
+          const float2 o2 = lnred[w * 4 + r];
+          const float dl = o2.x - acc0.x;
+          acc0.y += o2.y + 128.f * dl * dl;
+        }
+        const float mu = acc0.x;
+        const float rstd = rsqrtf(acc0.y * inv_k + a.ln_eps);
+        if (b < a.B && lc < a.K) {
+          uint2 y;
+          y.x = pack_bf16x2((xv[r].x - mu) * rstd * bf16_lo(ln_gg.x) + bf16_lo(ln_bb.x),
+                            (xv[r].y - mu) * rstd * bf16_hi(ln_gg.x) + bf16_hi(ln_bb.x));
+          y.y = pack_bf16x2((xv[r].z - mu) * rstd * bf16_lo(ln_gg.y) + bf16_lo(ln_bb.y),
+                            (xv[r].w - mu) * rstd * bf16_hi(ln_gg.y) + bf16_hi(ln_bb.y));
+          *reinterpret_cast<uint2 *>(stage + (size_t)b * stride + lc) = y;
+          if (blockIdx.x == 0 && a.ln_io && a.ln_io->out_hidden)
+            *reinterpret_cast<uint2 *>(a.ln_io->out_hidden + (size_t)(a.ln_out_slot ? a.ln_out_slot[b] : b) * a.K + lc) = y;
+        }
+      }
+      __syncthreads();
+    }
+  }
+
+  if (MODE == ACT_STAGED) {
+    const int k8 = a.K >> 3;
+    for (int idx = threadIdx.x; idx < a.B * k8; idx += kLinearThreads) {
+      const int b = idx / k8, c8 = idx - b * k8;
+      *reinterpret_cast<uint4 *>(stage + (size_t)b * stride + 8 * c8) =
+          *reinterpret_cast<const uint4 *>(a.act + (size_t)b * a.K + 8 * c8);
     }
     __syncthreads();
-    if (threadIdx.x < 16 * C) {
-      const int r = threadIdx.x / C, c = threadIdx.x % C;
-      const int n = nt * 16 + r, b = b0 + c;
-      if (n < a.N && b < a.B) {
+  }
+
+  trace_mark(a.trace, a.trace_slot, 3);
+  for (int m0 = 0; m0 < a.B; m0 += 16) {
+    // two accumulator sets per row tile (k-tiles alternate between them) shorten the dependent MMA chain
+    float acc2[2][RT][4];
+#pragma unroll
+    for (int j = 0; j < RT; ++j)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc2[0][j][q] = acc2[1][j][q] = 0.f;
+    const int r0 = m0 + g, r1 = m0 + g + 8;
+    const uint16_t *row0 = STAGED ? stage + (size_t)r0 * stride : a.act + (size_t)r0 * a.K;
+    const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K;
+    const bool v0 = r0 < a.B, v1 = r1 < a.B;
+    // the residual's old value, fetched while the MMAs run
+    float e_old[ER];
+#pragma unroll
+    for (int e = 0; e < ER; ++e) {
+      e_old[e] = 0.f;
+      const int o = threadIdx.x + e * kLinearThreads;
+      const int b = m0 + o / C;
+      if (a.mode == EPI_RESID && o < 16 * C && b < a.B && en < a.N) e_old[e] = a.out_f32[(size_t)b * a.out_stride + en];
+    }
+    // activation fragments: G k-tiles are fetched together so that their latencies overlap
+    constexpr int G = STAGED ? 1 : ((4 / AW) < KPW ? (4 / AW) : KPW);
+#pragma unroll
+    for (int i0 = 0; i0 < KPW; i0 += G) {
+      uint4 xg0[G][AW], xg1[G][AW];
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) {
+        const int kb = warp + (i0 + gi) * kLinearWarps;
+        const int col = kb * KT + t * (KT / 4);
+#pragma unroll
+        for (int q = 0; q < AW; ++q) {
+          xg0[gi][q] = (v0 && kb < KB) ? *reinterpret_cast<const uint4 *>(row0 + col + 8 * q) : make_uint4(0, 0, 0, 0);
+          xg1[gi][q] = (v1 && kb < KB) ? *reinterpret_cast<const uint4 *>(row1 + col + 8 * q) : make_uint4(0, 0, 0, 0);
+        }
+      }
+#pragma unroll
+      for (int gi = 0; gi < G; ++gi) {
+      const int i = i0 + gi;
+      const int kb = warp + i * kLinearWarps;
+      float (*acc)[4] = acc2[i & 1];
+      if (kb < KB) {
+        const uint4 *x0 = xg0[gi], *x1 = xg1[gi];
+#pragma unroll
+        for (int j = 0; j < RT; ++j) {
+          const uint32_t ww[4] = {wr[j][i].x, wr[j][i].y, wr[j][i].z, wr[j][i].w};
+          if (WF == WF_BF16) {
+            mma_bf16_16816(acc[j], x0[0].x, x1[0].x, x0[0].y, x1[0].y, ww[0], ww[1]);
+            mma_bf16_16816(acc[j], x0[0].z, x1[0].z, x0[0].w, x1[0].w, ww[2], ww[3]);
+          } else if (WF == WF_INT8) {
+#pragma unroll
+            for (int s = 0; s < 4; ++s) {
+              const uint32_t b0 = pack_bf16x2(biased_byte_to_float(ww[s], 0), biased_byte_to_float(ww[s], 1));
+              const uint32_t b1 = pack_bf16x2(biased_byte_to_float(ww[s], 2), biased_byte_to_float(ww[s], 3));
+              const uint4 xa = x0[s >> 1], xb = x1[s >> 1];
+              if (s & 1) mma_bf16_16816(acc[j], xa.z, xb.z, xa.w, xb.w, b0, b1);
+              else mma_bf16_16816(acc[j], xa.x, xb.x, xa.y, xb.y, b0, b1);
+            }
+          } else {
+            float tmp[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {
+              const uint4 xa = x0[wd], xb = x1[wd];
+              {
+                const uint32_t b0 = nib_pair_to_bf16x2(ww[wd] & 0x000F000Fu);
+                const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 4) & 0x000F000Fu);
+                mma_bf16_16816(tmp, xa.x, xb.x, xa.y, xb.y, b0, b1);
+              }
+              {
+                const uint32_t b0 = nib_pair_to_bf16x2((ww[wd] >> 8) & 0x000F000Fu);
+                const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 12) & 0x000F000Fu);
+                mma_bf16_16816(tmp, xa.z, xb.z, xa.w, xb.w, b0, b1);
+              }
+            }
+            const float s_lo = bf16_lo(sc2[j][i]), s_hi = bf16_hi(sc2[j][i]);  // weight rows 2t, 2t+1
+            acc[j][0] = fmaf(s_lo, tmp[0], acc[j][0]);
+            acc[j][1] = fmaf(s_hi, tmp[1], acc[j][1]);
+            acc[j][2] = fmaf(s_lo, tmp[2], acc[j][2]);
+            acc[j][3] = fmaf(s_hi, tmp[3], acc[j][3]);
+          }
+        }
+      }
+      }
+    }
+
+    trace_mark(a.trace, a.trace_slot, 4);
+    // partial sums of the warps meet in shared memory and are added in warp order
+    float acc[RT][4];
+#pragma unroll
+    for (int j = 0; j < RT; ++j)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[j][q] = acc2[0][j][q] + acc2[1][j][q];
+#pragma unroll
+    for (int j = 0; j < RT; ++j) {
+      *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g) * C + 8 * j + 2 * t) = make_float2(acc[j][0], acc[j][1]);
+      *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g + 8) * C + 8 * j + 2 * t) = make_float2(acc[j][2], acc[j][3]);
+    }
+    __syncthreads();
+    trace_mark(a.trace, a.trace_slot, 5);
+#pragma unroll
+    for (int e = 0; e < ER; ++e) {
+      const int o = threadIdx.x + e * kLinearThreads;
+      const int bl = o / C;
+      const int n = en, b = m0 + bl;
+      if (o < 16 * C && n < a.N && b < a.B) {
         float v = 0.f;
-        for (int w = 0; w < nwarps; ++w) v += red[((size_t)w * 16 + r) * C + c];
-        if (WF == WF_INT8) v *= bf16_bits_to_float(sc[(size_t)nt * 16 + r]);
-        if (a.bias) v += bf16_bits_to_float(a.bias[n]);
+#pragma unroll
+        for (int w = 0; w < kLinearWarps; ++w) v += red[((size_t)w * 16 + bl) * C + ecol];
+        if (WF == WF_INT8) v *= e_scale;
+        v += e_bias;
         if (a.mode == EPI_F32) {
           a.out_f32[(size_t)b * a.out_stride + n] = v;
         } else if (a.mode == EPI_RESID) {
-          a.out_f32[(size_t)b * a.out_stride + n] += v;
+          a.out_f32[(size_t)b * a.out_stride + n] = e_old[e] + v;
         } else if (a.mode == EPI_GELU) {
           v = a.gelu_tanh ? gelu_tanh_f(v) : gelu_erf_f(v);
           a.out_bf16[(size_t)b * a.N + n] = float_to_bf16_bits(v);
         } else {  // EPI_QKV
           if (n < a.d) {
             a.out_f32[(size_t)b * a.out_stride + n] = v;
+          } else if (m0 == 0) {
+            *kv_dst[e] = float_to_bf16_bits(v);
           } else {
             const int which = n >= 2 * a.d;  // 0 = K, 1 = V
             const int col = n - (which ? 2 * a.d : a.d);
-            const int head = col >> 6, e = col & 63;
+            const int head = col >> 6, ee = col & 63;
             const int pos = a.row_pos[b];
             const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
-            a.kv_layer[(((size_t)page * 2 + which) * a.H + head) * kPageElems + (size_t)(pos & 63) * kHeadDim + e] =
+            a.kv_layer[(((size_t)page * 2 + which) * a.H + head) * kPageElems + (size_t)(pos & 63) * kHeadDim + ee] =
                 float_to_bf16_bits(v);
           }
         }
@@ -272,30 +460,90 @@ __global__ void __launch_bounds__(kLinearThreads) linear_kernel(const LinearArgs
     }
     __syncthreads();
   }
+  trace_mark(a.trace, a.trace_slot, 2);
 }
 
-inline cudaError_t launch_linear(int wf, const LinearArgs &a, cudaStream_t st) {
-  const int grid = row_tiles(a.N);
-  const int nt = a.B > 8 ? 2 : 1;
-  const size_t smem = (size_t)(kLinearThreads / 32) * 16 * nt * 8 * sizeof(float);
-#define TTS_LAUNCH(WF, NT) linear_kernel<WF, NT><<<grid, kLinearThreads, smem, st>>>(a)
-  if (wf == WF_BF16) { if (nt == 1) TTS_LAUNCH(WF_BF16, 1); else TTS_LAUNCH(WF_BF16, 2); }
-  else if (wf == WF_INT8) { if (nt == 1) TTS_LAUNCH(WF_INT8, 1); else TTS_LAUNCH(WF_INT8, 2); }
-  else { if (nt == 1) TTS_LAUNCH(WF_INT4, 1); else TTS_LAUNCH(WF_INT4, 2); }
-#undef TTS_LAUNCH
-  return cudaGetLastError();
+// Launch shape: all CTAs of a launch should be resident at once (2 per SM), so that every weight
+// byte of the layer is requested before the kernel waits for its predecessor.
+struct LinearPlan { int rt, grid; };
+inline LinearPlan plan_linear(int N, int max_ctas) {
+  const int tiles = row_tiles(N);
+  LinearPlan p;
+  p.rt = 1;
+  while (p.rt < 4 && (tiles + p.rt - 1) / p.rt > max_ctas) p.rt *= 2;
+  p.grid = (tiles + p.rt - 1) / p.rt;
+  return p;
+}
+
+template <int WF, int KPW, int RT, int MODE>
+inline cudaError_t launch_linear_inst(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
+  size_t smem = (size_t)kLinearWarps * 16 * 8 * RT * sizeof(float);
+  if (MODE != ACT_DIRECT) smem += (size_t)a.B * ln_stage_stride(WF, a.K) * sizeof(uint16_t);
+  static bool attr_done = false;  // opt-in to more than 48 KB of dynamic shared memory, once
+  if (!attr_done) {
+    cudaFuncSetAttribute(linear_kernel<WF, KPW, RT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    attr_done = true;
+  }
+  return launch_kernel(linear_kernel<WF, KPW, RT, MODE>, dim3(grid), dim3(kLinearThreads), smem, st, pdl, a);
+}
+
+template <int WF, int KPW, int MODE>
+inline cudaError_t launch_linear_rt(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
+  if (KPW * p.rt > 16) {  // too many weight registers: fall back to more, smaller CTAs
+    p.rt = 16 / KPW;
+    p.grid = (row_tiles(a.N) + p.rt - 1) / p.rt;
+  }
+  if (p.rt == 1) return launch_linear_inst<WF, KPW, 1, MODE>(a, p.grid, st, pdl);
+  if (p.rt == 2) return launch_linear_inst<WF, KPW, (KPW <= 8 ? 2 : 1), MODE>(a, p.grid, st, pdl);
+  return launch_linear_inst<WF, KPW, (KPW <= 4 ? 4 : 1), MODE>(a, p.grid, st, pdl);
+}
+
+template <int WF, int MODE>
+inline cudaError_t launch_linear_wf(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
+  const int KB = a.K / k_per_tile(WF);
+  const int kpw = (KB + kLinearWarps - 1) / kLinearWarps;
+  if (kpw <= 1) return launch_linear_rt<WF, 1, MODE>(a, p, st, pdl);
+  if (kpw <= 2) return launch_linear_rt<WF, 2, MODE>(a, p, st, pdl);
+  if (kpw <= 4) return launch_linear_rt<WF, 4, MODE>(a, p, st, pdl);
+  if (MODE == ACT_LN) return cudaErrorInvalidValue;  // fused LayerNorm is built for K <= 1280 only
+  if (kpw <= 8) return launch_linear_rt<WF, 8, (MODE == ACT_LN ? ACT_STAGED : MODE)>(a, p, st, pdl);
+  if (kpw <= 16) return launch_linear_rt<WF, 16, (MODE == ACT_LN ? ACT_STAGED : MODE)>(a, p, st, pdl);
+  return cudaErrorInvalidValue;
+}
+
+// Whether LayerNorm can be fused in front of a linear with this shape.
+inline bool can_fuse_ln(int wf, int B, int K) {
+  const int kpw = (K / k_per_tile(wf) + kLinearWarps - 1) / kLinearWarps;
+  return B <= kLnFuseMaxRows && kpw <= 4 && K <= 4 * kLinearThreads;  // one float4 of the row per thread
+}
+
+template <int WF>
+inline cudaError_t launch_linear_mode(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
+  if (a.ln_x) return launch_linear_wf<WF, ACT_LN>(a, p, st, pdl);
+  if ((size_t)a.B * ln_stage_stride(WF, a.K) * sizeof(uint16_t) <= (size_t)kStageMaxBytes)
+    return launch_linear_wf<WF, ACT_STAGED>(a, p, st, pdl);
+  return launch_linear_wf<WF, ACT_DIRECT>(a, p, st, pdl);
+}
+
+// K must be a multiple of 128 and at most 160 k-tiles (K <= 5120 for bf16).
+inline cudaError_t launch_linear(int wf, const LinearArgs &a, cudaStream_t st, bool pdl = false, int max_ctas = 296) {
+  const LinearPlan p = plan_linear(a.N, max_ctas);
+  if (a.ln_x && !can_fuse_ln(wf, a.B, a.K)) return cudaErrorInvalidValue;
+  if (wf == WF_BF16) return launch_linear_mode<WF_BF16>(a, p, st, pdl);
+  if (wf == WF_INT8) return launch_linear_mode<WF_INT8>(a, p, st, pdl);
+  return launch_linear_mode<WF_INT4>(a, p, st, pdl);
 }
 
 inline cudaError_t launch_pack(int wf, int N, int K, const void *w, const void *s, void *dst_w, void *dst_s,
                                cudaStream_t st) {
-  const size_t units = (size_t)row_tiles(N) * (K / k_per_tile(wf)) * 64;
+  const size_t units = (size_t)row_tiles(N) * (K / k_per_tile(wf)) * 32;
   const int blocks = (int)((units + 255) / 256);
   if (wf == WF_BF16) pack_bf16_kernel<<<blocks, 256, 0, st>>>((const uint16_t *)w, N, K, (uint4 *)dst_w);
   else if (wf == WF_INT8) pack_int8_kernel<<<blocks, 256, 0, st>>>((const int8_t *)w, N, K, (uint4 *)dst_w);
   else pack_int4_kernel<<<blocks, 256, 0, st>>>((const uint32_t *)w, N, K, (uint4 *)dst_w);
   if (wf != WF_BF16) {
     const int G = wf == WF_INT8 ? 1 : K / 128;
-    const size_t n = (size_t)row_tiles(N) * G * 16;
+    const size_t n = (size_t)row_tiles(N) * G * 8;
     pack_scales_kernel<<<(int)((n + 255) / 256), 256, 0, st>>>((const uint16_t *)s, N, G, (uint16_t *)dst_s);
   }
   return cudaGetLastError();

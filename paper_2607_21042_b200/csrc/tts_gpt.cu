@@ -68,7 +68,11 @@ struct tts_gpt {
   std::map<int, cudaGraphExec_t> graphs;
   std::map<int, int> graph_nodes;
   bool use_graph;
-  unsigned long long launches = 0;  // kernels enqueued so far (graph nodes counted per replay)
+  bool use_pdl;
+  int n_sm = 148;
+  unsigned long long launches = 0;
+  unsigned long long *trace = nullptr;  // optional device buffer for kernel timelines
+  int trace_next = 0;  // kernels enqueued so far (graph nodes counted per replay)
 };
 
 namespace {
@@ -200,37 +204,67 @@ LinearArgs linear_args(const PackedLinear &pl, const uint16_t *act, int B, int m
   return a;
 }
 
+// gives the next traced kernel of a step its slot
+template <typename Args>
+void trace_attach(tts_gpt *h, Args &a) {
+  a.trace = h->trace;
+  a.trace_slot = h->trace ? h->trace_next++ : 0;
+}
+
 // The transformer blocks for R rows already described by the row table, x holding the input rows.
-int run_layers(tts_gpt *h, int R) {
+// Every kernel after the first of a step is launched with programmatic dependent launch, so its
+// weight loads overlap the tail of its predecessor.
+int run_layers(tts_gpt *h, int R, bool decode) {
+  h->trace_next = 0;
   const tts_gpt_config_t &c = h->cfg;
   const int d = c.d_model;
   cudaStream_t st = h->stream;
+  const bool pdl = h->use_pdl;
+  const bool fuse_ln = can_fuse_ln(c.wfmt, R, d);
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
-    layernorm_kernel<<<R, kLnThreads, 0, st>>>(h->x, d, L.ln1_g, L.ln1_b, c.ln_eps, h->a, nullptr, nullptr, nullptr);
     LinearArgs qa = linear_args(L.qkv, h->a, R, EPI_QKV);
+    if (fuse_ln) {
+      qa.ln_x = h->x; qa.ln_g = L.ln1_g; qa.ln_b = L.ln1_b; qa.ln_eps = c.ln_eps;
+    } else {
+      CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(R), dim3(kLnThreads), 0, st, pdl, (const float *)h->x, d,
+                                (const uint16_t *)L.ln1_g, (const uint16_t *)L.ln1_b, c.ln_eps, h->a,
+                                (const int *)nullptr, (const int *)nullptr, (const StepIO *)nullptr));
+      h->launches += 1;
+    }
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
-    CUDA_TRY(h, launch_linear(c.wfmt, qa, st));
+    trace_attach(h, qa);
+    CUDA_TRY(h, launch_linear(c.wfmt, qa, st, pdl, 2 * h->n_sm));
     AttnArgs aa;
     aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
     aa.row_pos = h->rt.row_pos; aa.out = h->o; aa.partials = h->attn_partials; aa.tickets = h->attn_tickets;
-    aa.H = c.n_head; aa.pps = h->pps;
-    CUDA_TRY(h, launch_attention(aa, R, c.max_context, st));
+    aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
+    trace_attach(h, aa);
+    CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
     LinearArgs oa = linear_args(L.o, h->o, R, EPI_RESID);
     oa.out_f32 = h->x; oa.out_stride = d;
-    CUDA_TRY(h, launch_linear(c.wfmt, oa, st));
-    layernorm_kernel<<<R, kLnThreads, 0, st>>>(h->x, d, L.ln2_g, L.ln2_b, c.ln_eps, h->a, nullptr, nullptr, nullptr);
+    trace_attach(h, oa);
+    CUDA_TRY(h, launch_linear(c.wfmt, oa, st, pdl, 2 * h->n_sm));
     LinearArgs f1 = linear_args(L.fc1, h->a, R, EPI_GELU);
+    if (fuse_ln) {
+      f1.ln_x = h->x; f1.ln_g = L.ln2_g; f1.ln_b = L.ln2_b; f1.ln_eps = c.ln_eps;
+    } else {
+      CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(R), dim3(kLnThreads), 0, st, pdl, (const float *)h->x, d,
+                                (const uint16_t *)L.ln2_g, (const uint16_t *)L.ln2_b, c.ln_eps, h->a,
+                                (const int *)nullptr, (const int *)nullptr, (const StepIO *)nullptr));
+      h->launches += 1;
+    }
     f1.out_bf16 = h->hbuf; f1.gelu_tanh = c.gelu_tanh;
-    CUDA_TRY(h, launch_linear(c.wfmt, f1, st));
+    trace_attach(h, f1);
+    CUDA_TRY(h, launch_linear(c.wfmt, f1, st, pdl, 2 * h->n_sm));
     LinearArgs f2 = linear_args(L.fc2, h->hbuf, R, EPI_RESID);
     f2.out_f32 = h->x; f2.out_stride = d;
-    CUDA_TRY(h, launch_linear(c.wfmt, f2, st));
+    trace_attach(h, f2);
+    CUDA_TRY(h, launch_linear(c.wfmt, f2, st, pdl, 2 * h->n_sm));
+    h->launches += 5;
   }
-  CUDA_TRY(h, cudaGetLastError());
-  h->launches += 7ull * c.n_layer;
   return TTS_GPT_OK;
 }
 
@@ -238,19 +272,27 @@ int run_layers(tts_gpt *h, int R) {
 int run_head(tts_gpt *h, int n_out) {
   const tts_gpt_config_t &c = h->cfg;
   cudaStream_t st = h->stream;
-  layernorm_kernel<<<n_out, kLnThreads, 0, st>>>(h->x, c.d_model, h->lnf_g, h->lnf_b, c.ln_eps, h->hf,
-                                                 h->rt.out_rows, h->rt.out_slot, h->io);
+  const bool pdl = h->use_pdl;
   LinearArgs ha = linear_args(h->head, h->hf, n_out, EPI_F32);
+  if (can_fuse_ln(WF_BF16, n_out, c.d_model)) {
+    ha.ln_x = h->x; ha.ln_g = h->lnf_g; ha.ln_b = h->lnf_b; ha.ln_eps = c.ln_eps;
+    ha.ln_gather = h->rt.out_rows; ha.ln_out_slot = h->rt.out_slot; ha.ln_io = h->io;
+  } else {
+    CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(n_out), dim3(kLnThreads), 0, st, pdl, (const float *)h->x,
+                              c.d_model, (const uint16_t *)h->lnf_g, (const uint16_t *)h->lnf_b, c.ln_eps, h->hf,
+                              (const int *)h->rt.out_rows, (const int *)h->rt.out_slot, (const StepIO *)h->io));
+    h->launches += 1;
+  }
   ha.out_f32 = h->logits; ha.out_stride = c.vocab;
-  CUDA_TRY(h, launch_linear(WF_BF16, ha, st));
+  trace_attach(h, ha);
+  CUDA_TRY(h, launch_linear(WF_BF16, ha, st, pdl, 2 * h->n_sm));
   SampleArgs sa;
   memset(&sa, 0, sizeof sa);
   sa.logits = h->logits; sa.V = c.vocab; sa.io = h->io; sa.out_slot = h->rt.out_slot; sa.out_rows = h->rt.out_rows;
   sa.row_stream = h->rt.row_stream; sa.last_token = h->ps.last_token; sa.stop_flag = h->ps.stop_flag;
   sa.stop_token = c.stop_token;
-  sample_kernel<<<n_out, kSampleThreads, (size_t)c.vocab * sizeof(float), st>>>(sa);
-  CUDA_TRY(h, cudaGetLastError());
-  h->launches += 3;
+  CUDA_TRY(h, launch_kernel(sample_kernel, dim3(n_out), dim3(kSampleThreads), (size_t)c.vocab * sizeof(float), st, pdl, sa));
+  h->launches += 2;
   return TTS_GPT_OK;
 }
 
@@ -349,6 +391,13 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   const char *ng = getenv("TTS_GPT_NO_GRAPH");
   // the legacy default stream cannot be captured
   h->use_graph = !(ng && ng[0] == '1') && h->stream != nullptr && h->stream != cudaStreamLegacy;
+  {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      h->n_sm = sms;
+  }
+  const char *np = getenv("TTS_GPT_NO_PDL");
+  h->use_pdl = !(np && np[0] == '1');
   *out = h;
   return TTS_GPT_OK;
 }
@@ -407,7 +456,7 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     h->launches += 1;
     int r = run_embed(h, ps.n_rows);
     if (r) return r;
-    r = run_layers(h, ps.n_rows);
+    r = run_layers(h, ps.n_rows, false);
     if (r) return r;
     if (ps.n_out > 0) r = run_head(h, ps.n_out);
     ps.n_rows = 0; ps.n_out = 0;
@@ -469,7 +518,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
       const unsigned long long before = h->launches;
       CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
       rc = run_embed(h, n);
-      if (!rc) rc = run_layers(h, n);
+      if (!rc) rc = run_layers(h, n, true);
       if (!rc) rc = run_head(h, n);
       cudaError_t e = cudaStreamEndCapture(h->stream, &g);
       if (rc) { if (g) cudaGraphDestroy(g); return rc; }
@@ -487,7 +536,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
     return TTS_GPT_OK;
   }
   rc = run_embed(h, n);
-  if (!rc) rc = run_layers(h, n);
+  if (!rc) rc = run_layers(h, n, true);
   if (!rc) rc = run_head(h, n);
   return rc;
 }
@@ -529,6 +578,17 @@ int32_t tts_gpt_stats(const tts_gpt_t *h, int32_t *open_streams, int32_t *free_p
 int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n) {
   if (!h || !n) return fail(nullptr, TTS_GPT_E_ARG, "null argument");
   *n = h->launches;
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second);  // slots are baked into captured graphs
+  h->graphs.clear();
+  h->graph_nodes.clear();
+  h->trace = (unsigned long long *)trace;
+  if (n_slots) *n_slots = 5 * h->cfg.n_layer + 1;
   return TTS_GPT_OK;
 }
 
@@ -585,7 +645,7 @@ int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed
   pl.bias = (uint16_t *)bias;
   LinearArgs a = linear_args(pl, (const uint16_t *)act, B, EPI_F32);
   a.out_f32 = out; a.out_stride = N;
-  CUDA_TRY(nullptr, launch_linear(wfmt, a, (cudaStream_t)cuda_stream));
+  CUDA_TRY(nullptr, launch_linear(wfmt, a, (cudaStream_t)cuda_stream, false));
   return TTS_GPT_OK;
 }
 
@@ -603,10 +663,11 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention: bad argument");
   AttnArgs a;
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
-  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream; a.old_pages_final = 0;
+  a.trace = nullptr; a.trace_slot = 0;
   a.partials = (float *)scratch;
   a.tickets = (unsigned int *)((char *)scratch + align256((size_t)R * n_head * kAttnMaxChunks * kAttnPartialFloats * sizeof(float)));
-  CUDA_TRY(nullptr, launch_attention(a, R, pages_per_stream * kPageTokens, (cudaStream_t)cuda_stream));
+  CUDA_TRY(nullptr, launch_attention_ticket(a, R, pages_per_stream * kPageTokens, (cudaStream_t)cuda_stream));
   return TTS_GPT_OK;
 }
 
@@ -657,12 +718,30 @@ int32_t tts_gpt_op_attention_static(int32_t R, int32_t n_head, const float *q, c
   cudaStream_t st = (cudaStream_t)cuda_stream;
   AttnArgs a;
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
-  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream; a.old_pages_final = 0;
+  a.trace = nullptr; a.trace_slot = 0;
   a.partials = (float *)base;
   a.tickets = (unsigned int *)(base + kStaticAttnPartialBytes);
   // The array keeps whatever the previous call left; the tickets have to start at zero.
   CUDA_TRY(nullptr, cudaMemsetAsync(a.tickets, 0, (size_t)R * n_head * sizeof(unsigned int), st));
-  CUDA_TRY(nullptr, launch_attention(a, R, pages_per_stream * kPageTokens, st));
+  CUDA_TRY(nullptr, launch_attention_ticket(a, R, pages_per_stream * kPageTokens, st));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
+                                     const int32_t *page_table, int32_t pages_per_stream,
+                                     const int32_t *row_stream, const int32_t *row_pos, void *out,
+                                     int32_t cluster_size, void *cuda_stream) {
+  if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
+      pages_per_stream < 1)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
+  if (cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be 1, 2, 4 or 8");
+  AttnArgs a;
+  memset(&a, 0, sizeof a);
+  a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
+  a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  CUDA_TRY(nullptr, launch_attention(a, R, cluster_size, (cudaStream_t)cuda_stream, false));
   return TTS_GPT_OK;
 }
 

@@ -130,6 +130,24 @@ def test_attention_matches_oracle(H, ctxs):
             assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (r, rep)
 
 
+@pytest.mark.parametrize("S", [1, 2, 4, 8])
+def test_attention_cluster_variant_matches_oracle(S):
+    rng = np.random.default_rng(40 + S)
+    H = 5
+    ctxs = [1, 64, 65, 300, 900, 2048, 513, 130]
+    kv, pt, Ks, Vs = _attention_case(rng, H, ctxs, sum((c + 63) // 64 for c in ctxs) + 2, 32)
+    R = len(ctxs)
+    q = (rng.standard_normal(size=(R, H * 64)) * 2.0).astype(np.float32)
+    out = B.op_attention_cluster(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                                 torch.arange(R, dtype=torch.int32, device=DEV),
+                                 torch.from_numpy(np.array([c - 1 for c in ctxs], dtype=np.int32)).to(DEV), S)
+    torch.cuda.synchronize()
+    got = bits_to_f64(out)
+    for r in range(R):
+        ref = _attention_ref(q[r].astype(np.float64), Ks[r], Vs[r], H)
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (r, S)
+
+
 def test_attention_rows_of_one_stream_share_pages():
     # several rows of the same stream at different positions (a prefill pass)
     rng = np.random.default_rng(77)
