@@ -171,13 +171,17 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   // this warp's pages: c + S*(warp + kAttnWarps*it)
   int page = c + S * warp;
   PageLoad pl;
-  // In a decode step every page but the row's last one holds only tokens of earlier steps: the
-  // first page's loads do not depend on the QKV kernel in front and are issued before waiting for it.
-  const bool early = a.old_pages_final && page < n_pages - 1;
+  // In a decode step the only K/V entry of the row that this step writes is the new token's own
+  // (position n_tok-1, by the QKV kernel in front).  The warp's first page is therefore requested
+  // before waiting for that kernel; if it is the row's last page, the new token's 128-byte K and V
+  // rows are fetched again after the wait.
+  const bool early = a.old_pages_final && page < n_pages;
+  const uint16_t *K0 = nullptr, *V0 = nullptr;
   if (early) {
     const int phys = pt[page];
-    load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
-              a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
+    K0 = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
+    V0 = a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems;
+    load_page(pl, K0, V0, tg, sub);
   }
   pdl_launch_dependents();
   pdl_wait();
@@ -189,6 +193,22 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   for (int e = 0; e < 8; ++e) o[e] = 0.f;
   float qv[8];
   load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+  if (early && page == n_pages - 1) {
+    const int tn = (n_tok - 1) & (kPageTokens - 1);   // the new token's slot in its page
+    if ((tn & 3) == tg) {
+      const uint4 kn = ld_cg_u4(K0 + (size_t)tn * kHeadDim + 8 * sub);
+      const uint4 vn = ld_cg_u4(V0 + (size_t)tn * kHeadDim + 8 * sub);
+      const int sel = tn >> 2;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {  // register selects (no dynamic indexing of the page registers)
+        const bool hit = i == sel;
+        pl.kk[i].x = hit ? kn.x : pl.kk[i].x; pl.kk[i].y = hit ? kn.y : pl.kk[i].y;
+        pl.kk[i].z = hit ? kn.z : pl.kk[i].z; pl.kk[i].w = hit ? kn.w : pl.kk[i].w;
+        pl.vv[i].x = hit ? vn.x : pl.vv[i].x; pl.vv[i].y = hit ? vn.y : pl.vv[i].y;
+        pl.vv[i].z = hit ? vn.z : pl.vv[i].z; pl.vv[i].w = hit ? vn.w : pl.vv[i].w;
+      }
+    }
+  }
   bool loaded = early;
   for (; page < n_pages; page += S * kAttnWarps) {
     if (!loaded) {
@@ -218,15 +238,25 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   cluster.sync();
   trace_mark(a.trace, a.trace_slot, 5);
   if (c == 0 && e < kHeadDim) {
+    // all remote reads are issued before any is used
+    float pm[kAttnMaxCluster], pl_[kAttnMaxCluster], po[kAttnMaxCluster];
+#pragma unroll
+    for (int rr = 0; rr < kAttnMaxCluster; ++rr) {
+      pm[rr] = -INFINITY; pl_[rr] = 0.f; po[rr] = 0.f;
+      if (rr < S) {
+        const float *p = cluster.map_shared_rank(cl_part, rr);
+        pm[rr] = p[0]; pl_[rr] = p[1]; po[rr] = p[2 + e];
+      }
+    }
     float MM = -INFINITY;
-    for (int rr = 0; rr < S; ++rr) MM = fmaxf(MM, cluster.map_shared_rank(cl_part, rr)[0]);
+#pragma unroll
+    for (int rr = 0; rr < kAttnMaxCluster; ++rr) MM = fmaxf(MM, pm[rr]);
     float LL = 0.f, OO = 0.f;
-    for (int rr = 0; rr < S; ++rr) {
-      const float *p = cluster.map_shared_rank(cl_part, rr);
-      const float pm = p[0];
-      const float f = (pm == -INFINITY) ? 0.f : exp2f(pm - MM);  // a rank without pages contributes nothing
-      LL = fmaf(p[1], f, LL);
-      OO = fmaf(p[2 + e], f, OO);
+#pragma unroll
+    for (int rr = 0; rr < kAttnMaxCluster; ++rr) {
+      const float f = (pm[rr] == -INFINITY) ? 0.f : exp2f(pm[rr] - MM);  // a rank without pages contributes nothing
+      LL = fmaf(pl_[rr], f, LL);
+      OO = fmaf(po[rr], f, OO);
     }
     out[e] = float_to_bf16_bits(OO / LL);
   }

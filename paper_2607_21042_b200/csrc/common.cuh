@@ -82,6 +82,13 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// 128-bit load served by L2 (never by a possibly stale L1 line).
+__device__ __forceinline__ uint4 ld_cg_u4(const void *p) {
+  uint4 r;
+  asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+
 // D(16x8,f32) += A(16x16,bf16,row) * B(16x8,bf16,col).  Fragment layout (g = lane/4, t = lane%4):
 // a0=(row g, k 2t..2t+1) a1=(row g+8, same k) a2=(row g, k 2t+8..2t+9) a3=(row g+8, same);
 // b0=(k 2t..2t+1, col g) b1=(k 2t+8..2t+9, col g); c0,c1=(row g, cols 2t,2t+1) c2,c3=(row g+8).

@@ -11,12 +11,15 @@
 // registers (exact) and the bf16 scale multiplies the fp32 partial sums (per row for int8, per row
 // and 128-column group for int4).
 //
-// A CTA owns one 8-row tile and splits K over its 10 warps.  Every lane loads ALL of its weights
-// into registers before anything else — weights do not depend on the previous kernel, so under
-// programmatic dependent launch these loads overlap the predecessor's tail — then waits for the
-// predecessor, builds the activation fragments, runs the MMAs, and the warps' partial sums meet in
-// shared memory in warp order (results do not depend on timing).  Batches above 16 loop over
-// m-tiles re-using the weight registers.
+// A CTA owns 1, 2 or 4 adjacent 8-row tiles (one contiguous block of the streaming layout) and
+// splits K over its 10 warps.  Its very first action is one bulk asynchronous copy (TMA, untiled,
+// completion on an mbarrier) of that whole block into shared memory: weights do not depend on the
+// previous kernel, so under programmatic dependent launch the copy overlaps the predecessor's
+// tail and occupies no registers.  Only then does the CTA wait for its predecessor, stage (or
+// layer-normalise) the activation rows, wait for the weights (bounded wait, error word on
+// expiry), form the products — fp32 FMAs for up to 4 batch rows, the tensor pipe above — and the
+// warps' partial sums meet in shared memory in warp order (results do not depend on timing).
+// Batches above 16 loop over m-tiles re-using the weights in shared memory.
 #pragma once
 #include "common.cuh"
 #include "elementwise.cuh"
@@ -139,6 +142,7 @@ struct LinearArgs {
   int pps, d, H;
   unsigned long long *trace;  // optional timeline trace (see trace_mark)
   int trace_slot;
+  int *err;                   // optional device error word: set to 1 if the weight copy never arrives
 };
 
 // exact int8 (biased byte) -> float via the 2^23 magic number
@@ -165,41 +169,82 @@ __host__ __device__ inline int ln_stage_stride(int wf, int K) { return K + (wf =
 //   ACT_LN      fp32 rows layer-normalised into shared memory first
 enum { ACT_DIRECT = 0, ACT_STAGED = 1, ACT_LN = 2 };
 constexpr int kStageMaxBytes = 44 * 1024;
+constexpr int kLinearSmemBudget = 108 * 1024;  // per CTA, so that two CTAs share an SM
 
-template <int WF, int KPW, int RT, int MODE>
+// ---- bulk asynchronous copy (TMA, untiled) of the CTA's weights into shared memory ----
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// both addresses 16-byte aligned, size a multiple of 16
+__device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst_smem)),
+               "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for the barrier's phase, at most about `limit_ns` nanoseconds.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, unsigned long long limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  while (!mbar_try_wait(bar, parity)) {
+    if (global_timer_ns() - t0 > limit_ns) return false;
+  }
+  return true;
+}
+
+// NB: 0 = tensor-pipe path (any batch, 16 rows per m-tile); 1 or 4 = CUDA-core path for batches of
+// at most NB rows.  On this part one warp-level MMA occupies the tensor pipe of its SM partition
+// for about 32 cycles whatever the number of real batch rows, so below 5 rows plain fp32 FMAs on
+// the widened weights are cheaper.
+template <int WF, int RT, int MODE, int NB>
 __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearArgs a) {
   constexpr bool LN = MODE == ACT_LN;
   constexpr bool STAGED = MODE != ACT_DIRECT;
   constexpr int KT = WF == WF_BF16 ? 32 : (WF == WF_INT8 ? 64 : 128);
   constexpr int AW = KT / 32;  // uint4 activation loads per lane, k-tile and batch row
   constexpr int C = 8 * RT;    // output columns (weight rows) of this CTA
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  float *red = reinterpret_cast<float *>(smem_raw);                                       // [warps][16][C]
-  uint16_t *stage = reinterpret_cast<uint16_t *>(smem_raw + kLinearWarps * 16 * C * 4);   // LN rows
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int KB = a.K / KT;
   const int tile0 = blockIdx.x * RT, n_rt = row_tiles(a.N);
   trace_mark(a.trace, a.trace_slot, 0);
 
-  // ---- all weights of this lane into registers (independent of the previous kernel) ----
-  uint4 wr[RT][KPW];
-  uint32_t sc2[RT][KPW];
-#pragma unroll
-  for (int j = 0; j < RT; ++j) {
-    const int rt = tile0 + j;
-    const uint4 *wt = reinterpret_cast<const uint4 *>(a.w) + (size_t)rt * KB * 32;
-#pragma unroll
-    for (int i = 0; i < KPW; ++i) {
-      const int kb = warp + i * kLinearWarps;
-      wr[j][i] = make_uint4(0, 0, 0, 0);
-      sc2[j][i] = 0u;
-      if (rt < n_rt && kb < KB) {
-        wr[j][i] = ld_stream_u4(wt + (size_t)kb * 32 + lane);
-        if (WF == WF_INT4) sc2[j][i] = *reinterpret_cast<const uint32_t *>(a.scales + ((size_t)rt * KB + kb) * 8 + 2 * t);
-      }
-    }
+  // shared memory: [barrier | weights RT*KB*512 | int4 scales RT*KB*16 | partial sums | activation rows]
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  uint64_t *wbar = reinterpret_cast<uint64_t *>(smem_raw);
+  unsigned char *wsm = smem_raw + 128;
+  uint16_t *ssm = reinterpret_cast<uint16_t *>(wsm + (size_t)RT * KB * 512);
+  float *red = reinterpret_cast<float *>(wsm + (size_t)RT * KB * (WF == WF_INT4 ? 528 : 512));  // [warps][16][C]
+  uint16_t *stage = reinterpret_cast<uint16_t *>(red + kLinearWarps * 16 * C);
+
+  // ---- the CTA's weights (contiguous in the streaming layout) start moving into shared memory
+  //      before anything else: they do not depend on the previous kernel ----
+  if (threadIdx.x == 0) {
+    const int n_valid = min(RT, n_rt - tile0);
+    const uint32_t wbytes = (uint32_t)n_valid * KB * 512u;
+    const uint32_t sbytes = WF == WF_INT4 ? (uint32_t)n_valid * KB * 16u : 0u;
+    mbar_init(wbar, 1);
+    mbar_expect_tx(wbar, wbytes + sbytes);
+    const unsigned char *gw = reinterpret_cast<const unsigned char *>(a.w) + (size_t)tile0 * KB * 512;
+    for (uint32_t off = 0; off < wbytes; off += 32768u)
+      bulk_copy_g2s(wsm + off, gw + off, min(32768u, wbytes - off), wbar);
+    if (sbytes) bulk_copy_g2s(ssm, a.scales + (size_t)tile0 * KB * 8, sbytes, wbar);
   }
+
   // ---- everything else that no kernel of the step writes: LN gamma/beta, bias, scales, KV slots ----
   const int ecol = threadIdx.x % C;             // this thread's output column in every epilogue round
   const int en = tile0 * 8 + ecol;              // = output feature n
@@ -289,17 +334,15 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
         // warp means, M2 = sum M2_w + 128 * sum (mean_w - mean)^2
         float msum = 0.f;
         for (int w = 0; w < nw_used; ++w) msum += lnred[w * 4 + r].x;
-        float2 acc0;
-        acc0.x = msum * inv_nw;
-        acc0.y = 0.f;
+        const float mu = msum * inv_nw;
+        float m2t = 0.f;
         for (int w = 0; w < nw_used; ++w) {
           const float2 o2 = lnred[w * 4 + r];
-          const float dl = o2.x - acc0.x;
-          acc0.y += o2.y + 128.f * dl * dl;
+          const float dl = o2.x - mu;
+          m2t += o2.y + 128.f * dl * dl;
         }
-        const float mu = acc0.x;
-        const float rstd = rsqrtf(acc0.y * inv_k + a.ln_eps);
-        if (b < a.B && lc < a.K) {
+        const float rstd = rsqrtf(m2t * inv_k + a.ln_eps);
+        if (lc < a.K) {
           uint2 y;
           y.x = pack_bf16x2((xv[r].x - mu) * rstd * bf16_lo(ln_gg.x) + bf16_lo(ln_bb.x),
                             (xv[r].y - mu) * rstd * bf16_hi(ln_gg.x) + bf16_hi(ln_bb.x));
@@ -312,9 +355,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       }
       __syncthreads();
     }
-  }
-
-  if (MODE == ACT_STAGED) {
+  } else if (MODE == ACT_STAGED) {
     const int k8 = a.K >> 3;
     for (int idx = threadIdx.x; idx < a.B * k8; idx += kLinearThreads) {
       const int b = idx / k8, c8 = idx - b * k8;
@@ -322,21 +363,23 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
           *reinterpret_cast<const uint4 *>(a.act + (size_t)b * a.K + 8 * c8);
     }
     __syncthreads();
+  } else {
+    __syncthreads();  // the barrier's initialisation by thread 0 must be visible before anyone polls it
   }
-
   trace_mark(a.trace, a.trace_slot, 3);
+
+  // ---- the weights must have landed by now (they were requested before the dependency wait) ----
+  if (!mbar_wait_bounded(wbar, 0, 2000000000ull)) {
+    if (a.err) atomicExch(a.err, 1);
+    // give the copies still in flight towards this CTA's shared memory a last chance to finish
+    mbar_wait_bounded(wbar, 0, 2000000000ull);
+    return;
+  }
+  const uint4 *wtile = reinterpret_cast<const uint4 *>(wsm);   // tile (j, kb) at ((j*KB + kb)*32 + lane)
+  trace_mark(a.trace, a.trace_slot, 6);
+
   for (int m0 = 0; m0 < a.B; m0 += 16) {
-    // two accumulator sets per row tile (k-tiles alternate between them) shorten the dependent MMA chain
-    float acc2[2][RT][4];
-#pragma unroll
-    for (int j = 0; j < RT; ++j)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc2[0][j][q] = acc2[1][j][q] = 0.f;
-    const int r0 = m0 + g, r1 = m0 + g + 8;
-    const uint16_t *row0 = STAGED ? stage + (size_t)r0 * stride : a.act + (size_t)r0 * a.K;
-    const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K;
-    const bool v0 = r0 < a.B, v1 = r1 < a.B;
-    // the residual's old value, fetched while the MMAs run
+    // the residual's old value, fetched while the products run
     float e_old[ER];
 #pragma unroll
     for (int e = 0; e < ER; ++e) {
@@ -345,81 +388,168 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       const int b = m0 + o / C;
       if (a.mode == EPI_RESID && o < 16 * C && b < a.B && en < a.N) e_old[e] = a.out_f32[(size_t)b * a.out_stride + en];
     }
-    // activation fragments: G k-tiles are fetched together so that their latencies overlap
-    constexpr int G = STAGED ? 1 : ((4 / AW) < KPW ? (4 / AW) : KPW);
+    if (NB > 0) {
+      // ---- CUDA-core path: lane (g,t) multiplies its 16 bytes of weight row g with the matching
+      //      activation columns of up to NB batch rows; the 4 lanes of a row meet by shuffles ----
+      constexpr int NBA = NB > 0 ? NB : 1;  // array extent (the branch is dead for NB == 0)
+      float facc[RT][NBA];
 #pragma unroll
-    for (int i0 = 0; i0 < KPW; i0 += G) {
-      uint4 xg0[G][AW], xg1[G][AW];
+      for (int j = 0; j < RT; ++j)
 #pragma unroll
-      for (int gi = 0; gi < G; ++gi) {
-        const int kb = warp + (i0 + gi) * kLinearWarps;
+        for (int b = 0; b < NBA; ++b) facc[j][b] = 0.f;
+#pragma unroll 4
+      for (int kb = warp; kb < KB; kb += kLinearWarps) {
         const int col = kb * KT + t * (KT / 4);
+        uint4 wq[RT];
+#pragma unroll
+        for (int j = 0; j < RT; ++j) wq[j] = wtile[((size_t)j * KB + kb) * 32 + lane];
+        float tacc[RT][NBA];  // int4: sums of one 128-column group, scaled afterwards
+        if (WF == WF_INT4) {
+#pragma unroll
+          for (int j = 0; j < RT; ++j)
+#pragma unroll
+            for (int b = 0; b < NBA; ++b) tacc[j][b] = 0.f;
+        }
 #pragma unroll
         for (int q = 0; q < AW; ++q) {
-          xg0[gi][q] = (v0 && kb < KB) ? *reinterpret_cast<const uint4 *>(row0 + col + 8 * q) : make_uint4(0, 0, 0, 0);
-          xg1[gi][q] = (v1 && kb < KB) ? *reinterpret_cast<const uint4 *>(row1 + col + 8 * q) : make_uint4(0, 0, 0, 0);
+          float xf[NBA][8];
+#pragma unroll
+          for (int b = 0; b < NBA; ++b) {
+            uint4 xv = make_uint4(0, 0, 0, 0);
+            if (b < a.B) xv = *reinterpret_cast<const uint4 *>(stage + (size_t)b * stride + col + 8 * q);
+            xf[b][0] = bf16_lo(xv.x); xf[b][1] = bf16_hi(xv.x); xf[b][2] = bf16_lo(xv.y); xf[b][3] = bf16_hi(xv.y);
+            xf[b][4] = bf16_lo(xv.z); xf[b][5] = bf16_hi(xv.z); xf[b][6] = bf16_lo(xv.w); xf[b][7] = bf16_hi(xv.w);
+          }
+#pragma unroll
+          for (int j = 0; j < RT; ++j) {
+            const uint32_t ww[4] = {wq[j].x, wq[j].y, wq[j].z, wq[j].w};
+            float wv[8];
+            if (WF == WF_BF16) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) { wv[2 * k] = bf16_lo(ww[k]); wv[2 * k + 1] = bf16_hi(ww[k]); }
+            } else if (WF == WF_INT8) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) wv[k] = biased_byte_to_float(ww[(2 * q + (k >> 2)) & 3], k & 3);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const uint32_t pr = ((ww[q & 3] >> (4 * e)) & 0x000F000Fu) | 0x43004300u;  // bf16 pair 128+u
+                wv[2 * e] = bf16_lo(pr) - 136.f;
+                wv[2 * e + 1] = bf16_hi(pr) - 136.f;
+              }
+            }
+#pragma unroll
+            for (int b = 0; b < NBA; ++b) {
+              // two independent chains of four products keep the FMA pipe busy
+              float s0 = (WF == WF_INT4) ? tacc[j][b] : facc[j][b];
+              float s1 = wv[4] * xf[b][4];
+              s0 = fmaf(wv[0], xf[b][0], s0); s1 = fmaf(wv[5], xf[b][5], s1);
+              s0 = fmaf(wv[1], xf[b][1], s0); s1 = fmaf(wv[6], xf[b][6], s1);
+              s0 = fmaf(wv[2], xf[b][2], s0); s1 = fmaf(wv[7], xf[b][7], s1);
+              s0 = fmaf(wv[3], xf[b][3], s0);
+              s0 += s1;
+              if (WF == WF_INT4) tacc[j][b] = s0; else facc[j][b] = s0;
+            }
+          }
         }
-      }
+        if (WF == WF_INT4) {
 #pragma unroll
-      for (int gi = 0; gi < G; ++gi) {
-      const int i = i0 + gi;
-      const int kb = warp + i * kLinearWarps;
-      float (*acc)[4] = acc2[i & 1];
-      if (kb < KB) {
-        const uint4 *x0 = xg0[gi], *x1 = xg1[gi];
+          for (int j = 0; j < RT; ++j) {
+            const float sc = bf16_bits_to_float(ssm[((size_t)j * KB + kb) * 8 + g]);  // this lane's row
 #pragma unroll
-        for (int j = 0; j < RT; ++j) {
-          const uint32_t ww[4] = {wr[j][i].x, wr[j][i].y, wr[j][i].z, wr[j][i].w};
-          if (WF == WF_BF16) {
-            mma_bf16_16816(acc[j], x0[0].x, x1[0].x, x0[0].y, x1[0].y, ww[0], ww[1]);
-            mma_bf16_16816(acc[j], x0[0].z, x1[0].z, x0[0].w, x1[0].w, ww[2], ww[3]);
-          } else if (WF == WF_INT8) {
-#pragma unroll
-            for (int s = 0; s < 4; ++s) {
-              const uint32_t b0 = pack_bf16x2(biased_byte_to_float(ww[s], 0), biased_byte_to_float(ww[s], 1));
-              const uint32_t b1 = pack_bf16x2(biased_byte_to_float(ww[s], 2), biased_byte_to_float(ww[s], 3));
-              const uint4 xa = x0[s >> 1], xb = x1[s >> 1];
-              if (s & 1) mma_bf16_16816(acc[j], xa.z, xb.z, xa.w, xb.w, b0, b1);
-              else mma_bf16_16816(acc[j], xa.x, xb.x, xa.y, xb.y, b0, b1);
-            }
-          } else {
-            float tmp[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int wd = 0; wd < 4; ++wd) {
-              const uint4 xa = x0[wd], xb = x1[wd];
-              {
-                const uint32_t b0 = nib_pair_to_bf16x2(ww[wd] & 0x000F000Fu);
-                const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 4) & 0x000F000Fu);
-                mma_bf16_16816(tmp, xa.x, xb.x, xa.y, xb.y, b0, b1);
-              }
-              {
-                const uint32_t b0 = nib_pair_to_bf16x2((ww[wd] >> 8) & 0x000F000Fu);
-                const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 12) & 0x000F000Fu);
-                mma_bf16_16816(tmp, xa.z, xb.z, xa.w, xb.w, b0, b1);
-              }
-            }
-            const float s_lo = bf16_lo(sc2[j][i]), s_hi = bf16_hi(sc2[j][i]);  // weight rows 2t, 2t+1
-            acc[j][0] = fmaf(s_lo, tmp[0], acc[j][0]);
-            acc[j][1] = fmaf(s_hi, tmp[1], acc[j][1]);
-            acc[j][2] = fmaf(s_lo, tmp[2], acc[j][2]);
-            acc[j][3] = fmaf(s_hi, tmp[3], acc[j][3]);
+            for (int b = 0; b < NBA; ++b) facc[j][b] = fmaf(sc, tacc[j][b], facc[j][b]);
           }
         }
       }
+      trace_mark(a.trace, a.trace_slot, 4);
+#pragma unroll
+      for (int j = 0; j < RT; ++j)
+#pragma unroll
+        for (int b = 0; b < NBA; ++b) {
+          float v = facc[j][b];
+          v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+          v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+          if (t == 0) red[((size_t)warp * 16 + b) * C + 8 * j + g] = v;
+        }
+    } else {
+      // ---- tensor-pipe path: the batch is the 16-row M operand, the 8 weight rows the N operand ----
+      float acc[RT][4];
+#pragma unroll
+      for (int j = 0; j < RT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
+      const int r0 = m0 + g, r1 = m0 + g + 8;
+      const uint16_t *row0 = STAGED ? stage + (size_t)r0 * stride : a.act + (size_t)r0 * a.K;
+      const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K;
+      const bool v0 = r0 < a.B, v1 = r1 < a.B;
+      // activation fragments: G k-tiles are fetched together so that their latencies overlap
+      constexpr int G = STAGED ? 1 : 4 / AW;
+      for (int kb0 = warp; kb0 < KB; kb0 += G * kLinearWarps) {
+        uint4 xg0[G][AW], xg1[G][AW];
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const int kb = kb0 + gi * kLinearWarps;
+          const int col = kb * KT + t * (KT / 4);
+#pragma unroll
+          for (int q = 0; q < AW; ++q) {
+            xg0[gi][q] = (v0 && kb < KB) ? *reinterpret_cast<const uint4 *>(row0 + col + 8 * q) : make_uint4(0, 0, 0, 0);
+            xg1[gi][q] = (v1 && kb < KB) ? *reinterpret_cast<const uint4 *>(row1 + col + 8 * q) : make_uint4(0, 0, 0, 0);
+          }
+        }
+#pragma unroll
+        for (int gi = 0; gi < G; ++gi) {
+          const int kb = kb0 + gi * kLinearWarps;
+          if (kb < KB) {
+            const uint4 *x0 = xg0[gi], *x1 = xg1[gi];
+#pragma unroll
+            for (int j = 0; j < RT; ++j) {
+              const uint4 wq = wtile[((size_t)j * KB + kb) * 32 + lane];
+              const uint32_t ww[4] = {wq.x, wq.y, wq.z, wq.w};
+              if (WF == WF_BF16) {
+                mma_bf16_16816(acc[j], x0[0].x, x1[0].x, x0[0].y, x1[0].y, ww[0], ww[1]);
+                mma_bf16_16816(acc[j], x0[0].z, x1[0].z, x0[0].w, x1[0].w, ww[2], ww[3]);
+              } else if (WF == WF_INT8) {
+#pragma unroll
+                for (int s = 0; s < 4; ++s) {
+                  const uint32_t b0 = pack_bf16x2(biased_byte_to_float(ww[s], 0), biased_byte_to_float(ww[s], 1));
+                  const uint32_t b1 = pack_bf16x2(biased_byte_to_float(ww[s], 2), biased_byte_to_float(ww[s], 3));
+                  const uint4 xa = x0[(s >> 1) % AW], xb = x1[(s >> 1) % AW];
+                  if (s & 1) mma_bf16_16816(acc[j], xa.z, xb.z, xa.w, xb.w, b0, b1);
+                  else mma_bf16_16816(acc[j], xa.x, xb.x, xa.y, xb.y, b0, b1);
+                }
+              } else {
+                float tmp[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int wd = 0; wd < 4; ++wd) {
+                  const uint4 xa = x0[wd % AW], xb = x1[wd % AW];
+                  {
+                    const uint32_t b0 = nib_pair_to_bf16x2(ww[wd] & 0x000F000Fu);
+                    const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 4) & 0x000F000Fu);
+                    mma_bf16_16816(tmp, xa.x, xb.x, xa.y, xb.y, b0, b1);
+                  }
+                  {
+                    const uint32_t b0 = nib_pair_to_bf16x2((ww[wd] >> 8) & 0x000F000Fu);
+                    const uint32_t b1 = nib_pair_to_bf16x2((ww[wd] >> 12) & 0x000F000Fu);
+                    mma_bf16_16816(tmp, xa.z, xb.z, xa.w, xb.w, b0, b1);
+                  }
+                }
+                // scales of weight rows 2t, 2t+1 for this 128-column group
+                const uint32_t s2 = *reinterpret_cast<const uint32_t *>(ssm + ((size_t)j * KB + kb) * 8 + 2 * t);
+                const float s_lo = bf16_lo(s2), s_hi = bf16_hi(s2);
+                acc[j][0] = fmaf(s_lo, tmp[0], acc[j][0]);
+                acc[j][1] = fmaf(s_hi, tmp[1], acc[j][1]);
+                acc[j][2] = fmaf(s_lo, tmp[2], acc[j][2]);
+                acc[j][3] = fmaf(s_hi, tmp[3], acc[j][3]);
+              }
+            }
+          }
+        }
       }
-    }
-
-    trace_mark(a.trace, a.trace_slot, 4);
-    // partial sums of the warps meet in shared memory and are added in warp order
-    float acc[RT][4];
+      trace_mark(a.trace, a.trace_slot, 4);
+      // partial sums of the warps meet in shared memory and are added in warp order
 #pragma unroll
-    for (int j = 0; j < RT; ++j)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[j][q] = acc2[0][j][q] + acc2[1][j][q];
-#pragma unroll
-    for (int j = 0; j < RT; ++j) {
-      *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g) * C + 8 * j + 2 * t) = make_float2(acc[j][0], acc[j][1]);
-      *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g + 8) * C + 8 * j + 2 * t) = make_float2(acc[j][2], acc[j][3]);
+      for (int j = 0; j < RT; ++j) {
+        *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g) * C + 8 * j + 2 * t) = make_float2(acc[j][0], acc[j][1]);
+        *reinterpret_cast<float2 *>(red + ((size_t)warp * 16 + g + 8) * C + 8 * j + 2 * t) = make_float2(acc[j][2], acc[j][3]);
+      }
     }
     __syncthreads();
     trace_mark(a.trace, a.trace_slot, 5);
@@ -463,75 +593,78 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
   trace_mark(a.trace, a.trace_slot, 2);
 }
 
+// Shared memory of one CTA.
+inline size_t linear_smem_bytes(int wf, int rt, int mode, int B, int K) {
+  const int KB = K / k_per_tile(wf);
+  size_t s = 128 + (size_t)rt * KB * (wf == WF_INT4 ? 528 : 512) + (size_t)kLinearWarps * 16 * 8 * rt * sizeof(float);
+  if (mode != ACT_DIRECT) s += (size_t)B * ln_stage_stride(wf, K) * sizeof(uint16_t);
+  return s;
+}
+
 // Launch shape: all CTAs of a launch should be resident at once (2 per SM), so that every weight
-// byte of the layer is requested before the kernel waits for its predecessor.
+// byte of the layer is requested before the kernel waits for its predecessor; a CTA's weights and
+// activation rows must fit its share of shared memory.
 struct LinearPlan { int rt, grid; };
-inline LinearPlan plan_linear(int N, int max_ctas) {
+inline LinearPlan plan_linear(int wf, int N, int K, int B, int mode, int max_ctas) {
   const int tiles = row_tiles(N);
   LinearPlan p;
   p.rt = 1;
-  while (p.rt < 4 && (tiles + p.rt - 1) / p.rt > max_ctas) p.rt *= 2;
+  while (p.rt < 4 && (tiles + p.rt - 1) / p.rt > max_ctas &&
+         linear_smem_bytes(wf, p.rt * 2, mode, B, K) <= (size_t)kLinearSmemBudget)
+    p.rt *= 2;
   p.grid = (tiles + p.rt - 1) / p.rt;
   return p;
 }
 
-template <int WF, int KPW, int RT, int MODE>
-inline cudaError_t launch_linear_inst(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
-  size_t smem = (size_t)kLinearWarps * 16 * 8 * RT * sizeof(float);
-  if (MODE != ACT_DIRECT) smem += (size_t)a.B * ln_stage_stride(WF, a.K) * sizeof(uint16_t);
+template <int WF, int RT, int MODE, int NB>
+inline cudaError_t launch_linear_nb(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
+  const size_t smem = linear_smem_bytes(WF, RT, MODE, a.B, a.K);
   static bool attr_done = false;  // opt-in to more than 48 KB of dynamic shared memory, once
   if (!attr_done) {
-    cudaFuncSetAttribute(linear_kernel<WF, KPW, RT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+    cudaFuncSetAttribute(linear_kernel<WF, RT, MODE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     attr_done = true;
   }
-  return launch_kernel(linear_kernel<WF, KPW, RT, MODE>, dim3(grid), dim3(kLinearThreads), smem, st, pdl, a);
+  return launch_kernel(linear_kernel<WF, RT, MODE, NB>, dim3(grid), dim3(kLinearThreads), smem, st, pdl, a);
 }
 
-template <int WF, int KPW, int MODE>
-inline cudaError_t launch_linear_rt(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
-  if (KPW * p.rt > 16) {  // too many weight registers: fall back to more, smaller CTAs
-    p.rt = 16 / KPW;
-    p.grid = (row_tiles(a.N) + p.rt - 1) / p.rt;
+template <int WF, int RT, int MODE>
+inline cudaError_t launch_linear_inst(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
+  if (MODE != ACT_DIRECT) {  // batches of up to 4 rows always fit the staging buffer
+    if (a.B == 1) return launch_linear_nb<WF, RT, (MODE == ACT_DIRECT ? ACT_STAGED : MODE), 1>(a, grid, st, pdl);
+    if (a.B <= 4) return launch_linear_nb<WF, RT, (MODE == ACT_DIRECT ? ACT_STAGED : MODE), 4>(a, grid, st, pdl);
   }
-  if (p.rt == 1) return launch_linear_inst<WF, KPW, 1, MODE>(a, p.grid, st, pdl);
-  if (p.rt == 2) return launch_linear_inst<WF, KPW, (KPW <= 8 ? 2 : 1), MODE>(a, p.grid, st, pdl);
-  return launch_linear_inst<WF, KPW, (KPW <= 4 ? 4 : 1), MODE>(a, p.grid, st, pdl);
+  return launch_linear_nb<WF, RT, MODE, 0>(a, grid, st, pdl);
 }
 
 template <int WF, int MODE>
-inline cudaError_t launch_linear_wf(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
-  const int KB = a.K / k_per_tile(WF);
-  const int kpw = (KB + kLinearWarps - 1) / kLinearWarps;
-  if (kpw <= 1) return launch_linear_rt<WF, 1, MODE>(a, p, st, pdl);
-  if (kpw <= 2) return launch_linear_rt<WF, 2, MODE>(a, p, st, pdl);
-  if (kpw <= 4) return launch_linear_rt<WF, 4, MODE>(a, p, st, pdl);
-  if (MODE == ACT_LN) return cudaErrorInvalidValue;  // fused LayerNorm is built for K <= 1280 only
-  if (kpw <= 8) return launch_linear_rt<WF, 8, (MODE == ACT_LN ? ACT_STAGED : MODE)>(a, p, st, pdl);
-  if (kpw <= 16) return launch_linear_rt<WF, 16, (MODE == ACT_LN ? ACT_STAGED : MODE)>(a, p, st, pdl);
-  return cudaErrorInvalidValue;
+inline cudaError_t launch_linear_wf(const LinearArgs &a, int max_ctas, cudaStream_t st, bool pdl) {
+  const LinearPlan p = plan_linear(WF, a.N, a.K, a.B, MODE, max_ctas);
+  if (linear_smem_bytes(WF, p.rt, MODE, a.B, a.K) > 200 * 1024) return cudaErrorInvalidValue;
+  if (p.rt == 1) return launch_linear_inst<WF, 1, MODE>(a, p.grid, st, pdl);
+  if (p.rt == 2) return launch_linear_inst<WF, 2, MODE>(a, p.grid, st, pdl);
+  return launch_linear_inst<WF, 4, MODE>(a, p.grid, st, pdl);
 }
 
-// Whether LayerNorm can be fused in front of a linear with this shape.
+// Whether LayerNorm can be fused in front of a linear with this shape (one float4 of the row per thread).
 inline bool can_fuse_ln(int wf, int B, int K) {
-  const int kpw = (K / k_per_tile(wf) + kLinearWarps - 1) / kLinearWarps;
-  return B <= kLnFuseMaxRows && kpw <= 4 && K <= 4 * kLinearThreads;  // one float4 of the row per thread
+  (void)wf;
+  return B <= kLnFuseMaxRows && K <= 4 * kLinearThreads;
 }
 
 template <int WF>
-inline cudaError_t launch_linear_mode(const LinearArgs &a, LinearPlan p, cudaStream_t st, bool pdl) {
-  if (a.ln_x) return launch_linear_wf<WF, ACT_LN>(a, p, st, pdl);
+inline cudaError_t launch_linear_mode(const LinearArgs &a, int max_ctas, cudaStream_t st, bool pdl) {
+  if (a.ln_x) return launch_linear_wf<WF, ACT_LN>(a, max_ctas, st, pdl);
   if ((size_t)a.B * ln_stage_stride(WF, a.K) * sizeof(uint16_t) <= (size_t)kStageMaxBytes)
-    return launch_linear_wf<WF, ACT_STAGED>(a, p, st, pdl);
-  return launch_linear_wf<WF, ACT_DIRECT>(a, p, st, pdl);
+    return launch_linear_wf<WF, ACT_STAGED>(a, max_ctas, st, pdl);
+  return launch_linear_wf<WF, ACT_DIRECT>(a, max_ctas, st, pdl);
 }
 
-// K must be a multiple of 128 and at most 160 k-tiles (K <= 5120 for bf16).
+// K must be a multiple of 128.
 inline cudaError_t launch_linear(int wf, const LinearArgs &a, cudaStream_t st, bool pdl = false, int max_ctas = 296) {
-  const LinearPlan p = plan_linear(a.N, max_ctas);
   if (a.ln_x && !can_fuse_ln(wf, a.B, a.K)) return cudaErrorInvalidValue;
-  if (wf == WF_BF16) return launch_linear_mode<WF_BF16>(a, p, st, pdl);
-  if (wf == WF_INT8) return launch_linear_mode<WF_INT8>(a, p, st, pdl);
-  return launch_linear_mode<WF_INT4>(a, p, st, pdl);
+  if (wf == WF_BF16) return launch_linear_mode<WF_BF16>(a, max_ctas, st, pdl);
+  if (wf == WF_INT8) return launch_linear_mode<WF_INT8>(a, max_ctas, st, pdl);
+  return launch_linear_mode<WF_INT4>(a, max_ctas, st, pdl);
 }
 
 inline cudaError_t launch_pack(int wf, int N, int K, const void *w, const void *s, void *dst_w, void *dst_s,

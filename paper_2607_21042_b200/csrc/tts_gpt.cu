@@ -71,6 +71,8 @@ struct tts_gpt {
   bool use_pdl;
   int n_sm = 148;
   unsigned long long launches = 0;
+  int *dev_err = nullptr;               // error word set by a kernel whose bounded wait expired:
+  volatile int *host_err = nullptr;     //   4 bytes of pinned, device-mapped host memory (read after a sync without a copy)
   unsigned long long *trace = nullptr;  // optional device buffer for kernel timelines
   int trace_next = 0;  // kernels enqueued so far (graph nodes counted per replay)
 };
@@ -203,6 +205,13 @@ LinearArgs linear_args(const PackedLinear &pl, const uint16_t *act, int B, int m
   a.N = pl.N; a.K = pl.K; a.B = B; a.mode = mode;
   return a;
 }
+LinearArgs linear_args(tts_gpt *h, const PackedLinear &pl, const uint16_t *act, int B, int mode);
+
+LinearArgs linear_args(tts_gpt *h, const PackedLinear &pl, const uint16_t *act, int B, int mode) {
+  LinearArgs a = linear_args(pl, act, B, mode);
+  a.err = h->dev_err;
+  return a;
+}
 
 // gives the next traced kernel of a step its slot
 template <typename Args>
@@ -224,7 +233,7 @@ int run_layers(tts_gpt *h, int R, bool decode) {
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
-    LinearArgs qa = linear_args(L.qkv, h->a, R, EPI_QKV);
+    LinearArgs qa = linear_args(h, L.qkv, h->a, R, EPI_QKV);
     if (fuse_ln) {
       qa.ln_x = h->x; qa.ln_g = L.ln1_g; qa.ln_b = L.ln1_b; qa.ln_eps = c.ln_eps;
     } else {
@@ -243,11 +252,11 @@ int run_layers(tts_gpt *h, int R, bool decode) {
     aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
     trace_attach(h, aa);
     CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
-    LinearArgs oa = linear_args(L.o, h->o, R, EPI_RESID);
+    LinearArgs oa = linear_args(h, L.o, h->o, R, EPI_RESID);
     oa.out_f32 = h->x; oa.out_stride = d;
     trace_attach(h, oa);
     CUDA_TRY(h, launch_linear(c.wfmt, oa, st, pdl, 2 * h->n_sm));
-    LinearArgs f1 = linear_args(L.fc1, h->a, R, EPI_GELU);
+    LinearArgs f1 = linear_args(h, L.fc1, h->a, R, EPI_GELU);
     if (fuse_ln) {
       f1.ln_x = h->x; f1.ln_g = L.ln2_g; f1.ln_b = L.ln2_b; f1.ln_eps = c.ln_eps;
     } else {
@@ -259,7 +268,7 @@ int run_layers(tts_gpt *h, int R, bool decode) {
     f1.out_bf16 = h->hbuf; f1.gelu_tanh = c.gelu_tanh;
     trace_attach(h, f1);
     CUDA_TRY(h, launch_linear(c.wfmt, f1, st, pdl, 2 * h->n_sm));
-    LinearArgs f2 = linear_args(L.fc2, h->hbuf, R, EPI_RESID);
+    LinearArgs f2 = linear_args(h, L.fc2, h->hbuf, R, EPI_RESID);
     f2.out_f32 = h->x; f2.out_stride = d;
     trace_attach(h, f2);
     CUDA_TRY(h, launch_linear(c.wfmt, f2, st, pdl, 2 * h->n_sm));
@@ -273,7 +282,7 @@ int run_head(tts_gpt *h, int n_out) {
   const tts_gpt_config_t &c = h->cfg;
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
-  LinearArgs ha = linear_args(h->head, h->hf, n_out, EPI_F32);
+  LinearArgs ha = linear_args(h, h->head, h->hf, n_out, EPI_F32);
   if (can_fuse_ln(WF_BF16, n_out, c.d_model)) {
     ha.ln_x = h->x; ha.ln_g = h->lnf_g; ha.ln_b = h->lnf_b; ha.ln_eps = c.ln_eps;
     ha.ln_gather = h->rt.out_rows; ha.ln_out_slot = h->rt.out_slot; ha.ln_io = h->io;
@@ -381,9 +390,23 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   const int init_n = std::max(std::max(c.n_pages, c.max_streams * h->pps), c.max_streams);
   init_pages_kernel<<<(init_n + 255) / 256, 256, 0, h->stream>>>(h->ps);
   cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)kMaxRows * c.n_head * sizeof(unsigned int), h->stream);
+  if (e == cudaSuccess) {
+    void *hp = nullptr, *dp = nullptr;
+    e = cudaHostAlloc(&hp, sizeof(int), cudaHostAllocMapped);
+    if (e == cudaSuccess) {
+      *(int *)hp = 0;
+      e = cudaHostGetDevicePointer(&dp, hp, 0);
+      h->host_err = (volatile int *)hp;
+      h->dev_err = (int *)dp;
+    }
+  }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
-  if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(e)); }
+  if (e != cudaSuccess) {
+    if (h->host_err) cudaFreeHost((void *)h->host_err);
+    delete h;
+    return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(e));
+  }
   h->open.assign(c.max_streams, 0);
   h->ctx.assign(c.max_streams, 0);
   h->pos_next.assign(c.max_streams, 0);
@@ -555,6 +578,10 @@ int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
 int32_t tts_gpt_sync(tts_gpt_t *h) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  if (h->host_err && *h->host_err) {
+    *h->host_err = 0;
+    return fail(h, TTS_GPT_E_TIMEOUT, "a kernel's bounded wait for its weight copy expired; results of the last steps are invalid");
+  }
   return TTS_GPT_OK;
 }
 
@@ -562,6 +589,7 @@ int32_t tts_gpt_destroy(tts_gpt_t *h) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   cudaStreamSynchronize(h->stream);
   for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second);
+  if (h->host_err) cudaFreeHost((void *)h->host_err);
   delete h;
   return TTS_GPT_OK;
 }
