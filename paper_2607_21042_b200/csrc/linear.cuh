@@ -31,7 +31,8 @@ enum { EPI_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_GELU = 3 };
 
 constexpr int kLinearWarps = 10;  // divides the k-tile counts of K=1280 and K=5120 in every format
 constexpr int kLinearThreads = kLinearWarps * 32;
-constexpr int kLnFuseMaxRows = 16;  // LayerNorm is fused into the linear up to this batch
+constexpr int kLnFuseMaxRows = 4;   // LayerNorm is fused into the linear up to this batch: every CTA repeats
+                                    // it, which beats a separate launch only while the rows are few
 
 __host__ __device__ inline int k_per_tile(int wf) { return wf == WF_BF16 ? 32 : (wf == WF_INT8 ? 64 : 128); }
 __host__ __device__ inline int row_tiles(int N) { return (N + 7) / 8; }
@@ -281,20 +282,21 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
   trace_mark(a.trace, a.trace_slot, 1);
 
   // ---- optional fused LayerNorm: the CTA splits each row over all threads (4 columns each) and
-  //      handles up to 4 rows per round.  Each thread forms the mean and the centered sum of
+  //      handles up to RPR rows per round.  Each thread forms the mean and the centered sum of
   //      squares of its 4 values; (mean, M2) pairs of equal weight are then merged pairwise
   //      (mean = (ma+mb)/2, M2 = M2a + M2b + (mb-ma)^2 * n/2), first by shuffles, then across the
   //      warps through shared memory: one block barrier, no cancellation.
   const int stride = ln_stage_stride(WF, a.K);
+  constexpr int RPR = 4;  // rows per LayerNorm round
   if (LN) {
-    float2 *lnred = reinterpret_cast<float2 *>(red);  // [warps][4] (mean, M2), reused later for the partial sums
+    float2 *lnred = reinterpret_cast<float2 *>(red);  // [warps][RPR] (mean, M2), reused later for the partial sums
     const int nw_used = (a.K / 4 + 31) / 32;           // warps that hold columns (K is a multiple of 128)
     const float inv_nw = 1.0f / nw_used, inv_k = 1.0f / a.K;
-    for (int b0 = 0; b0 < a.B; b0 += 4) {
-      float4 xv[4];
-      float mean[4], m2[4];
+    for (int b0 = 0; b0 < a.B; b0 += RPR) {
+      float4 xv[RPR];
+      float mean[RPR], m2[RPR];
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
+      for (int r = 0; r < RPR; ++r) {
         xv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
         const int b = b0 + r;
         if (b < a.B && lc < a.K) {
@@ -303,7 +305,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
         }
       }
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
+      for (int r = 0; r < RPR; ++r) {
         mean[r] = 0.f; m2[r] = 0.f;
         if (b0 + r >= a.B) break;
         mean[r] = 0.25f * ((xv[r].x + xv[r].y) + (xv[r].z + xv[r].w));
@@ -320,24 +322,25 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
           cnt *= 2.f;
         }
       }
-      if (lane < 4) {
-        const float mm = lane == 0 ? mean[0] : (lane == 1 ? mean[1] : (lane == 2 ? mean[2] : mean[3]));
-        const float qq = lane == 0 ? m2[0] : (lane == 1 ? m2[1] : (lane == 2 ? m2[2] : m2[3]));
-        lnred[warp * 4 + lane] = make_float2(mm, qq);
+      {  // lane r publishes row r (every lane holds every row's warp-level result)
+        float mm = mean[0], qq = m2[0];
+#pragma unroll
+        for (int r = 1; r < RPR; ++r) { mm = lane == r ? mean[r] : mm; qq = lane == r ? m2[r] : qq; }
+        if (lane < RPR) lnred[warp * RPR + lane] = make_float2(mm, qq);
       }
       __syncthreads();
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
+      for (int r = 0; r < RPR; ++r) {
         const int b = b0 + r;
         if (b >= a.B) break;
         // merge of the warps' (mean, M2), each over 128 values: the grand mean is the mean of the
         // warp means, M2 = sum M2_w + 128 * sum (mean_w - mean)^2
         float msum = 0.f;
-        for (int w = 0; w < nw_used; ++w) msum += lnred[w * 4 + r].x;
+        for (int w = 0; w < nw_used; ++w) msum += lnred[w * RPR + r].x;
         const float mu = msum * inv_nw;
         float m2t = 0.f;
         for (int w = 0; w < nw_used; ++w) {
-          const float2 o2 = lnred[w * 4 + r];
+          const float2 o2 = lnred[w * RPR + r];
           const float dl = o2.x - mu;
           m2t += o2.y + 128.f * dl * dl;
         }
@@ -481,7 +484,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K;
       const bool v0 = r0 < a.B, v1 = r1 < a.B;
       // activation fragments: G k-tiles are fetched together so that their latencies overlap
-      constexpr int G = STAGED ? 1 : 4 / AW;
+      constexpr int G = STAGED ? 1 : 8 / AW;   // up to 64 registers of activation fragments in flight
       for (int kb0 = warp; kb0 < KB; kb0 += G * kLinearWarps) {
         uint4 xg0[G][AW], xg1[G][AW];
 #pragma unroll
