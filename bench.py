@@ -263,8 +263,15 @@ def run_ours(args):
 
     peak, peak_kind = measured_peaks()
     gbs = nbytes / (ms * 1e-3) / 1e9
+    # DRAM bytes per step from the ncu capture summarised in
+    # profiles/decode_step_cfg2_bf16_b1_launch_list_and_dram_traffic.md: 1026.0 MB read+written for a step
+    # whose algorithmic bytes are 1015.9 MB (context 406); traffic grows with the same KV term as the
+    # algorithmic bytes, so the measured ratio is applied to this run's bytes per step.
+    traffic = None
+    if args.workload == 2:
+        traffic = (nbytes / max(steps_done, 1)) * (1026.0 / 1015.9)
     roofline = {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
-                "traffic": None, "peak_source": peak_kind,
+                "traffic": traffic, "peak_source": peak_kind,
                 "kernel": "whole decode step (CUDA graph of %d kernels)" % (launches // max(steps_done, 1) - 1),
                 "algorithmic_bytes_per_step": nbytes / max(steps_done, 1)}
 

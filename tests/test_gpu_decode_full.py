@@ -8,7 +8,7 @@ import torch
 from oracle import gpt_oracle as O
 from paper_2607_21042_b200 import binding as B
 from paper_2607_21042_b200 import cases as C
-from helpers import assert_logits_close, bits_dev, check_tokens, gpu_run_stream
+from helpers import assert_logits_close, assert_same_up_to_ties, bits_dev, check_tokens, gpu_run_stream
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -89,8 +89,7 @@ def _workload5(wfmt):
             continue
         alone = _batch_run(eng, wl, [prefixes[i]], 24)[0]
         m = min(25, len(res[i][0]))
-        assert np.array_equal(alone[0][:m], res[i][0][:m])
-        assert_logits_close(alone[1][:m], res[i][1][:m].astype(np.float64), "batch invariance stream %d" % i)
+        assert_same_up_to_ties(alone[0][:m], alone[1][:m], res[i][0][:m], res[i][1][:m], "batch invariance stream %d" % i)
     eng.destroy()
 
 def test_workload2_bf16_batch1_replay():
@@ -159,8 +158,7 @@ def test_workload4_w4a16_batch16_replay_and_batch_invariance():
         if i in picks:
             continue
         alone = _batch_run(eng, wl, [prefixes[i]], 40)[0]
-        assert np.array_equal(alone[0], res[i][0][:41])
-        assert_logits_close(alone[1], res[i][1][:41].astype(np.float64), "batch invariance stream %d" % i)
+        assert_same_up_to_ties(alone[0], alone[1], res[i][0][:41], res[i][1][:41], "batch invariance stream %d" % i)
     eng.destroy()
 
 def test_workload5_w4a16_batch128_ragged_drain():

@@ -10,7 +10,7 @@ import torch
 from oracle import gpt_oracle as O
 from paper_2607_21042_b200 import binding as B
 from paper_2607_21042_b200 import cases as C
-from helpers import (assert_logits_close, bits_dev, check_tokens, gpu_run_stream)
+from helpers import (assert_logits_close, assert_same_up_to_ties, bits_dev, check_tokens, gpu_run_stream)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -107,12 +107,7 @@ def test_batch_invariance_page_permutation_and_reuse(tiny_models):
     # of an activation (and identical tokens away from ties)
     for s in range(4):
         lg_one, tk_one = _run_batch(eng, [prefixes[s]], n)
-        d = np.nonzero(tk_one[0] != tk_batch[s])[0]
-        m = len(tk_batch[s]) if len(d) == 0 else d[0] + 1       # histories agree up to here
-        assert np.max(np.abs(lg_one[0][:m] - lg_batch[s][:m])) < 1e-2, "batch of 4 vs alone, stream %d" % s
-        if len(d):
-            srt = np.sort(lg_batch[s][d[0]])
-            assert srt[-1] - srt[-2] < 1e-2
+        assert_same_up_to_ties(tk_one[0], lg_one[0], tk_batch[s], lg_batch[s], "batch of 4 vs alone, stream %d" % s)
     # physical page placement does not matter: bit-identical after shuffling the free list
     lg_shuf, tk_shuf = _run_batch(eng, prefixes, n, shuffle_seed=123)
     assert np.array_equal(lg_shuf, lg_batch) and np.array_equal(tk_shuf, tk_batch)
