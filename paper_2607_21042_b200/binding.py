@@ -26,7 +26,7 @@ EXPORTS = [
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
     "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
-    "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static", "tts_gpt_op_attention_cluster",
+    "tts_gpt_op_linear_tc_scratch_bytes", "tts_gpt_op_linear_tc", "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static", "tts_gpt_op_attention_cluster",
     "tts_gpt_op_layernorm",
     "tts_gpt_op_sample",
 ]
@@ -274,6 +274,22 @@ def op_linear(wfmt, packed, N, K, act, bias=None, stream=None):
     out = torch.empty((B, N), dtype=torch.float32, device=act.device)
     _check(load().tts_gpt_op_linear(C.c_int32(wfmt), C.c_int32(N), C.c_int32(K), _ptr(packed), _ptr(bias),
                                     C.c_int32(B), _ptr(act), _ptr(out), _stream_ptr(stream)))
+    return out
+
+
+def op_linear_tc(w, act, bias=None, ksplit=1, stream=None):
+    """Tensor-core linear: w int16 (bf16 bits) [N,K] canonical, act int16 [B,K] -> fp32 [B,N]."""
+    N, K = w.shape
+    B = act.shape[0]
+    n = C.c_size_t(0)
+    _check(load().tts_gpt_op_linear_tc_scratch_bytes(C.c_int32(N), C.c_int32(K), C.byref(n)))
+    scratch = torch.zeros(n.value + 1024, dtype=torch.uint8, device=w.device)
+    base = (scratch.data_ptr() + 1023) // 1024 * 1024
+    out = torch.empty((B, N), dtype=torch.float32, device=w.device)
+    _check(load().tts_gpt_op_linear_tc(C.c_int32(N), C.c_int32(K), _ptr(w), _ptr(bias), C.c_int32(B), _ptr(act),
+                                       _ptr(out), C.c_int32(ksplit), C.c_void_p(base), _stream_ptr(stream)))
+    torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+    del scratch
     return out
 
 

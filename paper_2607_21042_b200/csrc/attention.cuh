@@ -21,6 +21,7 @@
 #pragma once
 #include <cooperative_groups.h>
 #include "common.cuh"
+#include "elementwise.cuh"
 
 namespace ttsgpt {
 
@@ -47,6 +48,7 @@ struct AttnArgs {
   int H, pps;
   unsigned long long *trace;  // optional timeline trace
   int trace_slot;
+  int out_image;             // 1: `out` is an activation image for the tensor-core linear (see act_image_offset)
   int old_pages_final;       // 1: one row per stream (decode step), pages before a row's last are not written by this step
 };
 
@@ -224,9 +226,13 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
   trace_mark(a.trace, a.trace_slot, 4);
   const int e = threadIdx.x;
-  uint16_t *out = a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim;
+  // plain row-major bf16, or the image layout of the tensor-core linear that consumes it
+  uint16_t *out = nullptr;
+  if (e < kHeadDim)
+    out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
+                      : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
   if (S == 1) {
-    if (e < kHeadDim) out[e] = float_to_bf16_bits(O / L);
+    if (e < kHeadDim) *out = float_to_bf16_bits(O / L);
     trace_mark(a.trace, a.trace_slot, 2);
     return;
   }
@@ -258,7 +264,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
       LL = fmaf(pl_[rr], f, LL);
       OO = fmaf(po[rr], f, OO);
     }
-    out[e] = float_to_bf16_bits(OO / LL);
+    *out = float_to_bf16_bits(OO / LL);
   }
   cluster.sync();  // keep every rank's shared memory alive until rank 0 has read it
   trace_mark(a.trace, a.trace_slot, 2);

@@ -101,6 +101,72 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_kernel(const float *__re
   }
 }
 
+// byte offset of element (row, k) inside an activation image: blocks of 128 rows x 64 columns
+// (16 KB each, one per k-chunk), row r at byte r*128, its 16-byte unit u stored at unit u ^ (r % 8)
+__host__ __device__ inline size_t act_image_offset(int row, int k) {
+  const int kc = k >> 6, u = (k & 63) >> 3;
+  return (size_t)kc * (kMaxRows * 128) + (size_t)row * 128 + (size_t)((u ^ (row & 7)) << 4) + (size_t)(k & 7) * 2;
+}
+
+// LayerNorm in front of a tensor-core linear.  First folds what the previous k-split linear left
+// behind into the residual stream, in a fixed order: x[r] += bias + partial[0][r] + partial[1][r] + ...
+// (written back unless `write_back` is 0), then normalises and writes the row into the activation
+// image (`out_img`) and/or a plain bf16 row (`out_plain`, row j).  With `gather`, row j is x row gather[j].
+struct LnTcArgs {
+  float *x; int d;
+  const float *partials; int n_part, part_cols;   // [n_part][kMaxRows][part_cols]
+  const uint16_t *add_bias;
+  const uint16_t *g, *b; float eps;
+  void *out_img; uint16_t *out_plain;
+  const int *gather, *out_slot; const StepIO *io;
+  int write_back;
+};
+__global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs a) {
+  __shared__ float sm[kLnThreads / 32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int j = blockIdx.x;
+  const int r = a.gather ? a.gather[j] : j;
+  float *xr = a.x + (size_t)r * a.d;
+  float v[kLnMaxPerThread];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    v[i] = 0.f;
+    if (c < a.d) {
+      float t = xr[c];
+      if (a.n_part > 0) {
+        if (a.add_bias) t += bf16_bits_to_float(a.add_bias[c]);
+        for (int p = 0; p < a.n_part; ++p) t += a.partials[((size_t)p * kMaxRows + r) * a.part_cols + c];
+        if (a.write_back) xr[c] = t;
+      }
+      v[i] = t;
+    }
+    s += v[i];
+  }
+  const float mu = block_sum(s, sm) / a.d;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    const float t = c < a.d ? v[i] - mu : 0.f;
+    q += t * t;
+  }
+  const float rstd = rsqrtf(block_sum(q, sm) / a.d + a.eps);
+  uint16_t *hid = (a.io && a.io->out_hidden) ? a.io->out_hidden + (size_t)(a.out_slot ? a.out_slot[j] : j) * a.d : nullptr;
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    if (c < a.d) {
+      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * bf16_bits_to_float(a.g[c]) + bf16_bits_to_float(a.b[c]));
+      if (a.out_img) *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset(j, c)) = y;
+      if (a.out_plain) a.out_plain[(size_t)j * a.d + c] = y;
+      if (hid) hid[c] = y;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // sampling
 // ------------------------------------------------------------------------------------------

@@ -1,0 +1,303 @@
+// Batched linear on the 5th-generation tensor cores (tcgen05) for more than 16 rows: at these
+// batch sizes the layer is a dense contraction out[b,n] = sum_k W[n,k] act[b,k], bf16 operands,
+// fp32 accumulation in tensor memory (Table I / III regime: many concurrent utterances).
+//
+// Operand images.  Both operands are kept in global memory in exactly the byte order the tensor
+// core wants them in shared memory (K-major, 128-byte swizzle): a k-chunk of 64 columns of 128
+// rows is one 16 KB block in which row r sits at byte r*128 and the 16-byte unit u of that row is
+// stored at unit (u ^ (r % 8)).  Weights [N,K] become blocks [n/128][k/64]; activations of up to
+// 128 rows become blocks [k/64] (rows are batch rows, so the 32 rows of a batch chunk are 4 KB
+// contiguous inside a block).  A stage of the pipeline is therefore filled by two plain bulk
+// asynchronous copies (16 KB of weights, 4 KB of activations): no tensor maps, no alignment rules
+// beyond 16 bytes.  The kernels that produce activations (LayerNorm, attention, the GELU epilogue
+// below) write this image directly.
+//
+// A CTA owns a 128-row weight tile (the M operand), one chunk of 32 batch rows (the N operand) and
+// a contiguous range of k-chunks; with 4 batch chunks and, for the two linears that feed the
+// residual stream, 4 k-ranges, every linear of the block runs on 120-160 CTAs.  Warp 0 produces
+// (bulk copies into a 5-stage ring guarded by full/empty mbarriers; the weight copies of the first
+// stages are issued before the dependency wait), warp 1 issues the MMAs (4 per k-chunk, M=128,
+// N=32, K=16) and commits each stage back to the producer, then all 4 warps read the 128x32 fp32
+// accumulator out of tensor memory and run the epilogue.  K-split partial sums go to a scratch
+// array that the following LayerNorm kernel folds into the residual stream in a fixed order.
+// Every wait is bounded; on expiry the CTA sets the error word, stops waiting and still releases
+// its tensor memory.
+#pragma once
+#include "common.cuh"
+#include "linear.cuh"
+
+namespace ttsgpt {
+
+constexpr int kTcStages = 5;            // 5 x 20 KB: two CTAs fit one SM
+constexpr int kTcTileM = 128;          // weight rows per CTA
+constexpr int kTcChunkN = 32;          // batch rows per CTA
+constexpr int kTcKChunk = 64;          // columns per pipeline stage (128 bytes of bf16)
+constexpr uint32_t kTcABytes = kTcTileM * 128;   // 16 KB
+constexpr uint32_t kTcBBytes = kTcChunkN * 128;  // 4 KB
+constexpr int kTcThreads = 128;
+constexpr int kTcKSplit = 4;            // k-ranges of the two linears that feed the residual stream
+constexpr unsigned long long kTcWaitNs = 2000000000ull;
+
+// byte offset of element (row, k) inside an operand image whose blocks hold `rows_per_block` rows
+__host__ __device__ inline size_t image_offset(int row, int k, int rows_per_block) {
+  const int kc = k >> 6, u = (k & 63) >> 3;
+  return (size_t)kc * rows_per_block * 128 + (size_t)row * 128 + (size_t)((u ^ (row & 7)) << 4) + (size_t)(k & 7) * 2;
+}
+inline size_t weight_image_bytes(int N, int K) { return (size_t)((N + 127) / 128) * (K / 64) * kTcABytes; }
+inline size_t act_image_bytes(int K) { return (size_t)(K / 64) * kMaxRows * 128; }
+
+// canonical bf16 [N,K] -> weight image, one thread per 16-byte unit of the destination
+__global__ void pack_weight_image_kernel(const uint16_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
+  const int KC = K / 64;
+  const size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t total = (size_t)((N + 127) / 128) * KC * (kTcABytes / 16);
+  if (unit >= total) return;
+  const int within = unit % (kTcABytes / 16);
+  const size_t blk = unit / (kTcABytes / 16);
+  const int kc = blk % KC, nt = blk / KC;
+  const int r = within >> 3, pu = within & 7;   // row in tile, physical 16-byte unit
+  const int u = pu ^ (r & 7);                   // logical unit stored there
+  const int n = nt * 128 + r, k = kc * 64 + u * 8;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (n < N) v = *reinterpret_cast<const uint4 *>(w + (size_t)n * K + k);
+  dst[unit] = v;
+}
+
+// plain bf16 [B,K] -> activation image (used by the stand-alone entry point)
+__global__ void pack_act_image_kernel(const uint16_t *__restrict__ act, int B, int K, unsigned char *__restrict__ dst) {
+  const int k8 = K >> 3;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (size_t)B * k8) return;
+  const int b = idx / k8, k = (int)(idx % k8) * 8;
+  *reinterpret_cast<uint4 *>(dst + image_offset(b, k, kMaxRows)) = *reinterpret_cast<const uint4 *>(act + (size_t)b * K + k);
+}
+
+// ---- tcgen05 / tensor-memory primitives ----
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// arrives on the mbarrier once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// K-major, 128-byte swizzle: 8-row groups 1024 bytes apart, version 1, layout type 2
+__device__ __forceinline__ uint64_t tc_smem_desc(const void *p) {
+  const uint32_t a = smem_u32(p);
+  uint64_t d = 0;
+  d |= (uint64_t)((a >> 4) & 0x3FFF);
+  d |= (uint64_t)1 << 16;                 // leading-dimension byte offset (unused with swizzle), in 16-byte units
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride-dimension byte offset: next 8-row group
+  d |= (uint64_t)1 << 46;                 // descriptor version
+  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+  return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major
+__device__ __forceinline__ uint32_t tc_instr_desc(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// 32 lanes x 32 columns of 32-bit: register c of lane l = TMEM[lane base + l][column base + c]
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+struct GemmTcArgs {
+  const void *w_img;        // weight image [N/128][K/64] blocks
+  const void *act_img;      // activation image [K/64] blocks of 128 rows
+  const uint16_t *bias;     // bf16 [N] or null
+  int N, K, B, mode;        // mode: EPI_* of linear.cuh
+  int ksplit;               // k-ranges (gridDim.z)
+  float *out_f32;           // EPI_F32: out[b*out_stride+n]; EPI_QKV: q; EPI_RESID: x (ksplit == 1) or partials [ksplit][128][N]
+  int out_stride;
+  void *out_img;            // EPI_GELU: activation image of the next linear (row length N)
+  int gelu_tanh;
+  uint16_t *kv_layer;
+  const int *page_table, *row_stream, *row_pos;
+  int pps, d, H;
+  int *err;
+};
+
+// a wait that gives up for good once any wait of the CTA has expired
+__device__ __forceinline__ void tc_wait(uint64_t *bar, uint32_t parity, volatile int *failed, int *err) {
+  if (*failed) return;
+  if (!mbar_wait_bounded(bar, parity, kTcWaitNs)) {
+    *failed = 1;
+    if (err) atomicExch(err, 1);
+  }
+}
+
+__global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a) {
+  extern __shared__ __align__(16) unsigned char tc_smem_raw[];
+  // [stages x (A 16 KB | B 4 KB)] on a 1024-byte boundary (the swizzle pattern repeats every 1024
+  // bytes of shared-memory address), then barriers and small state
+  unsigned char *ring = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+  uint64_t *full = reinterpret_cast<uint64_t *>(ring + kTcStages * (kTcABytes + kTcBBytes));
+  uint64_t *empty = full + kTcStages;
+  uint64_t *acc_done = empty + kTcStages;
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_done + 1);
+  volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  uint16_t **kv_base = reinterpret_cast<uint16_t **>(tmem_slot + 4);   // [32] EPI_QKV: page slot of each batch row
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nt = blockIdx.x, bc = blockIdx.y, ks = blockIdx.z;
+  const int KC = a.K / kTcKChunk;
+  const int per = (KC + a.ksplit - 1) / a.ksplit;
+  const int kc0 = ks * per, kc1 = min(KC, kc0 + per);
+  const int n_it = kc1 - kc0;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    mbar_init(acc_done, 1);
+    *failed = 0;
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, 32);
+  if (a.mode == EPI_QKV && threadIdx.x >= 32 && threadIdx.x < 64) {   // page slots of this chunk's batch rows
+    const int b = bc * kTcChunkN + lane;
+    uint16_t *p = nullptr;
+    if (b < a.B) {
+      const int pos = a.row_pos[b];
+      const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
+      p = a.kv_layer + ((size_t)page * 2 * a.H) * kPageElems + (size_t)(pos & 63) * kHeadDim;
+    }
+    kv_base[lane] = p;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+
+  const unsigned char *gA = reinterpret_cast<const unsigned char *>(a.w_img) + ((size_t)nt * KC + kc0) * kTcABytes;
+  const unsigned char *gB = reinterpret_cast<const unsigned char *>(a.act_img) + (size_t)kc0 * (kMaxRows * 128) + (size_t)bc * kTcBBytes;
+
+  const int pre = min(n_it, kTcStages);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < pre; ++i) {   // weights do not depend on the previous kernel
+      mbar_expect_tx(full + i, kTcABytes + kTcBBytes);
+      bulk_copy_g2s(ring + (size_t)i * (kTcABytes + kTcBBytes), gA + (size_t)i * kTcABytes, kTcABytes, full + i);
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (warp == 0) {
+    // ---- producer ----
+    if (lane == 0) {
+      for (int i = 0; i < pre; ++i)
+        bulk_copy_g2s(ring + (size_t)i * (kTcABytes + kTcBBytes) + kTcABytes, gB + (size_t)i * (kMaxRows * 128), kTcBBytes, full + i);
+      for (int i = pre; i < n_it; ++i) {
+        const int s = i % kTcStages;
+        tc_wait(empty + s, ((i / kTcStages) - 1) & 1, failed, a.err);
+        mbar_expect_tx(full + s, kTcABytes + kTcBBytes);
+        bulk_copy_g2s(ring + (size_t)s * (kTcABytes + kTcBBytes), gA + (size_t)i * kTcABytes, kTcABytes, full + s);
+        bulk_copy_g2s(ring + (size_t)s * (kTcABytes + kTcBBytes) + kTcABytes, gB + (size_t)i * (kMaxRows * 128), kTcBBytes, full + s);
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ----
+    if (lane == 0) {
+      const uint32_t idesc = tc_instr_desc(kTcTileM, kTcChunkN);
+      for (int i = 0; i < n_it; ++i) {
+        const int s = i % kTcStages;
+        tc_wait(full + s, (i / kTcStages) & 1, failed, a.err);
+        tc_fence_after_sync();
+        const unsigned char *sa = ring + (size_t)s * (kTcABytes + kTcBBytes);
+        const uint64_t da = tc_smem_desc(sa), db = tc_smem_desc(sa + kTcABytes);
+#pragma unroll
+        for (int j = 0; j < kTcKChunk / 16; ++j)   // 32 bytes further along K per step: +2 in 16-byte units
+          tc_mma(tmem_d, da + 2 * j, db + 2 * j, idesc, (i > 0 || j > 0) ? 1u : 0u);
+        tc_commit(empty + s);   // the stage may be refilled once these MMAs have read it
+      }
+      tc_commit(acc_done);
+    }
+  }
+  __syncwarp();   // the other lanes of warps 0 and 1 wait here for their lane 0
+
+  // ---- epilogue: warp w owns accumulator lanes 32w..32w+31 = weight rows n; columns = batch rows ----
+  tc_wait(acc_done, 0, failed, a.err);
+  tc_fence_after_sync();
+  __syncwarp();
+  float v[32];
+  tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16), v);
+  if (n_it <= 0) {   // an empty k-range contributes nothing (the accumulator was never written)
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = 0.f;
+  }
+  const int n = nt * kTcTileM + warp * 32 + lane;
+  if (n < a.N && !*failed) {
+    const float bias = (a.bias && (a.mode != EPI_RESID || a.ksplit == 1)) ? bf16_bits_to_float(a.bias[n]) : 0.f;
+#pragma unroll
+    for (int c = 0; c < kTcChunkN; ++c) {
+      const int b = bc * kTcChunkN + c;
+      if (b >= a.B) break;
+      float r = v[c] + bias;
+      if (a.mode == EPI_F32) {
+        a.out_f32[(size_t)b * a.out_stride + n] = r;
+      } else if (a.mode == EPI_RESID) {
+        if (a.ksplit == 1) a.out_f32[(size_t)b * a.out_stride + n] += r;
+        else a.out_f32[((size_t)ks * kMaxRows + b) * a.N + n] = r;
+      } else if (a.mode == EPI_GELU) {
+        r = a.gelu_tanh ? gelu_tanh_f(r) : gelu_erf_f(r);
+        *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + image_offset(b, n, kMaxRows)) = float_to_bf16_bits(r);
+      } else {  // EPI_QKV
+        if (n < a.d) {
+          a.out_f32[(size_t)b * a.out_stride + n] = r;
+        } else {
+          const int which = n >= 2 * a.d;
+          const int col = n - (which ? 2 * a.d : a.d);
+          kv_base[c][((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63)] = float_to_bf16_bits(r);
+        }
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_d, 32);
+}
+
+// out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)
+__global__ void fold_partials_kernel(const float *__restrict__ part, int n_part, int B, int N,
+                                     const uint16_t *__restrict__ bias, float *__restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)B * N) return;
+  const int b = i / N, n = i % N;
+  float v = bias ? bf16_bits_to_float(bias[n]) : 0.f;
+  for (int p = 0; p < n_part; ++p) v += part[((size_t)p * kMaxRows + b) * N + n];
+  out[i] = v;
+}
+
+inline size_t gemm_tc_smem_bytes() { return (size_t)kTcStages * (kTcABytes + kTcBBytes) + 1024 + 512; }
+
+inline cudaError_t launch_gemm_tc(const GemmTcArgs &a, cudaStream_t st, bool pdl) {
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
+    attr_done = true;
+  }
+  dim3 grid((a.N + kTcTileM - 1) / kTcTileM, (a.B + kTcChunkN - 1) / kTcChunkN, a.ksplit);
+  return launch_kernel(gemm_tc_kernel, grid, dim3(kTcThreads), gemm_tc_smem_bytes(), st, pdl, a);
+}
+
+}  // namespace ttsgpt

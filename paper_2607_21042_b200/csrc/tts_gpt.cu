@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "linear.cuh"
 #include "attention.cuh"
+#include "gemm_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
 
@@ -25,6 +26,7 @@ namespace {
 thread_local std::string g_last_error;
 
 struct PackedLinear {
+  void *w_img = nullptr;   // bf16 only: operand image for the tensor-core path (rows padded to 128)
   void *w = nullptr;
   uint16_t *s = nullptr;
   uint16_t *bias = nullptr;
@@ -57,6 +59,10 @@ struct tts_gpt {
   // activations
   float *x, *q, *logits;
   uint16_t *a, *o, *hbuf, *hf;
+  // tensor-core path (more than 16 rows, bf16 weights): activation images and k-split partial sums
+  void *a_img = nullptr, *o_img = nullptr, *h_img = nullptr, *hf_img = nullptr;
+  float *partials = nullptr;
+  bool have_tc = false;
   // attention scratch
   float *attn_partials;
   unsigned int *attn_tickets;
@@ -69,6 +75,7 @@ struct tts_gpt {
   std::map<int, int> graph_nodes;
   bool use_graph;
   bool use_pdl;
+  bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
   int n_sm = 148;
   unsigned long long launches = 0;
   int *dev_err = nullptr;               // error word set by a kernel whose bounded wait expired:
@@ -127,6 +134,7 @@ struct Carver {
 
 void carve_linear(Carver &cv, PackedLinear &pl, int wf, int N, int K) {
   pl.N = N; pl.K = K;
+  pl.w_img = (wf == WF_BF16 && K % 64 == 0) ? cv.take<char>(weight_image_bytes(N, K)) : nullptr;
   pl.w = cv.take<char>(packed_weight_bytes(wf, N, K));
   size_t sb = packed_scale_bytes(wf, N, K);
   pl.s = sb ? cv.take<uint16_t>(sb / 2) : nullptr;
@@ -182,6 +190,14 @@ size_t carve(tts_gpt *h, void *base) {
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
   h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
+  h->have_tc = c.wfmt == WF_BF16;
+  if (h->have_tc) {
+    h->a_img = cv.take<char>(act_image_bytes(d));
+    h->o_img = cv.take<char>(act_image_bytes(d));
+    h->h_img = cv.take<char>(act_image_bytes(F));
+    h->hf_img = cv.take<char>(act_image_bytes(d));
+    h->partials = cv.take<float>((size_t)kTcKSplit * kMaxRows * d);
+  }
   return cv.off;
 }
 
@@ -194,6 +210,11 @@ int copy_bf16(tts_gpt *h, uint16_t *dst, const void *src, size_t n, const char *
 int load_linear(tts_gpt *h, PackedLinear &pl, int wf, const void *w, const void *s, const void *b, const char *what) {
   if (!w || !b || (wf != WF_BF16 && !s)) return fail(h, TTS_GPT_E_ARG, "weights: %s has a null tensor", what);
   CUDA_TRY(h, launch_pack(wf, pl.N, pl.K, w, s, pl.w, pl.s, h->stream));
+  if (pl.w_img) {
+    const size_t units = weight_image_bytes(pl.N, pl.K) / 16;
+    pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, h->stream>>>((const uint16_t *)w, pl.N, pl.K, (uint4 *)pl.w_img);
+    CUDA_TRY(h, cudaGetLastError());
+  }
   CUDA_TRY(h, cudaMemcpyAsync(pl.bias, b, (size_t)pl.N * 2, cudaMemcpyDeviceToDevice, h->stream));
   return TTS_GPT_OK;
 }
@@ -223,8 +244,101 @@ void trace_attach(tts_gpt *h, Args &a) {
 // The transformer blocks for R rows already described by the row table, x holding the input rows.
 // Every kernel after the first of a step is launched with programmatic dependent launch, so its
 // weight loads overlap the tail of its predecessor.
+// ---- tensor-core path: more than 16 rows, bf16 weights ----
+GemmTcArgs gemm_args(tts_gpt *h, const PackedLinear &pl, const void *act_img, int B, int mode, int ksplit) {
+  GemmTcArgs a;
+  memset(&a, 0, sizeof a);
+  a.w_img = pl.w_img; a.act_img = act_img; a.bias = pl.bias; a.N = pl.N; a.K = pl.K; a.B = B; a.mode = mode;
+  a.ksplit = ksplit; a.err = h->dev_err;
+  return a;
+}
+
+int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int n_part, const uint16_t *add_bias,
+                 void *out_img, uint16_t *out_plain, const int *gather, const int *out_slot, const StepIO *io,
+                 int write_back) {
+  LnTcArgs la;
+  memset(&la, 0, sizeof la);
+  la.x = h->x; la.d = h->cfg.d_model; la.partials = h->partials; la.n_part = n_part; la.part_cols = h->cfg.d_model;
+  la.add_bias = add_bias; la.g = g; la.b = b; la.eps = h->cfg.ln_eps; la.out_img = out_img; la.out_plain = out_plain;
+  la.gather = gather; la.out_slot = out_slot; la.io = io; la.write_back = write_back;
+  CUDA_TRY(h, launch_kernel(layernorm_tc_kernel, dim3(rows), dim3(kLnThreads), 0, h->stream, h->use_pdl, la));
+  h->launches += 1;
+  return TTS_GPT_OK;
+}
+
+int run_layers_tc(tts_gpt *h, int R, bool decode) {
+  const tts_gpt_config_t &c = h->cfg;
+  const int d = c.d_model;
+  cudaStream_t st = h->stream;
+  const bool pdl = h->use_pdl;
+  for (int l = 0; l < c.n_layer; ++l) {
+    LayerW &L = h->layers[l];
+    uint16_t *kvl = h->kv + h->kv_layer_elems * l;
+    // fold the previous layer's FC2 partial sums into x, then LN1 -> image
+    int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : kTcKSplit, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
+                          h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
+    if (rc) return rc;
+    GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
+    qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
+    qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+    CUDA_TRY(h, launch_gemm_tc(qa, st, pdl));
+    AttnArgs aa;
+    memset(&aa, 0, sizeof aa);
+    aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
+    aa.row_pos = h->rt.row_pos; aa.out = (uint16_t *)h->o_img; aa.out_image = 1;
+    aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
+    CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
+    GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, kTcKSplit);
+    oa.out_f32 = h->partials; oa.out_stride = d;
+    CUDA_TRY(h, launch_gemm_tc(oa, st, pdl));
+    rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, kTcKSplit, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
+    if (rc) return rc;
+    GemmTcArgs f1 = gemm_args(h, L.fc1, h->a_img, R, EPI_GELU, 1);
+    f1.out_img = h->h_img; f1.gelu_tanh = c.gelu_tanh;
+    CUDA_TRY(h, launch_gemm_tc(f1, st, pdl));
+    GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, kTcKSplit);
+    f2.out_f32 = h->partials; f2.out_stride = d;
+    CUDA_TRY(h, launch_gemm_tc(f2, st, pdl));
+    h->launches += 5;
+  }
+  return TTS_GPT_OK;
+}
+
+// Final LayerNorm (folding the last FC2's partial sums), LM head, sampling after run_layers_tc.
+int run_head_tc(tts_gpt *h, int n_out) {
+  const tts_gpt_config_t &c = h->cfg;
+  cudaStream_t st = h->stream;
+  const bool pdl = h->use_pdl;
+  const bool big = n_out > 16;
+  int rc = launch_ln_tc(h, n_out, h->lnf_g, h->lnf_b, kTcKSplit, h->layers[c.n_layer - 1].fc2.bias,
+                        big ? h->hf_img : nullptr, big ? nullptr : h->hf, h->rt.out_rows, h->rt.out_slot, h->io, 0);
+  if (rc) return rc;
+  if (big) {
+    GemmTcArgs ha = gemm_args(h, h->head, h->hf_img, n_out, EPI_F32, 1);
+    ha.out_f32 = h->logits; ha.out_stride = c.vocab;
+    CUDA_TRY(h, launch_gemm_tc(ha, st, pdl));
+  } else {
+    LinearArgs ha = linear_args(h, h->head, h->hf, n_out, EPI_F32);
+    ha.out_f32 = h->logits; ha.out_stride = c.vocab;
+    CUDA_TRY(h, launch_linear(WF_BF16, ha, st, pdl, 2 * h->n_sm));
+  }
+  SampleArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.logits = h->logits; sa.V = c.vocab; sa.io = h->io; sa.out_slot = h->rt.out_slot; sa.out_rows = h->rt.out_rows;
+  sa.row_stream = h->rt.row_stream; sa.last_token = h->ps.last_token; sa.stop_flag = h->ps.stop_flag;
+  sa.stop_token = c.stop_token;
+  CUDA_TRY(h, launch_kernel(sample_kernel, dim3(n_out), dim3(kSampleThreads), (size_t)c.vocab * sizeof(float), st, pdl, sa));
+  h->launches += 2;
+  return TTS_GPT_OK;
+}
+
+bool use_tc_path(const tts_gpt *h, int R) {
+  return h->have_tc && h->use_tc && R > 16;
+}
+
 int run_layers(tts_gpt *h, int R, bool decode) {
   h->trace_next = 0;
+  if (use_tc_path(h, R)) return run_layers_tc(h, R, decode);
   const tts_gpt_config_t &c = h->cfg;
   const int d = c.d_model;
   cudaStream_t st = h->stream;
@@ -278,7 +392,8 @@ int run_layers(tts_gpt *h, int R, bool decode) {
 }
 
 // Final LayerNorm (gathered to the wanted rows), LM head, sampling.
-int run_head(tts_gpt *h, int n_out) {
+int run_head(tts_gpt *h, int n_out, int R) {
+  if (use_tc_path(h, R)) return run_head_tc(h, n_out);
   const tts_gpt_config_t &c = h->cfg;
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
@@ -359,6 +474,11 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   if (!w->head_w) { delete h; return fail(nullptr, TTS_GPT_E_ARG, "weights: head_w is null"); }
   {
     cudaError_t e = launch_pack(WF_BF16, h->head.N, h->head.K, w->head_w, nullptr, h->head.w, nullptr, h->stream);
+    if (e == cudaSuccess && h->head.w_img) {
+      const size_t units = weight_image_bytes(h->head.N, h->head.K) / 16;
+      pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, h->stream>>>((const uint16_t *)w->head_w, h->head.N, h->head.K, (uint4 *)h->head.w_img);
+      e = cudaGetLastError();
+    }
     if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "pack head: %s", cudaGetErrorString(e)); }
     if (w->head_b) {
       TRY_(copy_bf16(h, h->head.bias, w->head_b, c.vocab, "head_b"));
@@ -419,6 +539,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
     if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
       h->n_sm = sms;
   }
+  const char *ntc = getenv("TTS_GPT_NO_TC");
+  h->use_tc = !(ntc && ntc[0] == '1');
   const char *np = getenv("TTS_GPT_NO_PDL");
   h->use_pdl = !(np && np[0] == '1');
   *out = h;
@@ -481,7 +603,7 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     if (r) return r;
     r = run_layers(h, ps.n_rows, false);
     if (r) return r;
-    if (ps.n_out > 0) r = run_head(h, ps.n_out);
+    if (ps.n_out > 0) r = run_head(h, ps.n_out, ps.n_rows);
     ps.n_rows = 0; ps.n_out = 0;
     return r;
   };
@@ -542,7 +664,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
       CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
       rc = run_embed(h, n);
       if (!rc) rc = run_layers(h, n, true);
-      if (!rc) rc = run_head(h, n);
+      if (!rc) rc = run_head(h, n, n);
       cudaError_t e = cudaStreamEndCapture(h->stream, &g);
       if (rc) { if (g) cudaGraphDestroy(g); return rc; }
       if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph capture: %s", cudaGetErrorString(e));
@@ -560,7 +682,7 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   }
   rc = run_embed(h, n);
   if (!rc) rc = run_layers(h, n, true);
-  if (!rc) rc = run_head(h, n);
+  if (!rc) rc = run_head(h, n, n);
   return rc;
 }
 
@@ -674,6 +796,45 @@ int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed
   LinearArgs a = linear_args(pl, (const uint16_t *)act, B, EPI_F32);
   a.out_f32 = out; a.out_stride = N;
   CUDA_TRY(nullptr, launch_linear(wfmt, a, (cudaStream_t)cuda_stream, false));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_linear_tc_scratch_bytes(int32_t N, int32_t K, size_t *bytes) {
+  if (N < 1 || K < 64 || K % 64 || !bytes) return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad shape");
+  *bytes = align256(weight_image_bytes(N, K)) + align256(act_image_bytes(K)) +
+           align256((size_t)kTcKSplit * kMaxRows * N * sizeof(float));
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_op_linear_tc(int32_t N, int32_t K, const void *w, const void *bias, int32_t B, const void *act,
+                             float *out, int32_t ksplit, void *scratch, void *cuda_stream) {
+  size_t bytes;
+  int rc = tts_gpt_op_linear_tc_scratch_bytes(N, K, &bytes);
+  if (rc) return rc;
+  if (!w || !act || !out || !scratch || B < 1 || B > kMaxRows || (uintptr_t)scratch % 1024 ||
+      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad argument");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char *wimg = (char *)scratch;
+  char *aimg = wimg + align256(weight_image_bytes(N, K));
+  float *part = (float *)(aimg + align256(act_image_bytes(K)));
+  const size_t units = weight_image_bytes(N, K) / 16;
+  pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, st>>>((const uint16_t *)w, N, K, (uint4 *)wimg);
+  const size_t au = (size_t)B * (K / 8);
+  pack_act_image_kernel<<<(unsigned)((au + 255) / 256), 256, 0, st>>>((const uint16_t *)act, B, K, (unsigned char *)aimg);
+  CUDA_TRY(nullptr, cudaGetLastError());
+  GemmTcArgs a;
+  memset(&a, 0, sizeof a);
+  a.w_img = wimg; a.act_img = aimg; a.N = N; a.K = K; a.B = B; a.ksplit = ksplit;
+  if (ksplit == 1) {
+    a.mode = EPI_F32; a.bias = (const uint16_t *)bias; a.out_f32 = out; a.out_stride = N;
+    CUDA_TRY(nullptr, launch_gemm_tc(a, st, false));
+  } else {   // partial sums per k-range, then folded in range order (what the following LayerNorm does in the engine)
+    a.mode = EPI_RESID; a.out_f32 = part; a.out_stride = N;
+    CUDA_TRY(nullptr, launch_gemm_tc(a, st, false));
+    fold_partials_kernel<<<(unsigned)(((size_t)B * N + 255) / 256), 256, 0, st>>>(part, ksplit, B, N, (const uint16_t *)bias, out);
+    CUDA_TRY(nullptr, cudaGetLastError());
+  }
   return TTS_GPT_OK;
 }
 
