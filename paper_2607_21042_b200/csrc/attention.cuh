@@ -6,9 +6,9 @@
 //
 // Work split.  A (row, head) pair is handled by a thread-block cluster of S CTAs (S = 1, 2, 4 or 8,
 // picked per launch so that the grid fills the GPU: S = 8 at batch 1, S = 1 at batch 128).  The
-// row's pages are dealt round-robin: CTA c of the cluster takes pages c, c+S, c+2S, ...; inside a
-// CTA its 4 warps take those in turn.  One warp streams a page's 8 KB K block and 8 KB V block
-// with 16+16 independent 128-bit loads per lane, keeps scores, the running softmax statistics
+// row's pages are cut into quarter-page units of 16 tokens dealt round-robin over all 4*S warps of
+// the cluster (with S = 1: whole pages over the CTA's 4 warps).  One warp streams 64 tokens of K and
+// V at a time (a whole page, or four quarters) with 16+16 independent 128-bit loads per lane, keeps scores, the running softmax statistics
 // (max, sum) and the running output in fp32 registers (online softmax across its pages), and uses
 // shuffles for the reductions.  The warps of a CTA meet in shared memory; the CTAs of a cluster
 // meet in distributed shared memory: rank 0 reads the other ranks' (max, sum, output) triples and
@@ -64,15 +64,17 @@ __device__ __forceinline__ void load_page(PageLoad &pl, const uint16_t *K, const
   for (int i = 0; i < 16; ++i) pl.vv[i] = ld_stream_u4(V + (size_t)(tg + 4 * i) * kHeadDim + 8 * sub);
 }
 
-// Folds one page into the warp's running (m, l, o).  Lane (tg, sub) = (lane/8, lane%8) sees tokens
-// tg, tg+4, ... and elements 8*sub..8*sub+7 of the head; m and l are warp-uniform, o[e] is the
-// lane's partial over its tokens (summed over tg at the very end).
-__device__ __forceinline__ void fold_page(PageLoad &pl, const float (&qv)[8], int n_here, int tg, float &m, float &l,
-                                          float (&o)[8]) {
-  float s[16];
+// Folds the 16 token slots a lane holds into the warp's running (m, l, o).  Lane (tg, sub) =
+// (lane/8, lane%8) holds elements 8*sub..8*sub+7 of 16 tokens (bit i of vmask: slot i is a real
+// token); m and l are warp-uniform, o[e] is the lane's partial over its tokens (summed over tg at
+// the very end).  At least one slot of the warp must be valid.
+template <int NS>
+__device__ __forceinline__ void fold_first(PageLoad &pl, const float (&qv)[8], uint32_t vmask, float &m, float &l,
+                                           float (&o)[8]) {
+  float s[NS];
   float pm = -INFINITY;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < NS; ++i) {
     float d = qv[0] * bf16_lo(pl.kk[i].x);
     d = fmaf(qv[1], bf16_hi(pl.kk[i].x), d);
     d = fmaf(qv[2], bf16_lo(pl.kk[i].y), d);
@@ -84,20 +86,20 @@ __device__ __forceinline__ void fold_page(PageLoad &pl, const float (&qv)[8], in
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
-    const bool valid = tg + 4 * i < n_here;
+    const bool valid = (vmask >> i) & 1u;
     s[i] = valid ? d : -INFINITY;
     if (!valid) pl.vv[i] = make_uint4(0, 0, 0, 0);  // stale page contents may hold NaN: 0 * NaN must not reach o
     pm = fmaxf(pm, s[i]);
   }
   pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 8));
   pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 16));
-  const float m_new = fmaxf(m, pm);           // finite: every page has at least one valid token
-  const float rescale = exp2f(m - m_new);     // first page: exp2(-inf) = 0
+  const float m_new = fmaxf(m, pm);           // finite: the caller only folds batches with a valid token
+  const float rescale = exp2f(m - m_new);     // first batch: exp2(-inf) = 0
   float lp = 0.f;
 #pragma unroll
   for (int e = 0; e < 8; ++e) o[e] *= rescale;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
+  for (int i = 0; i < NS; ++i) {
     const float p = exp2f(s[i] - m_new);  // masked tokens: exp2(-inf) = 0
     lp += p;
     o[0] = fmaf(p, bf16_lo(pl.vv[i].x), o[0]);
@@ -113,6 +115,57 @@ __device__ __forceinline__ void fold_page(PageLoad &pl, const float (&qv)[8], in
   lp += __shfl_xor_sync(0xFFFFFFFFu, lp, 16);
   l = l * rescale + lp;
   m = m_new;
+}
+
+// ng (warp-uniform): how many groups of 4 slots hold tokens at all; they are always the first ones,
+// and the absent ones are not even looked at, which is what makes short batches cheap
+__device__ __forceinline__ void fold_slots(PageLoad &pl, const float (&qv)[8], uint32_t vmask, int ng, float &m,
+                                           float &l, float (&o)[8]) {
+  if (ng >= 4) fold_first<16>(pl, qv, vmask, m, l, o);
+  else if (ng == 3) fold_first<12>(pl, qv, vmask, m, l, o);
+  else if (ng == 2) fold_first<8>(pl, qv, vmask, m, l, o);
+  else fold_first<4>(pl, qv, vmask, m, l, o);
+}
+
+__device__ __forceinline__ void fold_page(PageLoad &pl, const float (&qv)[8], int n_here, int tg, float &m, float &l,
+                                          float (&o)[8]) {
+  uint32_t vmask = 0u;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) vmask |= (tg + 4 * i < n_here) ? (1u << i) : 0u;
+  fold_first<16>(pl, qv, vmask, m, l, o);
+}
+
+// Quarter-page batches for clusters: the row's pages are cut into units of 16 tokens, unit u =
+// 4*page + quarter; a warp's batch holds 4 units u0, u0+stride, ... (slots 4j..4j+3 = unit j, tokens
+// tg, tg+4, tg+8, tg+12 of the quarter), so that even a short context keeps every warp of every
+// CTA of the cluster busy with 32 loads in flight.
+__device__ __forceinline__ uint32_t load_quarters(PageLoad &pl, const uint16_t *kv_layer, const int *pt, int H, int h,
+                                                  int u0, int stride, int n_units, int n_tok, int tg, int sub,
+                                                  int &ng) {
+  uint32_t vmask = 0u;
+  ng = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int u = u0 + stride * j;
+    if (u < n_units) {
+      ng = j + 1;
+      const int page = u >> 2, qt = u & 3;
+      const int phys = pt[page];
+      const uint16_t *K = kv_layer + (((size_t)phys * 2 + 0) * H + h) * kPageElems + (size_t)(16 * qt) * kHeadDim;
+      const uint16_t *V = kv_layer + (((size_t)phys * 2 + 1) * H + h) * kPageElems + (size_t)(16 * qt) * kHeadDim;
+      const int left = n_tok - page * kPageTokens - 16 * qt;   // tokens of the row from this quarter on
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii) {
+        pl.kk[4 * j + ii] = ld_stream_u4(K + (size_t)(tg + 4 * ii) * kHeadDim + 8 * sub);
+        pl.vv[4 * j + ii] = ld_stream_u4(V + (size_t)(tg + 4 * ii) * kHeadDim + 8 * sub);
+        if (tg + 4 * ii < left) vmask |= 1u << (4 * j + ii);
+      }
+    } else {
+#pragma unroll
+      for (int ii = 0; ii < 4; ++ii) { pl.kk[4 * j + ii] = make_uint4(0, 0, 0, 0); pl.vv[4 * j + ii] = make_uint4(0, 0, 0, 0); }
+    }
+  }
+  return vmask;
 }
 
 __device__ __forceinline__ void load_q(float (&qv)[8], const float *q) {
@@ -170,39 +223,73 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
   __shared__ float cl_part[kAttnPartialFloats];  // this CTA's (M, L, O[64]) for the cluster merge
 
-  // this warp's pages: c + S*(warp + kAttnWarps*it)
-  int page = c + S * warp;
-  PageLoad pl;
-  // In a decode step the only K/V entry of the row that this step writes is the new token's own
-  // (position n_tok-1, by the QKV kernel in front).  The warp's first page is therefore requested
-  // before waiting for that kernel; if it is the row's last page, the new token's 128-byte K and V
-  // rows are fetched again after the wait.
-  const bool early = a.old_pages_final && page < n_pages;
-  const uint16_t *K0 = nullptr, *V0 = nullptr;
-  if (early) {
-    const int phys = pt[page];
-    K0 = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
-    V0 = a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems;
-    load_page(pl, K0, V0, tg, sub);
-  }
-  pdl_launch_dependents();
-  pdl_wait();
-  trace_mark(a.trace, a.trace_slot, 1);
-
   float m = -INFINITY, l = 0.f;
   float o[8];
 #pragma unroll
   for (int e = 0; e < 8; ++e) o[e] = 0.f;
   float qv[8];
-  load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
-  if (early && page == n_pages - 1) {
-    const int tn = (n_tok - 1) & (kPageTokens - 1);   // the new token's slot in its page
-    if ((tn & 3) == tg) {
+  PageLoad pl;
+  // In a decode step the only K/V entry of the row that this step writes is the new token's own
+  // (position n_tok-1, by the QKV kernel in front).  The warp's first batch of loads is therefore
+  // requested before waiting for that kernel; if it covers the new token, that token's 128-byte K
+  // and V rows are fetched again after the wait.
+  const int tn = (n_tok - 1) & (kPageTokens - 1);   // the new token's slot in the last page
+  if (S > 1) {
+    // ---- cluster: quarter-page units dealt round-robin over all warps of the cluster ----
+    const int GW = S * kAttnWarps, gw = c * kAttnWarps + warp;
+    const int n_units = (n_tok + 15) >> 4;   // units that hold at least one token
+    const bool early = a.old_pages_final && gw < n_units;
+    uint32_t vmask = 0u;
+    int ng = 0;
+    if (early) vmask = load_quarters(pl, a.kv_layer, pt, a.H, h, gw, GW, n_units, n_tok, tg, sub, ng);
+    pdl_launch_dependents();
+    pdl_wait();
+    trace_mark(a.trace, a.trace_slot, 1);
+    load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+    if (early) {
+      const int us = 4 * (n_pages - 1) + (tn >> 4);   // unit of the new token
+      if (us % GW == gw && us / GW < 4 && (tn & 3) == tg) {
+        const int phys = pt[n_pages - 1];
+        const uint4 kn = ld_cg_u4(a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems + (size_t)tn * kHeadDim + 8 * sub);
+        const uint4 vn = ld_cg_u4(a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems + (size_t)tn * kHeadDim + 8 * sub);
+        const int sel = 4 * (us / GW) + ((tn & 15) >> 2);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {  // register selects (no dynamic indexing of the page registers)
+          const bool hit = i == sel;
+          pl.kk[i].x = hit ? kn.x : pl.kk[i].x; pl.kk[i].y = hit ? kn.y : pl.kk[i].y;
+          pl.kk[i].z = hit ? kn.z : pl.kk[i].z; pl.kk[i].w = hit ? kn.w : pl.kk[i].w;
+          pl.vv[i].x = hit ? vn.x : pl.vv[i].x; pl.vv[i].y = hit ? vn.y : pl.vv[i].y;
+          pl.vv[i].z = hit ? vn.z : pl.vv[i].z; pl.vv[i].w = hit ? vn.w : pl.vv[i].w;
+        }
+      }
+    }
+    bool loaded = early;
+    for (int u0 = gw; u0 < n_units; u0 += 4 * GW) {
+      if (!loaded) vmask = load_quarters(pl, a.kv_layer, pt, a.H, h, u0, GW, n_units, n_tok, tg, sub, ng);
+      loaded = false;
+      fold_slots(pl, qv, vmask, ng, m, l, o);
+    }
+  } else {
+    // ---- one CTA per (row, head): whole pages, warp w takes pages w, w+4, ... ----
+    int page = warp;
+    const bool early = a.old_pages_final && page < n_pages;
+    const uint16_t *K0 = nullptr, *V0 = nullptr;
+    if (early) {
+      const int phys = pt[page];
+      K0 = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
+      V0 = a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems;
+      load_page(pl, K0, V0, tg, sub);
+    }
+    pdl_launch_dependents();
+    pdl_wait();
+    trace_mark(a.trace, a.trace_slot, 1);
+    load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+    if (early && page == n_pages - 1 && (tn & 3) == tg) {
       const uint4 kn = ld_cg_u4(K0 + (size_t)tn * kHeadDim + 8 * sub);
       const uint4 vn = ld_cg_u4(V0 + (size_t)tn * kHeadDim + 8 * sub);
       const int sel = tn >> 2;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {  // register selects (no dynamic indexing of the page registers)
+      for (int i = 0; i < 16; ++i) {
         const bool hit = i == sel;
         pl.kk[i].x = hit ? kn.x : pl.kk[i].x; pl.kk[i].y = hit ? kn.y : pl.kk[i].y;
         pl.kk[i].z = hit ? kn.z : pl.kk[i].z; pl.kk[i].w = hit ? kn.w : pl.kk[i].w;
@@ -210,16 +297,16 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
         pl.vv[i].z = hit ? vn.z : pl.vv[i].z; pl.vv[i].w = hit ? vn.w : pl.vv[i].w;
       }
     }
-  }
-  bool loaded = early;
-  for (; page < n_pages; page += S * kAttnWarps) {
-    if (!loaded) {
-      const int phys = pt[page];
-      load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
-                a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
+    bool loaded = early;
+    for (; page < n_pages; page += kAttnWarps) {
+      if (!loaded) {
+        const int phys = pt[page];
+        load_page(pl, a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems,
+                  a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems, tg, sub);
+      }
+      loaded = false;
+      fold_page(pl, qv, min(kPageTokens, n_tok - page * kPageTokens), tg, m, l, o);
     }
-    loaded = false;
-    fold_page(pl, qv, min(kPageTokens, n_tok - page * kPageTokens), tg, m, l, o);
   }
   trace_mark(a.trace, a.trace_slot, 3);
   float M, L, O;

@@ -128,19 +128,35 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   const int j = blockIdx.x;
   const int r = a.gather ? a.gather[j] : j;
   float *xr = a.x + (size_t)r * a.d;
-  float v[kLnMaxPerThread];
+  // all loads of the row (x, bias and up to 4 partial sums per element) are issued before any is
+  // used; the sum itself is taken in a fixed order
+  constexpr int kMaxPart = 4;
+  float v[kLnMaxPerThread], bs[kLnMaxPerThread], pp[kLnMaxPerThread][kMaxPart];
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    v[i] = 0.f; bs[i] = 0.f;
+#pragma unroll
+    for (int p = 0; p < kMaxPart; ++p) pp[i][p] = 0.f;
+    if (c < a.d) {
+      v[i] = xr[c];
+      if (a.n_part > 0) {
+        if (a.add_bias) bs[i] = bf16_bits_to_float(a.add_bias[c]);
+#pragma unroll
+        for (int p = 0; p < kMaxPart; ++p)
+          if (p < a.n_part) pp[i][p] = __ldcg(a.partials + ((size_t)p * kMaxRows + r) * a.part_cols + c);
+      }
+    }
+  }
   float s = 0.f;
 #pragma unroll
   for (int i = 0; i < kLnMaxPerThread; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
-    v[i] = 0.f;
-    if (c < a.d) {
-      float t = xr[c];
-      if (a.n_part > 0) {
-        if (a.add_bias) t += bf16_bits_to_float(a.add_bias[c]);
-        for (int p = 0; p < a.n_part; ++p) t += a.partials[((size_t)p * kMaxRows + r) * a.part_cols + c];
-        if (a.write_back) xr[c] = t;
-      }
+    if (c < a.d && a.n_part > 0) {
+      float t = v[i] + bs[i];
+#pragma unroll
+      for (int p = 0; p < kMaxPart; ++p) t += pp[i][p];
+      if (a.write_back) xr[c] = t;
       v[i] = t;
     }
     s += v[i];
