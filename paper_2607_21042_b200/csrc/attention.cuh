@@ -10,9 +10,9 @@
 // the cluster (with S = 1: whole pages over the CTA's 4 warps).  One warp streams 64 tokens of K and
 // V at a time (a whole page, or four quarters) with 16+16 independent 128-bit loads per lane, keeps scores, the running softmax statistics
 // (max, sum) and the running output in fp32 registers (online softmax across its pages), and uses
-// shuffles for the reductions.  The warps of a CTA meet in shared memory; the CTAs of a cluster
-// meet in distributed shared memory: rank 0 reads the other ranks' (max, sum, output) triples and
-// merges them by log-sum-exp in rank order.  No global scratch, no atomics, no spinning; the
+// shuffles for the reductions.  The warps of a CTA meet in shared memory; in a cluster every CTA
+// stores its (max, sum, output) triple into rank 0's shared memory (distributed shared memory) and,
+// after one cluster barrier, rank 0 merges them by log-sum-exp in rank order.  No global scratch, no atomics, no spinning; the
 // result does not depend on timing.
 //
 // A second variant (`attention_ticket_kernel`) exchanges the partial results through global
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   const int *pt = a.page_table + (size_t)a.row_stream[r] * a.pps;
 
   __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
-  __shared__ float cl_part[kAttnPartialFloats];  // this CTA's (M, L, O[64]) for the cluster merge
+  __shared__ float cl_all[kAttnMaxCluster][kAttnPartialFloats];  // rank 0: every rank's (M, L, O[64])
 
   float m = -INFINITY, l = 0.f;
   float o[8];
@@ -309,9 +309,6 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
     }
   }
   trace_mark(a.trace, a.trace_slot, 3);
-  float M, L, O;
-  cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
-  trace_mark(a.trace, a.trace_slot, 4);
   const int e = threadIdx.x;
   // plain row-major bf16, or the image layout of the tensor-core linear that consumes it
   uint16_t *out = nullptr;
@@ -319,27 +316,32 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
     out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
                       : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
   if (S == 1) {
+    float M, L, O;
+    cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
     if (e < kHeadDim) *out = float_to_bf16_bits(O / L);
     trace_mark(a.trace, a.trace_slot, 2);
     return;
   }
+  // ---- cluster merge: the CTA merges its warps locally, stores its (M, L, O[64]) straight into
+  //      rank 0's shared memory (distributed shared memory), one cluster barrier, then rank 0 merges
+  //      the S partial results in rank order; the other ranks are done once the barrier is passed ----
   cg::cluster_group cluster = cg::this_cluster();
+  float M, L, O;
+  cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
   if (e < kHeadDim) {
-    if (e == 0) { cl_part[0] = M; cl_part[1] = L; }
-    cl_part[2 + e] = O;
+    float *dst = cluster.map_shared_rank(&cl_all[0][0], 0) + (size_t)c * kAttnPartialFloats;
+    if (e == 0) { dst[0] = M; dst[1] = L; }
+    dst[2 + e] = O;
   }
+  trace_mark(a.trace, a.trace_slot, 4);
   cluster.sync();
   trace_mark(a.trace, a.trace_slot, 5);
   if (c == 0 && e < kHeadDim) {
-    // all remote reads are issued before any is used
     float pm[kAttnMaxCluster], pl_[kAttnMaxCluster], po[kAttnMaxCluster];
 #pragma unroll
-    for (int rr = 0; rr < kAttnMaxCluster; ++rr) {
+    for (int rr = 0; rr < kAttnMaxCluster; ++rr) {   // all reads issued before any is used
       pm[rr] = -INFINITY; pl_[rr] = 0.f; po[rr] = 0.f;
-      if (rr < S) {
-        const float *p = cluster.map_shared_rank(cl_part, rr);
-        pm[rr] = p[0]; pl_[rr] = p[1]; po[rr] = p[2 + e];
-      }
+      if (rr < S) { pm[rr] = cl_all[rr][0]; pl_[rr] = cl_all[rr][1]; po[rr] = cl_all[rr][2 + e]; }
     }
     float MM = -INFINITY;
 #pragma unroll
@@ -347,13 +349,12 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
     float LL = 0.f, OO = 0.f;
 #pragma unroll
     for (int rr = 0; rr < kAttnMaxCluster; ++rr) {
-      const float f = (pm[rr] == -INFINITY) ? 0.f : exp2f(pm[rr] - MM);  // a rank without pages contributes nothing
+      const float f = (pm[rr] == -INFINITY) ? 0.f : exp2f(pm[rr] - MM);  // a rank without tokens contributes nothing
       LL = fmaf(pl_[rr], f, LL);
       OO = fmaf(po[rr], f, OO);
     }
     *out = float_to_bf16_bits(OO / LL);
   }
-  cluster.sync();  // keep every rank's shared memory alive until rank 0 has read it
   trace_mark(a.trace, a.trace_slot, 2);
 }
 
