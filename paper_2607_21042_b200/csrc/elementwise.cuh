@@ -281,15 +281,29 @@ __global__ void __launch_bounds__(kSampleThreads) sample_kernel(const SampleArgs
         if (q < per && i < V && (ok[q] & mask) == prefix) atomicAdd(&hist[(ok[q] >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        unsigned int rem = sh_remaining, cum = 0u;
-        int bin = 255;
-        for (; bin > 0; --bin) {
-          if (cum + hist[bin] >= rem) break;
-          cum += hist[bin];
+      if (warp == 0) {
+        // find the bin (from the top) in which the running count reaches `rem`: lane L owns bins
+        // 8L..8L+7; counts above the lane come from a suffix scan over the lanes' totals
+        const unsigned int rem = sh_remaining;
+        unsigned int hb[8], tot = 0u;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) { hb[b] = hist[8 * lane + b]; tot += hb[b]; }
+        unsigned int suf = tot;   // inclusive suffix sum over lanes >= this one
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned int n = __shfl_down_sync(0xFFFFFFFFu, suf, o);
+          if (lane + o < 32) suf += n;
         }
-        sh_remaining = rem - cum;
-        sh_prefix = prefix | ((uint32_t)bin << shift);
+        unsigned int cum = suf - tot;   // entries in bins above this lane's
+        if (cum < rem && cum + tot >= rem) {   // the crossing happens inside this lane's bins
+          int bin = 7;
+          for (; bin > 0; --bin) {
+            if (cum + hb[bin] >= rem) break;
+            cum += hb[bin];
+          }
+          sh_remaining = rem - cum;
+          sh_prefix = prefix | ((uint32_t)(8 * lane + bin) << shift);
+        }
       }
       mask |= 255u << shift;
       __syncthreads();
