@@ -117,6 +117,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
     from paper_2607_21042_b200 import binding as B
+    from paper_2607_21042_b200 import replicas as R
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -211,12 +212,10 @@ def run_ours(args):
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
     launches = eng.kernel_launches() - l0
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    total_tokens = R.sum_over_ranks(tokens, device)     # replicas: every rank decodes its own copy of the workload
+    ms = R.max_over_ranks(ms, device)
     steps_done = min(K, max_dec)
-    value = world * tokens / (ms * 1e-3)
+    value = total_tokens / (ms * 1e-3)
 
     # ---- end to end: host buffers in, host buffers out, every step ----
     ids = open_all()
@@ -250,14 +249,12 @@ def run_ours(args):
             e2e_tokens += n
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_total = R.sum_over_ranks(e2e_tokens, device)
+    e2e_s = R.max_over_ranks(e2e_s, device)
     for s in ids:
         eng.release_stream(s)
     eng.sync()
-    e2e = {"value": world * e2e_tokens / e2e_s, "unit": UNIT,
+    e2e = {"value": e2e_total / e2e_s, "unit": UNIT,
            "h2d_bytes_per_step": 4 * S, "d2h_bytes_per_step": S * (4 + 4 * V + 2 * d),
            "steps": n_e2e, "note": "host sync every step: token in from pinned host memory; token, logits and hidden row back"}
 

@@ -176,13 +176,16 @@ int32_t tts_gpt_op_linear_pack(int32_t wfmt, int32_t N, int32_t K, const void *w
 int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed, const void *bias,
                           int32_t B, const void *act, float *out, void *cuda_stream);
 
-/* The same linear on the 5th-generation tensor cores (the engine's path for more than 16 rows with
- * bf16 weights): w bf16 [N,K] canonical, K a multiple of 64, 1 <= B <= 128, ksplit 1 or 4 (4: the
- * k-range partial sums are folded in range order, as the engine's next LayerNorm does).  `scratch`
- * (1024-byte aligned, >= scratch_bytes) receives the operand images. */
+/* The same linear on the 5th-generation tensor cores (the engine's path for more than 16 rows):
+ * w, s in the canonical formats above, K a multiple of 128, 1 <= B <= 128, ksplit 1 or 4 (4: the
+ * k-range partial sums are folded in range order, as the engine's next LayerNorm does).  Quantized
+ * codes enter the tensor cores as exact bf16 integers; scales multiply fp32 sums (per row for int8,
+ * per row and 128-column group for int4).  `scratch` (1024-byte aligned, >= scratch_bytes) receives
+ * the operand images. */
 int32_t tts_gpt_op_linear_tc_scratch_bytes(int32_t N, int32_t K, size_t *bytes);
-int32_t tts_gpt_op_linear_tc(int32_t N, int32_t K, const void *w, const void *bias, int32_t B, const void *act,
-                             float *out, int32_t ksplit, void *scratch, void *cuda_stream);
+int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, const void *s, const void *bias,
+                             int32_t B, const void *act, float *out, int32_t ksplit, void *scratch,
+                             void *cuda_stream);
 
 /* Bytes of scratch tts_gpt_op_attention needs for R rows of n_head heads. */
 int32_t tts_gpt_op_attention_scratch_bytes(int32_t R, int32_t n_head, size_t *bytes);

@@ -277,18 +277,20 @@ def op_linear(wfmt, packed, N, K, act, bias=None, stream=None):
     return out
 
 
-def op_linear_tc(w, act, bias=None, ksplit=1, stream=None):
-    """Tensor-core linear: w int16 (bf16 bits) [N,K] canonical, act int16 [B,K] -> fp32 [B,N]."""
-    N, K = w.shape
+def op_linear_tc(wfmt, w, s, act, bias=None, ksplit=1, stream=None):
+    """Tensor-core linear: w/s in the canonical formats, act int16 (bf16 bits) [B,K] -> fp32 [B,N]."""
+    N = w.shape[0]
+    K = w.shape[1] * (8 if wfmt == 2 else 1)
     B = act.shape[0]
     n = C.c_size_t(0)
     _check(load().tts_gpt_op_linear_tc_scratch_bytes(C.c_int32(N), C.c_int32(K), C.byref(n)))
     scratch = torch.zeros(n.value + 1024, dtype=torch.uint8, device=w.device)
     base = (scratch.data_ptr() + 1023) // 1024 * 1024
     out = torch.empty((B, N), dtype=torch.float32, device=w.device)
-    _check(load().tts_gpt_op_linear_tc(C.c_int32(N), C.c_int32(K), _ptr(w), _ptr(bias), C.c_int32(B), _ptr(act),
-                                       _ptr(out), C.c_int32(ksplit), C.c_void_p(base), _stream_ptr(stream)))
-    torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+    _check(load().tts_gpt_op_linear_tc(C.c_int32(wfmt), C.c_int32(N), C.c_int32(K), _ptr(w), _ptr(s), _ptr(bias),
+                                       C.c_int32(B), _ptr(act), _ptr(out), C.c_int32(ksplit), C.c_void_p(base),
+                                       _stream_ptr(stream)))
+    (torch.cuda.current_stream() if stream is None else stream).synchronize()
     del scratch
     return out
 

@@ -17,7 +17,7 @@
 // residual stream, 4 k-ranges, every linear of the block runs on 120-160 CTAs.  Warp 0 produces
 // (bulk copies into a 5-stage ring guarded by full/empty mbarriers; the weight copies of the first
 // stages are issued before the dependency wait), warp 1 issues the MMAs (4 per k-chunk, M=128,
-// N=32, K=16) and commits each stage back to the producer, then all 4 warps read the 128x32 fp32
+// N=32, K=16) and commits each stage back to the producer, and warps 2-5 read the 128x32 fp32
 // accumulator out of tensor memory and run the epilogue.  K-split partial sums go to a scratch
 // array that the following LayerNorm kernel folds into the residual stream in a fixed order.
 // Every wait is bounded; on expiry the CTA sets the error word, stops waiting and still releases
@@ -34,7 +34,8 @@ constexpr int kTcChunkN = 32;          // batch rows per CTA
 constexpr int kTcKChunk = 64;          // columns per pipeline stage (128 bytes of bf16)
 constexpr uint32_t kTcABytes = kTcTileM * 128;   // 16 KB
 constexpr uint32_t kTcBBytes = kTcChunkN * 128;  // 4 KB
-constexpr int kTcThreads = 128;
+constexpr int kTcThreads = 192;          // warp 0: producer, warp 1: MMA issuer, warps 2-5: epilogue
+constexpr int kTcEpiThreads = 128;
 constexpr int kTcKSplit = 4;            // k-ranges of the two linears that feed the residual stream
 constexpr unsigned long long kTcWaitNs = 2000000000ull;
 
@@ -61,6 +62,59 @@ __global__ void pack_weight_image_kernel(const uint16_t *__restrict__ w, int N, 
   uint4 v = make_uint4(0, 0, 0, 0);
   if (n < N) v = *reinterpret_cast<const uint4 *>(w + (size_t)n * K + k);
   dst[unit] = v;
+}
+
+// Quantized formats: the image holds the integer codes widened to bf16 (exact: |q| <= 127), the
+// scales multiply fp32 sums later (per row in the epilogue for int8, per row and 128-column group
+// for int4), so the tensor-core path dequantizes exactly like the register path does.
+__device__ __forceinline__ uint32_t two_ints_to_bf16x2(int lo, int hi) {
+  return pack_bf16x2((float)lo, (float)hi);
+}
+__global__ void pack_weight_image_int8_kernel(const int8_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
+  const int KC = K / 64;
+  const size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (unit >= (size_t)((N + 127) / 128) * KC * (kTcABytes / 16)) return;
+  const int within = unit % (kTcABytes / 16);
+  const size_t blk = unit / (kTcABytes / 16);
+  const int kc = blk % KC, nt = blk / KC;
+  const int r = within >> 3, u = (within & 7) ^ (r & 7);
+  const int n = nt * 128 + r, k = kc * 64 + u * 8;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (n < N) {
+    const int8_t *p = w + (size_t)n * K + k;
+    v.x = two_ints_to_bf16x2(p[0], p[1]); v.y = two_ints_to_bf16x2(p[2], p[3]);
+    v.z = two_ints_to_bf16x2(p[4], p[5]); v.w = two_ints_to_bf16x2(p[6], p[7]);
+  }
+  dst[unit] = v;
+}
+__global__ void pack_weight_image_int4_kernel(const uint32_t *__restrict__ w, int N, int K, uint4 *__restrict__ dst) {
+  const int KC = K / 64;
+  const size_t unit = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (unit >= (size_t)((N + 127) / 128) * KC * (kTcABytes / 16)) return;
+  const int within = unit % (kTcABytes / 16);
+  const size_t blk = unit / (kTcABytes / 16);
+  const int kc = blk % KC, nt = blk / KC;
+  const int r = within >> 3, u = (within & 7) ^ (r & 7);
+  const int n = nt * 128 + r, k = kc * 64 + u * 8;
+  uint4 v = make_uint4(0, 0, 0, 0);
+  if (n < N) {
+    const uint32_t word = w[(size_t)n * (K / 8) + k / 8];   // canonical: nibble j = column k + j, stored as q + 8
+    int q[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q[j] = (int)((word >> (4 * j)) & 15u) - 8;
+    v.x = two_ints_to_bf16x2(q[0], q[1]); v.y = two_ints_to_bf16x2(q[2], q[3]);
+    v.z = two_ints_to_bf16x2(q[4], q[5]); v.w = two_ints_to_bf16x2(q[6], q[7]);
+  }
+  dst[unit] = v;
+}
+
+inline cudaError_t launch_pack_image(int wf, int N, int K, const void *w, void *img, cudaStream_t st) {
+  const size_t units = weight_image_bytes(N, K) / 16;
+  const unsigned blocks = (unsigned)((units + 255) / 256);
+  if (wf == WF_BF16) pack_weight_image_kernel<<<blocks, 256, 0, st>>>((const uint16_t *)w, N, K, (uint4 *)img);
+  else if (wf == WF_INT8) pack_weight_image_int8_kernel<<<blocks, 256, 0, st>>>((const int8_t *)w, N, K, (uint4 *)img);
+  else pack_weight_image_int4_kernel<<<blocks, 256, 0, st>>>((const uint32_t *)w, N, K, (uint4 *)img);
+  return cudaGetLastError();
 }
 
 // plain bf16 [B,K] -> activation image (used by the stand-alone entry point)
@@ -129,6 +183,8 @@ struct GemmTcArgs {
   const void *w_img;        // weight image [N/128][K/64] blocks
   const void *act_img;      // activation image [K/64] blocks of 128 rows
   const uint16_t *bias;     // bf16 [N] or null
+  const uint16_t *scales;   // tiled scales of linear.cuh: int8 [N/8][8]; int4 [N/8][K/128][8]
+  int wfmt;                 // WF_* : bf16 = no scale, int8 = per row, int4 = per row and 128-column group
   int N, K, B, mode;        // mode: EPI_* of linear.cuh
   int ksplit;               // k-ranges (gridDim.z)
   float *out_f32;           // EPI_F32: out[b*out_stride+n]; EPI_QKV: q; EPI_RESID: x (ksplit == 1) or partials [ksplit][128][N]
@@ -150,6 +206,15 @@ __device__ __forceinline__ void tc_wait(uint64_t *bar, uint32_t parity, volatile
   }
 }
 
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// GROUPED (int4 weights): the MMAs of each 128-column group accumulate into one of two 32-column
+// tensor-memory buffers; while the next group runs in the other buffer, the four warps read the
+// finished group out, multiply it by the group's scale of their weight row and add it to fp32
+// registers.  Otherwise one 32-column accumulator collects the whole k-range.
+template <bool GROUPED>
 __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a) {
   extern __shared__ __align__(16) unsigned char tc_smem_raw[];
   // [stages x (A 16 KB | B 4 KB)] on a 1024-byte boundary (the swizzle pattern repeats every 1024
@@ -158,24 +223,29 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   uint64_t *full = reinterpret_cast<uint64_t *>(ring + kTcStages * (kTcABytes + kTcBBytes));
   uint64_t *empty = full + kTcStages;
   uint64_t *acc_done = empty + kTcStages;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_done + 1);
+  uint64_t *grp_done = acc_done + 1;   // [2] group buffer filled (MMA warp -> all)
+  uint64_t *grp_free = grp_done + 2;   // [2] group buffer read out (all 128 threads -> MMA warp)
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(grp_free + 2);
   volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
   uint16_t **kv_base = reinterpret_cast<uint16_t **>(tmem_slot + 4);   // [32] EPI_QKV: page slot of each batch row
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = blockIdx.x, bc = blockIdx.y, ks = blockIdx.z;
   const int KC = a.K / kTcKChunk;
-  const int per = (KC + a.ksplit - 1) / a.ksplit;
+  int per = (KC + a.ksplit - 1) / a.ksplit;
+  if (GROUPED) per = (per + 1) & ~1;   // k-ranges hold whole 128-column groups (2 k-chunks each)
   const int kc0 = ks * per, kc1 = min(KC, kc0 + per);
   const int n_it = kc1 - kc0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
     mbar_init(acc_done, 1);
+    mbar_init(grp_done, 1); mbar_init(grp_done + 1, 1);
+    mbar_init(grp_free, kTcEpiThreads); mbar_init(grp_free + 1, kTcEpiThreads);
     *failed = 0;
   }
-  if (warp == 0) tmem_alloc(tmem_slot, 32);
-  if (a.mode == EPI_QKV && threadIdx.x >= 32 && threadIdx.x < 64) {   // page slots of this chunk's batch rows
+  if (warp == 0) tmem_alloc(tmem_slot, GROUPED ? 64 : 32);
+  if (a.mode == EPI_QKV && threadIdx.x >= 64 && threadIdx.x < 96) {   // page slots of this chunk's batch rows
     const int b = bc * kTcChunkN + lane;
     uint16_t *p = nullptr;
     if (b < a.B) {
@@ -222,31 +292,65 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       for (int i = 0; i < n_it; ++i) {
         const int s = i % kTcStages;
         tc_wait(full + s, (i / kTcStages) & 1, failed, a.err);
+        const int g = i >> 1;   // group of this k-chunk inside the k-range
+        if (GROUPED && (i & 1) == 0 && g >= 2) tc_wait(grp_free + (g & 1), ((g >> 1) - 1) & 1, failed, a.err);
         tc_fence_after_sync();
         const unsigned char *sa = ring + (size_t)s * (kTcABytes + kTcBBytes);
         const uint64_t da = tc_smem_desc(sa), db = tc_smem_desc(sa + kTcABytes);
+        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * 32u : tmem_d;
 #pragma unroll
-        for (int j = 0; j < kTcKChunk / 16; ++j)   // 32 bytes further along K per step: +2 in 16-byte units
-          tc_mma(tmem_d, da + 2 * j, db + 2 * j, idesc, (i > 0 || j > 0) ? 1u : 0u);
+        for (int j = 0; j < kTcKChunk / 16; ++j) {  // 32 bytes further along K per step: +2 in 16-byte units
+          const bool fresh = GROUPED ? ((i & 1) == 0 && j == 0) : (i == 0 && j == 0);
+          tc_mma(dst, da + 2 * j, db + 2 * j, idesc, fresh ? 0u : 1u);
+        }
         tc_commit(empty + s);   // the stage may be refilled once these MMAs have read it
+        if (GROUPED && ((i & 1) == 1 || i == n_it - 1)) tc_commit(grp_done + (g & 1));
       }
-      tc_commit(acc_done);
+      if (!GROUPED) tc_commit(acc_done);
     }
   }
-  __syncwarp();   // the other lanes of warps 0 and 1 wait here for their lane 0
 
-  // ---- epilogue: warp w owns accumulator lanes 32w..32w+31 = weight rows n; columns = batch rows ----
-  tc_wait(acc_done, 0, failed, a.err);
-  tc_fence_after_sync();
-  __syncwarp();
+  // ---- epilogue (warps 2-5): a warp may touch the 32 accumulator lanes 32*(warp%4)..+31 = weight
+  //      rows n; columns = batch rows ----
+  if (warp >= 2) {
+  const int lw = warp & 3;
+  const int n = nt * kTcTileM + lw * 32 + lane;
   float v[32];
-  tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16), v);
+  if (GROUPED) {
+#pragma unroll
+    for (int c = 0; c < 32; ++c) v[c] = 0.f;
+    const int n_groups = (n_it + 1) >> 1;
+    const int KG = a.K / 128;
+    for (int g = 0; g < n_groups; ++g) {
+      // scale of this thread's weight row for the group (tiled scales: [n/8][K/128][8])
+      float sc = 0.f;
+      if (n < a.N) sc = bf16_bits_to_float(a.scales[((size_t)(n >> 3) * KG + (kc0 >> 1) + g) * 8 + (n & 7)]);
+      tc_wait(grp_done + (g & 1), (g >> 1) & 1, failed, a.err);
+      tc_fence_after_sync();
+      __syncwarp();
+      float t[32];
+      tmem_ld32(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)(g & 1) * 32u, t);
+      tc_fence_before_sync();
+      mbar_arrive(grp_free + (g & 1));   // the buffer may take the group after next
+#pragma unroll
+      for (int c = 0; c < 32; ++c) v[c] = fmaf(sc, t[c], v[c]);
+    }
+  } else {
+    tc_wait(acc_done, 0, failed, a.err);
+    tc_fence_after_sync();
+    __syncwarp();
+    tmem_ld32(tmem_d + ((uint32_t)(lw * 32) << 16), v);
+  }
   if (n_it <= 0) {   // an empty k-range contributes nothing (the accumulator was never written)
 #pragma unroll
     for (int c = 0; c < 32; ++c) v[c] = 0.f;
   }
-  const int n = nt * kTcTileM + warp * 32 + lane;
   if (n < a.N && !*failed) {
+    if (a.wfmt == WF_INT8) {   // per-row scale of the integer codes
+      const float sc = bf16_bits_to_float(a.scales[n]);
+#pragma unroll
+      for (int c = 0; c < 32; ++c) v[c] *= sc;
+    }
     const float bias = (a.bias && (a.mode != EPI_RESID || a.ksplit == 1)) ? bf16_bits_to_float(a.bias[n]) : 0.f;
 #pragma unroll
     for (int c = 0; c < kTcChunkN; ++c) {
@@ -272,9 +376,10 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       }
     }
   }
+  }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_d, 32);
+  if (warp == 0) tmem_dealloc(tmem_d, GROUPED ? 64 : 32);
 }
 
 // out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)
@@ -293,11 +398,14 @@ inline size_t gemm_tc_smem_bytes() { return (size_t)kTcStages * (kTcABytes + kTc
 inline cudaError_t launch_gemm_tc(const GemmTcArgs &a, cudaStream_t st, bool pdl) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
+    cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
+    cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
     attr_done = true;
   }
   dim3 grid((a.N + kTcTileM - 1) / kTcTileM, (a.B + kTcChunkN - 1) / kTcChunkN, a.ksplit);
-  return launch_kernel(gemm_tc_kernel, grid, dim3(kTcThreads), gemm_tc_smem_bytes(), st, pdl, a);
+  if (a.wfmt == WF_INT4)
+    return launch_kernel(gemm_tc_kernel<true>, grid, dim3(kTcThreads), gemm_tc_smem_bytes(), st, pdl, a);
+  return launch_kernel(gemm_tc_kernel<false>, grid, dim3(kTcThreads), gemm_tc_smem_bytes(), st, pdl, a);
 }
 
 }  // namespace ttsgpt

@@ -76,6 +76,7 @@ struct tts_gpt {
   bool use_graph;
   bool use_pdl;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
+  int tc_min_rows = 17; // rows from which the tensor-core path is taken (TTS_GPT_TC_MIN_ROWS overrides)
   int n_sm = 148;
   unsigned long long launches = 0;
   int *dev_err = nullptr;               // error word set by a kernel whose bounded wait expired:
@@ -134,7 +135,7 @@ struct Carver {
 
 void carve_linear(Carver &cv, PackedLinear &pl, int wf, int N, int K) {
   pl.N = N; pl.K = K;
-  pl.w_img = (wf == WF_BF16 && K % 64 == 0) ? cv.take<char>(weight_image_bytes(N, K)) : nullptr;
+  pl.w_img = (K % 128 == 0) ? cv.take<char>(weight_image_bytes(N, K)) : nullptr;
   pl.w = cv.take<char>(packed_weight_bytes(wf, N, K));
   size_t sb = packed_scale_bytes(wf, N, K);
   pl.s = sb ? cv.take<uint16_t>(sb / 2) : nullptr;
@@ -190,7 +191,7 @@ size_t carve(tts_gpt *h, void *base) {
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
   h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
-  h->have_tc = c.wfmt == WF_BF16;
+  h->have_tc = true;
   if (h->have_tc) {
     h->a_img = cv.take<char>(act_image_bytes(d));
     h->o_img = cv.take<char>(act_image_bytes(d));
@@ -210,11 +211,7 @@ int copy_bf16(tts_gpt *h, uint16_t *dst, const void *src, size_t n, const char *
 int load_linear(tts_gpt *h, PackedLinear &pl, int wf, const void *w, const void *s, const void *b, const char *what) {
   if (!w || !b || (wf != WF_BF16 && !s)) return fail(h, TTS_GPT_E_ARG, "weights: %s has a null tensor", what);
   CUDA_TRY(h, launch_pack(wf, pl.N, pl.K, w, s, pl.w, pl.s, h->stream));
-  if (pl.w_img) {
-    const size_t units = weight_image_bytes(pl.N, pl.K) / 16;
-    pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, h->stream>>>((const uint16_t *)w, pl.N, pl.K, (uint4 *)pl.w_img);
-    CUDA_TRY(h, cudaGetLastError());
-  }
+  if (pl.w_img) CUDA_TRY(h, launch_pack_image(wf, pl.N, pl.K, w, pl.w_img, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(pl.bias, b, (size_t)pl.N * 2, cudaMemcpyDeviceToDevice, h->stream));
   return TTS_GPT_OK;
 }
@@ -248,6 +245,8 @@ void trace_attach(tts_gpt *h, Args &a) {
 GemmTcArgs gemm_args(tts_gpt *h, const PackedLinear &pl, const void *act_img, int B, int mode, int ksplit) {
   GemmTcArgs a;
   memset(&a, 0, sizeof a);
+  a.wfmt = pl.s ? h->cfg.wfmt : WF_BF16;   // the LM head has no scales: bf16 in every format
+  a.scales = pl.s;
   a.w_img = pl.w_img; a.act_img = act_img; a.bias = pl.bias; a.N = pl.N; a.K = pl.K; a.B = B; a.mode = mode;
   a.ksplit = ksplit; a.err = h->dev_err;
   return a;
@@ -333,7 +332,7 @@ int run_head_tc(tts_gpt *h, int n_out) {
 }
 
 bool use_tc_path(const tts_gpt *h, int R) {
-  return h->have_tc && h->use_tc && R > 16;
+  return h->have_tc && h->use_tc && R >= h->tc_min_rows;
 }
 
 int run_layers(tts_gpt *h, int R, bool decode) {
@@ -474,11 +473,7 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   if (!w->head_w) { delete h; return fail(nullptr, TTS_GPT_E_ARG, "weights: head_w is null"); }
   {
     cudaError_t e = launch_pack(WF_BF16, h->head.N, h->head.K, w->head_w, nullptr, h->head.w, nullptr, h->stream);
-    if (e == cudaSuccess && h->head.w_img) {
-      const size_t units = weight_image_bytes(h->head.N, h->head.K) / 16;
-      pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, h->stream>>>((const uint16_t *)w->head_w, h->head.N, h->head.K, (uint4 *)h->head.w_img);
-      e = cudaGetLastError();
-    }
+    if (e == cudaSuccess && h->head.w_img) e = launch_pack_image(WF_BF16, h->head.N, h->head.K, w->head_w, h->head.w_img, h->stream);
     if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "pack head: %s", cudaGetErrorString(e)); }
     if (w->head_b) {
       TRY_(copy_bf16(h, h->head.bias, w->head_b, c.vocab, "head_b"));
@@ -541,6 +536,7 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   }
   const char *ntc = getenv("TTS_GPT_NO_TC");
   h->use_tc = !(ntc && ntc[0] == '1');
+  if (const char *mr = getenv("TTS_GPT_TC_MIN_ROWS")) { const int v = atoi(mr); if (v >= 1 && v <= kMaxRows) h->tc_min_rows = v; }
   const char *np = getenv("TTS_GPT_NO_PDL");
   h->use_pdl = !(np && np[0] == '1');
   *out = h;
@@ -802,30 +798,35 @@ int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed
 int32_t tts_gpt_op_linear_tc_scratch_bytes(int32_t N, int32_t K, size_t *bytes) {
   if (N < 1 || K < 64 || K % 64 || !bytes) return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad shape");
   *bytes = align256(weight_image_bytes(N, K)) + align256(act_image_bytes(K)) +
-           align256((size_t)kTcKSplit * kMaxRows * N * sizeof(float));
+           align256((size_t)kTcKSplit * kMaxRows * N * sizeof(float)) + align256(packed_scale_bytes(WF_INT4, N, K) + 256);
   return TTS_GPT_OK;
 }
 
-int32_t tts_gpt_op_linear_tc(int32_t N, int32_t K, const void *w, const void *bias, int32_t B, const void *act,
-                             float *out, int32_t ksplit, void *scratch, void *cuda_stream) {
+int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, const void *s, const void *bias,
+                             int32_t B, const void *act, float *out, int32_t ksplit, void *scratch, void *cuda_stream) {
   size_t bytes;
   int rc = tts_gpt_op_linear_tc_scratch_bytes(N, K, &bytes);
   if (rc) return rc;
-  if (!w || !act || !out || !scratch || B < 1 || B > kMaxRows || (uintptr_t)scratch % 1024 ||
-      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit)
+  if (wfmt < 0 || wfmt > 2 || !w || !act || !out || !scratch || B < 1 || B > kMaxRows || (uintptr_t)scratch % 1024 ||
+      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit || K % 128 || (wfmt != WF_BF16 && !s))
     return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad argument");
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char *wimg = (char *)scratch;
   char *aimg = wimg + align256(weight_image_bytes(N, K));
   float *part = (float *)(aimg + align256(act_image_bytes(K)));
-  const size_t units = weight_image_bytes(N, K) / 16;
-  pack_weight_image_kernel<<<(unsigned)((units + 255) / 256), 256, 0, st>>>((const uint16_t *)w, N, K, (uint4 *)wimg);
+  uint16_t *tiled_s = (uint16_t *)(part + (size_t)kTcKSplit * kMaxRows * N);
+  CUDA_TRY(nullptr, launch_pack_image(wfmt, N, K, w, wimg, st));
+  if (wfmt != WF_BF16) {
+    const int G = wfmt == WF_INT8 ? 1 : K / 128;
+    const size_t n = (size_t)row_tiles(N) * G * 8;
+    pack_scales_kernel<<<(int)((n + 255) / 256), 256, 0, st>>>((const uint16_t *)s, N, G, tiled_s);
+  }
   const size_t au = (size_t)B * (K / 8);
   pack_act_image_kernel<<<(unsigned)((au + 255) / 256), 256, 0, st>>>((const uint16_t *)act, B, K, (unsigned char *)aimg);
   CUDA_TRY(nullptr, cudaGetLastError());
   GemmTcArgs a;
   memset(&a, 0, sizeof a);
-  a.w_img = wimg; a.act_img = aimg; a.N = N; a.K = K; a.B = B; a.ksplit = ksplit;
+  a.w_img = wimg; a.act_img = aimg; a.N = N; a.K = K; a.B = B; a.ksplit = ksplit; a.wfmt = wfmt; a.scales = tiled_s;
   if (ksplit == 1) {
     a.mode = EPI_F32; a.bias = (const uint16_t *)bias; a.out_f32 = out; a.out_stride = N;
     CUDA_TRY(nullptr, launch_gemm_tc(a, st, false));

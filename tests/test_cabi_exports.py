@@ -58,9 +58,9 @@ def test_query_workspace_and_config_errors_need_no_gpu(lib):
     with pytest.raises(binding.TtsGptError) as e:
         binding.query_workspace(bad)
     assert e.value.code == binding.E_ARG
-    # quantized formats need less
+    # quantized formats need less: 264 MB packed + 985 MB of bf16 integer images for the tensor cores
     n4 = binding.query_workspace(cases.workload(4).cfg)
-    assert n4 < 16 * 32 * 7.9e6 + 0.4e9
+    assert n4 < 16 * 32 * 7.9e6 + 1.4e9
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):

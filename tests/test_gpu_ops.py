@@ -75,15 +75,22 @@ def test_linear_int8_extreme_codes_exact():
     assert np.array_equal(got.astype(np.float64), ref)
 
 
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
 @pytest.mark.parametrize("N,K,Bn,ksplit", [(128, 256, 32, 1), (256, 256, 17, 1), (200, 1280, 128, 1),
                                              (1280, 1280, 66, 4), (130, 5120, 100, 4), (8194, 1280, 40, 1)])
-def test_tensor_core_linear_matches_oracle(N, K, Bn, ksplit):
-    rng = np.random.default_rng(N + K + Bn)
+def test_tensor_core_linear_matches_oracle(wfmt, N, K, Bn, ksplit):
+    rng = np.random.default_rng(N + K + Bn + wfmt)
     wb = _rand_bf16(rng, (N, K), 0.02)
+    if wfmt == C.W_BF16:
+        w, s = wb, None
+    elif wfmt == C.W_INT8_PC:
+        w, s = C.quantize_int8_per_channel(wb)
+    else:
+        w, s = C.quantize_int4_group128(wb)
     bias = _rand_bf16(rng, (N,), 0.02)
     act = _rand_bf16(rng, (Bn, K), 1.0)
-    ref = O.bf16_to_f64(act) @ O.bf16_to_f64(wb).T + O.bf16_to_f64(bias)
-    out = B.op_linear_tc(bits_dev(wb), bits_dev(act), bits_dev(bias), ksplit)
+    ref = O.bf16_to_f64(act) @ O.dequant(wfmt, w, s).T + O.bf16_to_f64(bias)
+    out = B.op_linear_tc(wfmt, bits_dev(w), None if s is None else bits_dev(s), bits_dev(act), bits_dev(bias), ksplit)
     got = out.cpu().numpy().astype(np.float64)
     scale = np.abs(ref).max()
     assert np.max(np.abs(got - ref)) <= 2e-5 * scale + 1e-6
