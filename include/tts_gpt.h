@@ -148,7 +148,8 @@ int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n);
 
 /* Timeline tracing (off by default).  `trace` is a DEVICE array of 8 * n_slots uint64, or NULL to
  * switch tracing off; *n_slots (HOST, may be NULL) receives the number of traced kernels per step
- * (5 per layer: QKV, attention, O-proj, FC1, FC2; then the LM head).  While set, CTA 0 of each
+ * (an upper bound: 5 per layer — QKV, attention, O-proj, FC1, FC2 — then the LM head on the
+ * small-batch path; 7 per layer — LN1, QKV, attention, O-proj, LN2, FC1, FC2 — on the tensor-core path).  While set, CTA 0 of each
  * traced kernel stores the GPU's global nanosecond timer at entry, after its dependency wait and
  * at its end into trace[8*slot + 0..2] (3..5: inner points of the linear kernels).  Synchronises and drops captured graphs. */
 int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots);

@@ -11,6 +11,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtts_gpt.so")
+EXTRA = os.environ.get("TTS_EXTRA_NVCC", "").split()
 SOURCES = [os.path.join(CSRC, "tts_gpt.cu")]
 
 
@@ -40,7 +41,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     cmd = [nvcc_path(), "-std=c++17", "-O3", "-lineinfo", "-shared", "-Xcompiler", "-fPIC",
-           "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + SOURCES
+           "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + EXTRA + SOURCES
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

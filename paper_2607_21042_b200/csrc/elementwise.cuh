@@ -120,11 +120,15 @@ struct LnTcArgs {
   void *out_img; uint16_t *out_plain;
   const int *gather, *out_slot; const StepIO *io;
   int write_back;
+  unsigned long long *trace;  // optional timeline trace
+  int trace_slot;
 };
 __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs a) {
   __shared__ float sm[kLnThreads / 32];
+  trace_mark(a.trace, a.trace_slot, 0);
   pdl_launch_dependents();
   pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
   const int j = blockIdx.x;
   const int r = a.gather ? a.gather[j] : j;
   float *xr = a.x + (size_t)r * a.d;
@@ -181,6 +185,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
       if (hid) hid[c] = y;
     }
   }
+  trace_mark(a.trace, a.trace_slot, 2);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -13,7 +13,7 @@
 // below) write this image directly.
 //
 // A CTA owns a 128-row weight tile (the M operand), one chunk of 32 batch rows (the N operand) and
-// a contiguous range of k-chunks; with 4 batch chunks and, for the two linears that feed the
+// a contiguous range of k-chunks; with 4 batch chunks of 32 and, for the two linears that feed the
 // residual stream, 4 k-ranges, every linear of the block runs on 120-160 CTAs.  Warp 0 produces
 // (bulk copies into a 5-stage ring guarded by full/empty mbarriers; the weight copies of the first
 // stages are issued before the dependency wait), warp 1 issues the MMAs (4 per k-chunk, M=128,
@@ -28,12 +28,16 @@
 
 namespace ttsgpt {
 
+// Measured on B200 (FC1 shape, 128 rows): chunks of 32 rows with a 5-stage ring (160 CTAs, two per
+// SM) beat chunks of 64 rows with 4 or 8 stages by 6-13 us per linear although the latter re-read
+// the weights from L2 only twice: more CTAs keep more copies in flight and overlap their epilogues.
 constexpr int kTcStages = 5;            // 5 x 20 KB: two CTAs fit one SM
 constexpr int kTcTileM = 128;          // weight rows per CTA
-constexpr int kTcChunkN = 32;          // batch rows per CTA
+constexpr int kTcChunkN = 32;          // batch rows per CTA (the N operand; weights are re-read once per chunk)
 constexpr int kTcKChunk = 64;          // columns per pipeline stage (128 bytes of bf16)
 constexpr uint32_t kTcABytes = kTcTileM * 128;   // 16 KB
 constexpr uint32_t kTcBBytes = kTcChunkN * 128;  // 4 KB
+static_assert(kTcChunkN == 32, "the epilogue reads one 32-column accumulator slice per thread");
 constexpr int kTcThreads = 192;          // warp 0: producer, warp 1: MMA issuer, warps 2-5: epilogue
 constexpr int kTcEpiThreads = 128;
 constexpr int kTcKSplit = 4;            // k-ranges of the two linears that feed the residual stream
@@ -195,6 +199,8 @@ struct GemmTcArgs {
   const int *page_table, *row_stream, *row_pos;
   int pps, d, H;
   int *err;
+  unsigned long long *trace;  // optional timeline trace (see trace_mark)
+  int trace_slot;
 };
 
 // a wait that gives up for good once any wait of the CTA has expired
@@ -231,6 +237,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nt = blockIdx.x, bc = blockIdx.y, ks = blockIdx.z;
+  trace_mark(a.trace, a.trace_slot, 0);
   const int KC = a.K / kTcKChunk;
   int per = (KC + a.ksplit - 1) / a.ksplit;
   if (GROUPED) per = (per + 1) & ~1;   // k-ranges hold whole 128-column groups (2 k-chunks each)
@@ -244,16 +251,17 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     mbar_init(grp_free, kTcEpiThreads); mbar_init(grp_free + 1, kTcEpiThreads);
     *failed = 0;
   }
-  if (warp == 0) tmem_alloc(tmem_slot, GROUPED ? 64 : 32);
-  if (a.mode == EPI_QKV && threadIdx.x >= 64 && threadIdx.x < 96) {   // page slots of this chunk's batch rows
-    const int b = bc * kTcChunkN + lane;
+  if (warp == 0) tmem_alloc(tmem_slot, GROUPED ? 2 * kTcChunkN : kTcChunkN);
+  if (a.mode == EPI_QKV && threadIdx.x >= 64 && threadIdx.x < 64 + kTcChunkN) {   // page slots of this chunk's batch rows
+    const int bl = threadIdx.x - 64;
+    const int b = bc * kTcChunkN + bl;
     uint16_t *p = nullptr;
     if (b < a.B) {
       const int pos = a.row_pos[b];
       const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
       p = a.kv_layer + ((size_t)page * 2 * a.H) * kPageElems + (size_t)(pos & 63) * kHeadDim;
     }
-    kv_base[lane] = p;
+    kv_base[bl] = p;
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -272,6 +280,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   }
   pdl_launch_dependents();
   pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
   if (warp == 0) {
     // ---- producer ----
     if (lane == 0) {
@@ -284,6 +293,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
         bulk_copy_g2s(ring + (size_t)s * (kTcABytes + kTcBBytes), gA + (size_t)i * kTcABytes, kTcABytes, full + s);
         bulk_copy_g2s(ring + (size_t)s * (kTcABytes + kTcBBytes) + kTcABytes, gB + (size_t)i * (kMaxRows * 128), kTcBBytes, full + s);
       }
+      trace_mark(a.trace, a.trace_slot, 3);   // last copy issued
     }
   } else if (warp == 1) {
     // ---- MMA issuer ----
@@ -297,7 +307,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
         tc_fence_after_sync();
         const unsigned char *sa = ring + (size_t)s * (kTcABytes + kTcBBytes);
         const uint64_t da = tc_smem_desc(sa), db = tc_smem_desc(sa + kTcABytes);
-        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * 32u : tmem_d;
+        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * kTcChunkN : tmem_d;
 #pragma unroll
         for (int j = 0; j < kTcKChunk / 16; ++j) {  // 32 bytes further along K per step: +2 in 16-byte units
           const bool fresh = GROUPED ? ((i & 1) == 0 && j == 0) : (i == 0 && j == 0);
@@ -379,7 +389,8 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_d, GROUPED ? 64 : 32);
+  trace_mark(a.trace, a.trace_slot, 2);
+  if (warp == 0) tmem_dealloc(tmem_d, GROUPED ? 2 * kTcChunkN : kTcChunkN);
 }
 
 // out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)

@@ -260,6 +260,7 @@ int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int
   la.x = h->x; la.d = h->cfg.d_model; la.partials = h->partials; la.n_part = n_part; la.part_cols = h->cfg.d_model;
   la.add_bias = add_bias; la.g = g; la.b = b; la.eps = h->cfg.ln_eps; la.out_img = out_img; la.out_plain = out_plain;
   la.gather = gather; la.out_slot = out_slot; la.io = io; la.write_back = write_back;
+  trace_attach(h, la);
   CUDA_TRY(h, launch_kernel(layernorm_tc_kernel, dim3(rows), dim3(kLnThreads), 0, h->stream, h->use_pdl, la));
   h->launches += 1;
   return TTS_GPT_OK;
@@ -280,23 +281,28 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+    trace_attach(h, qa);
     CUDA_TRY(h, launch_gemm_tc(qa, st, pdl));
     AttnArgs aa;
     memset(&aa, 0, sizeof aa);
     aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
     aa.row_pos = h->rt.row_pos; aa.out = (uint16_t *)h->o_img; aa.out_image = 1;
     aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
+    trace_attach(h, aa);
     CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
     GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, kTcKSplit);
     oa.out_f32 = h->partials; oa.out_stride = d;
+    trace_attach(h, oa);
     CUDA_TRY(h, launch_gemm_tc(oa, st, pdl));
     rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, kTcKSplit, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs f1 = gemm_args(h, L.fc1, h->a_img, R, EPI_GELU, 1);
     f1.out_img = h->h_img; f1.gelu_tanh = c.gelu_tanh;
+    trace_attach(h, f1);
     CUDA_TRY(h, launch_gemm_tc(f1, st, pdl));
     GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, kTcKSplit);
     f2.out_f32 = h->partials; f2.out_stride = d;
+    trace_attach(h, f2);
     CUDA_TRY(h, launch_gemm_tc(f2, st, pdl));
     h->launches += 5;
   }
@@ -734,7 +740,7 @@ int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots) {
   h->graphs.clear();
   h->graph_nodes.clear();
   h->trace = (unsigned long long *)trace;
-  if (n_slots) *n_slots = 5 * h->cfg.n_layer + 1;
+  if (n_slots) *n_slots = 7 * h->cfg.n_layer + 2;   // upper bound: the tensor-core path traces 7 kernels per layer
   return TTS_GPT_OK;
 }
 
