@@ -50,6 +50,8 @@ struct AttnArgs {
   int trace_slot;
   int out_image;             // 1: `out` is an activation image for the tensor-core linear (see act_image_offset)
   int old_pages_final;       // 1: one row per stream (decode step), pages before a row's last are not written by this step
+  const int *row_order;      // streaming variant: grid slot z handles row row_order[z] (null: row z)
+  int *err;                  // set to 1 if a bounded wait of the streaming variant expires (may be null)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -68,31 +70,35 @@ __device__ __forceinline__ void load_page(PageLoad &pl, const uint16_t *K, const
 // (lane/8, lane%8) holds elements 8*sub..8*sub+7 of 16 tokens (bit i of vmask: slot i is a real
 // token); m and l are warp-uniform, o[e] is the lane's partial over its tokens (summed over tg at
 // the very end).  At least one slot of the warp must be valid.
+// first half: scores of NS slots (log2 units, -inf for slots without a token) and their maximum over the warp
 template <int NS>
-__device__ __forceinline__ void fold_first(PageLoad &pl, const float (&qv)[8], uint32_t vmask, float &m, float &l,
-                                           float (&o)[8]) {
-  float s[NS];
+__device__ __forceinline__ float score_slots(const uint4 (&kk)[16], const float (&qv)[8], uint32_t vmask, float (&s)[16]) {
   float pm = -INFINITY;
 #pragma unroll
   for (int i = 0; i < NS; ++i) {
-    float d = qv[0] * bf16_lo(pl.kk[i].x);
-    d = fmaf(qv[1], bf16_hi(pl.kk[i].x), d);
-    d = fmaf(qv[2], bf16_lo(pl.kk[i].y), d);
-    d = fmaf(qv[3], bf16_hi(pl.kk[i].y), d);
-    d = fmaf(qv[4], bf16_lo(pl.kk[i].z), d);
-    d = fmaf(qv[5], bf16_hi(pl.kk[i].z), d);
-    d = fmaf(qv[6], bf16_lo(pl.kk[i].w), d);
-    d = fmaf(qv[7], bf16_hi(pl.kk[i].w), d);
+    float d = qv[0] * bf16_lo(kk[i].x);
+    d = fmaf(qv[1], bf16_hi(kk[i].x), d);
+    d = fmaf(qv[2], bf16_lo(kk[i].y), d);
+    d = fmaf(qv[3], bf16_hi(kk[i].y), d);
+    d = fmaf(qv[4], bf16_lo(kk[i].z), d);
+    d = fmaf(qv[5], bf16_hi(kk[i].z), d);
+    d = fmaf(qv[6], bf16_lo(kk[i].w), d);
+    d = fmaf(qv[7], bf16_hi(kk[i].w), d);
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 1);
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 2);
     d += __shfl_xor_sync(0xFFFFFFFFu, d, 4);
-    const bool valid = (vmask >> i) & 1u;
-    s[i] = valid ? d : -INFINITY;
-    if (!valid) pl.vv[i] = make_uint4(0, 0, 0, 0);  // stale page contents may hold NaN: 0 * NaN must not reach o
+    s[i] = ((vmask >> i) & 1u) ? d : -INFINITY;
     pm = fmaxf(pm, s[i]);
   }
   pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 8));
   pm = fmaxf(pm, __shfl_xor_sync(0xFFFFFFFFu, pm, 16));
+  return pm;
+}
+
+// second half: rescale the running (m, l, o) to the new maximum and add the NS slots' weighted values
+template <int NS>
+__device__ __forceinline__ void accum_slots(uint4 (&vv)[16], const float (&s)[16], float pm, uint32_t vmask, float &m,
+                                            float &l, float (&o)[8]) {
   const float m_new = fmaxf(m, pm);           // finite: the caller only folds batches with a valid token
   const float rescale = exp2f(m - m_new);     // first batch: exp2(-inf) = 0
   float lp = 0.f;
@@ -100,21 +106,30 @@ __device__ __forceinline__ void fold_first(PageLoad &pl, const float (&qv)[8], u
   for (int e = 0; e < 8; ++e) o[e] *= rescale;
 #pragma unroll
   for (int i = 0; i < NS; ++i) {
+    if (!((vmask >> i) & 1u)) vv[i] = make_uint4(0, 0, 0, 0);  // stale page contents may hold NaN: 0 * NaN must not reach o
     const float p = exp2f(s[i] - m_new);  // masked tokens: exp2(-inf) = 0
     lp += p;
-    o[0] = fmaf(p, bf16_lo(pl.vv[i].x), o[0]);
-    o[1] = fmaf(p, bf16_hi(pl.vv[i].x), o[1]);
-    o[2] = fmaf(p, bf16_lo(pl.vv[i].y), o[2]);
-    o[3] = fmaf(p, bf16_hi(pl.vv[i].y), o[3]);
-    o[4] = fmaf(p, bf16_lo(pl.vv[i].z), o[4]);
-    o[5] = fmaf(p, bf16_hi(pl.vv[i].z), o[5]);
-    o[6] = fmaf(p, bf16_lo(pl.vv[i].w), o[6]);
-    o[7] = fmaf(p, bf16_hi(pl.vv[i].w), o[7]);
+    o[0] = fmaf(p, bf16_lo(vv[i].x), o[0]);
+    o[1] = fmaf(p, bf16_hi(vv[i].x), o[1]);
+    o[2] = fmaf(p, bf16_lo(vv[i].y), o[2]);
+    o[3] = fmaf(p, bf16_hi(vv[i].y), o[3]);
+    o[4] = fmaf(p, bf16_lo(vv[i].z), o[4]);
+    o[5] = fmaf(p, bf16_hi(vv[i].z), o[5]);
+    o[6] = fmaf(p, bf16_lo(vv[i].w), o[6]);
+    o[7] = fmaf(p, bf16_hi(vv[i].w), o[7]);
   }
   lp += __shfl_xor_sync(0xFFFFFFFFu, lp, 8);
   lp += __shfl_xor_sync(0xFFFFFFFFu, lp, 16);
   l = l * rescale + lp;
   m = m_new;
+}
+
+template <int NS>
+__device__ __forceinline__ void fold_first(PageLoad &pl, const float (&qv)[8], uint32_t vmask, float &m, float &l,
+                                           float (&o)[8]) {
+  float s[16];
+  const float pm = score_slots<NS>(pl.kk, qv, vmask, s);
+  accum_slots<NS>(pl.vv, s, pm, vmask, m, l, o);
 }
 
 // ng (warp-uniform): how many groups of 4 slots hold tokens at all; they are always the first ones,
@@ -386,6 +401,136 @@ inline cudaError_t launch_attention(const AttnArgs &a, int R, int cluster, cudaS
   cfg.attrs = at;
   cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, attention_kernel, a);
+}
+
+// ------------------------------------------------------------------------------------------
+// streaming variant (the engine's path once there are enough (row, head) pairs to fill the GPU
+// several times): one CTA per (row, head), warp w takes pages w, w+4, ...  A page's K and V blocks
+// (8 KB each, contiguous in the pool) come in by two bulk asynchronous copies into the warp's own
+// 16 KB stage of shared memory; as soon as the warp has pulled the stage into registers, lane 0
+// requests the warp's next page into the same stage, so that the copy runs under the arithmetic
+// of the current page and every resident warp keeps 16 KB in flight with no registers tied up by
+// outstanding loads.  Only the tokens that exist are copied from a partial last page.
+// ------------------------------------------------------------------------------------------
+constexpr uint32_t kAttnHalfStage = kPageElems * 2;          // one K or V block: 8 KB
+constexpr uint32_t kAttnStageBytes = 2 * kAttnHalfStage;
+constexpr unsigned long long kAttnWaitNs = 2000000000ull;
+
+__device__ __forceinline__ void stream_issue(const AttnArgs &a, const int *pt, int h, int page, int n_tok,
+                                             unsigned char *stage, uint64_t *bar) {
+  const int n_here = min(kPageTokens, n_tok - page * kPageTokens);
+  const uint32_t bytes = (uint32_t)n_here * kHeadDim * 2;
+  const int phys = pt[page];
+  const uint16_t *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
+  const uint16_t *V = a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems;
+  mbar_expect_tx(bar, 2 * bytes);
+  bulk_copy_g2s(stage, K, bytes, bar);
+  bulk_copy_g2s(stage + kAttnHalfStage, V, bytes, bar);
+}
+
+__global__ void __launch_bounds__(kAttnWarps * 32, 3) attention_stream_kernel(const AttnArgs a) {
+  extern __shared__ __align__(128) unsigned char attn_stages[];   // [warp][K 8 KB | V 8 KB]
+  __shared__ __align__(8) uint64_t bars[kAttnWarps];
+  __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
+  const int h = blockIdx.y, r = a.row_order ? a.row_order[blockIdx.z] : blockIdx.z;
+  trace_mark(a.trace, a.trace_slot, 0);
+  const int n_tok = a.row_pos[r] + 1;   // row and page tables are final before the step's first kernel starts
+  const int n_pages = (n_tok + kPageTokens - 1) / kPageTokens;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tg = lane >> 3, sub = lane & 7;
+  const int *pt = a.page_table + (size_t)a.row_stream[r] * a.pps;
+  unsigned char *stage = attn_stages + (size_t)warp * kAttnStageBytes;
+  uint64_t *bar = bars + warp;
+
+  float m = -INFINITY, l = 0.f;
+  float o[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) o[e] = 0.f;
+  float qv[8];
+  const int tn = (n_tok - 1) & (kPageTokens - 1);   // the new token's slot in the last page
+  int page = warp;
+  // In a decode step only the new token's own K/V rows are written by the kernel in front, so the
+  // warp's first page is requested ahead of the dependency wait and those two rows are read again
+  // afterwards if the page holds them.
+  const bool early = a.old_pages_final && page < n_pages;
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    if (early) stream_issue(a, pt, h, page, n_tok, stage, bar);
+  }
+  __syncwarp();
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+  load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+  if (!early && page < n_pages && lane == 0) stream_issue(a, pt, h, page, n_tok, stage, bar);
+  uint32_t phase = 0;
+  bool first = true;
+  for (; page < n_pages; page += kAttnWarps) {
+    if (!mbar_wait_bounded(bar, phase, kAttnWaitNs)) {
+      if (a.err) atomicExch(a.err, 1);
+      mbar_wait_bounded(bar, phase, kAttnWaitNs);   // a last chance for the copy in flight towards this CTA
+      break;
+    }
+    phase ^= 1u;
+    const int n_here = min(kPageTokens, n_tok - page * kPageTokens);
+    uint32_t vmask = 0u;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) vmask |= (tg + 4 * i < n_here) ? (1u << i) : 0u;
+    // the new token's rows, if this page was copied before the kernel in front had written them
+    const bool patch = first && early && page == n_pages - 1 && (tn & 3) == tg;
+    const int sel = tn >> 2;
+    uint4 kn = make_uint4(0, 0, 0, 0), vn = kn;
+    if (patch) {
+      const int phys = pt[page];
+      kn = ld_cg_u4(a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems + (size_t)tn * kHeadDim + 8 * sub);
+      vn = ld_cg_u4(a.kv_layer + (((size_t)phys * 2 + 1) * a.H + h) * kPageElems + (size_t)tn * kHeadDim + 8 * sub);
+    }
+    first = false;
+    uint4 kk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      kk[i] = *reinterpret_cast<const uint4 *>(stage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
+      if (patch && i == sel) kk[i] = kn;
+    }
+    float s[16];
+    const float pm = score_slots<16>(kk, qv, vmask, s);
+    uint4 vv[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      vv[i] = *reinterpret_cast<const uint4 *>(stage + kAttnHalfStage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
+      if (patch && i == sel) vv[i] = vn;
+    }
+    __syncwarp();   // every lane has read the stage
+    if (page + kAttnWarps < n_pages && lane == 0) {
+      fence_proxy_async_smem();
+      stream_issue(a, pt, h, page + kAttnWarps, n_tok, stage, bar);
+    }
+    accum_slots<16>(vv, s, pm, vmask, m, l, o);
+  }
+  trace_mark(a.trace, a.trace_slot, 3);
+  const int e = threadIdx.x;
+  float M, L, O;
+  cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
+  if (e < kHeadDim) {
+    uint16_t *out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
+                                : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
+    *out = float_to_bf16_bits(O / L);
+  }
+  trace_mark(a.trace, a.trace_slot, 2);
+}
+
+// (row, head) pairs from which the streaming variant is used: the GPU is then covered four times
+// over with one CTA per pair (at 16 rows of 20 heads the cluster variant still measured faster)
+inline bool attention_use_stream(int R, int H, int n_sm) { return R * H >= 4 * n_sm; }
+
+inline cudaError_t launch_attention_stream(const AttnArgs &a, int R, cudaStream_t st, bool pdl) {
+  static bool attr_done = false;
+  const size_t smem = (size_t)kAttnWarps * kAttnStageBytes;
+  if (!attr_done) {
+    cudaFuncSetAttribute(attention_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    attr_done = true;
+  }
+  return launch_kernel(attention_stream_kernel, dim3(1, a.H, R), dim3(kAttnWarps * 32), smem, st, pdl, a);
 }
 
 // ------------------------------------------------------------------------------------------

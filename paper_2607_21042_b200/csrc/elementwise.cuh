@@ -26,6 +26,7 @@ struct RowTable {
   const uint16_t **row_emb;   // bf16 [d] embedding of a prefix row
   int *out_rows;              // rows whose logits are wanted, compacted
   int *out_slot;              // position of that row's results in the caller's output arrays
+  int *row_order;             // decode steps: rows by descending context length (longest first)
 };
 
 // x[r,:] = tok_emb[token] + pos_emb[posidx]   (generated tokens take a positional embedding from

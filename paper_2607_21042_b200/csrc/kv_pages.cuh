@@ -74,7 +74,15 @@ __global__ void __launch_bounds__(kMaxRows) step_setup_kernel(const StepParams p
     ps.ctx_len[s] = t + 1;
     ps.pos_next[s] += 1;
   }
+  // attention works through the rows longest first, so that the short ones fill the tail of its grid
+  __shared__ int len_s[kMaxRows];
+  len_s[i] = i < p.n ? t : -1;
   __syncthreads();
+  if (i < p.n) {
+    int before = 0;
+    for (int j = 0; j < p.n; ++j) before += (len_s[j] > t || (len_s[j] == t && j < i)) ? 1 : 0;
+    rt.row_order[before] = i;
+  }
   if (i == 0) { *ps.free_top = top - total; *io = p.io; }
 }
 

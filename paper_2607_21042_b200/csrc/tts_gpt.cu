@@ -76,6 +76,7 @@ struct tts_gpt {
   bool use_graph;
   bool use_pdl;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
+  bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
   int tc_min_rows = 17; // rows from which the tensor-core path is taken (TTS_GPT_TC_MIN_ROWS overrides)
   int n_sm = 148;
   unsigned long long launches = 0;
@@ -181,6 +182,7 @@ size_t carve(tts_gpt *h, void *base) {
   rt.row_emb = cv.take<const uint16_t *>(kMaxRows);
   rt.out_rows = cv.take<int>(kMaxRows);
   rt.out_slot = cv.take<int>(kMaxRows);
+  rt.row_order = cv.take<int>(kMaxRows);
   h->io = cv.take<StepIO>(1);
   h->x = cv.take<float>((size_t)kMaxRows * d);
   h->q = cv.take<float>((size_t)kMaxRows * d);
@@ -238,6 +240,15 @@ void trace_attach(tts_gpt *h, Args &a) {
   a.trace_slot = h->trace ? h->trace_next++ : 0;
 }
 
+// Attention for R rows: clusters while (row, head) pairs are scarce, one streaming CTA per pair
+// once they cover the GPU several times.
+cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool pdl) {
+  aa.err = h->dev_err;
+  aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
+  if (h->use_attn_stream && attention_use_stream(R, aa.H, h->n_sm)) return launch_attention_stream(aa, R, st, pdl);
+  return launch_attention(aa, R, attention_cluster_size(R, aa.H, h->n_sm), st, pdl);
+}
+
 // The transformer blocks for R rows already described by the row table, x holding the input rows.
 // Every kernel after the first of a step is launched with programmatic dependent launch, so its
 // weight loads overlap the tail of its predecessor.
@@ -289,7 +300,7 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     aa.row_pos = h->rt.row_pos; aa.out = (uint16_t *)h->o_img; aa.out_image = 1;
     aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
     trace_attach(h, aa);
-    CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
+    CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, kTcKSplit);
     oa.out_f32 = h->partials; oa.out_stride = d;
     trace_attach(h, oa);
@@ -366,11 +377,12 @@ int run_layers(tts_gpt *h, int R, bool decode) {
     trace_attach(h, qa);
     CUDA_TRY(h, launch_linear(c.wfmt, qa, st, pdl, 2 * h->n_sm));
     AttnArgs aa;
+    memset(&aa, 0, sizeof aa);
     aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
     aa.row_pos = h->rt.row_pos; aa.out = h->o; aa.partials = h->attn_partials; aa.tickets = h->attn_tickets;
     aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
     trace_attach(h, aa);
-    CUDA_TRY(h, launch_attention(aa, R, attention_cluster_size(R, c.n_head, h->n_sm), st, pdl));
+    CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     LinearArgs oa = linear_args(h, L.o, h->o, R, EPI_RESID);
     oa.out_f32 = h->x; oa.out_stride = d;
     trace_attach(h, oa);
@@ -542,6 +554,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   }
   const char *ntc = getenv("TTS_GPT_NO_TC");
   h->use_tc = !(ntc && ntc[0] == '1');
+  const char *nas = getenv("TTS_GPT_NO_ATTN_STREAM");
+  h->use_attn_stream = !(nas && nas[0] == '1');
   if (const char *mr = getenv("TTS_GPT_TC_MIN_ROWS")) { const int v = atoi(mr); if (v >= 1 && v <= kMaxRows) h->tc_min_rows = v; }
   const char *np = getenv("TTS_GPT_NO_PDL");
   h->use_pdl = !(np && np[0] == '1');
@@ -931,12 +945,16 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
-  if (cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
-    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be 1, 2, 4 or 8");
+  if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be 0, 1, 2, 4 or 8");
   AttnArgs a;
   memset(&a, 0, sizeof a);
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
   a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
+  if (cluster_size == 0) {
+    CUDA_TRY(nullptr, launch_attention_stream(a, R, (cudaStream_t)cuda_stream, false));
+    return TTS_GPT_OK;
+  }
   CUDA_TRY(nullptr, launch_attention(a, R, cluster_size, (cudaStream_t)cuda_stream, false));
   return TTS_GPT_OK;
 }

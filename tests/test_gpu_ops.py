@@ -151,7 +151,7 @@ def test_attention_matches_oracle(H, ctxs):
             assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (r, rep)
 
 
-@pytest.mark.parametrize("S", [1, 2, 4, 8])
+@pytest.mark.parametrize("S", [0, 1, 2, 4, 8])      # 0: the streaming variant
 def test_attention_cluster_variant_matches_oracle(S):
     rng = np.random.default_rng(40 + S)
     H = 5
@@ -181,6 +181,22 @@ def test_attention_rows_of_one_stream_share_pages():
                          torch.zeros(R, dtype=torch.int32, device=DEV), torch.from_numpy(pos).to(DEV))
     got = bits_to_f64(out)
     for r in range(R):
+        ref = _attention_ref(q[r].astype(np.float64), Ks[0][:pos[r] + 1], Vs[0][:pos[r] + 1], H)
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5
+
+
+def test_attention_streaming_variant_rows_of_one_stream():
+    # the streaming variant on a prefill-like pass: many rows of one stream, every page boundary
+    rng = np.random.default_rng(78)
+    H, n = 3, 330
+    kv, pt, Ks, Vs = _attention_case(rng, H, [n], 8, 32)
+    pos = np.arange(n, dtype=np.int32)
+    q = rng.standard_normal(size=(n, H * 64)).astype(np.float32)
+    out = B.op_attention_cluster(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                                 torch.zeros(n, dtype=torch.int32, device=DEV), torch.from_numpy(pos).to(DEV), 0)
+    torch.cuda.synchronize()
+    got = bits_to_f64(out)
+    for r in range(0, n, 7):
         ref = _attention_ref(q[r].astype(np.float64), Ks[0][:pos[r] + 1], Vs[0][:pos[r] + 1], H)
         assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5
 
