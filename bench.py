@@ -282,7 +282,7 @@ def run_ours(args):
                    "parallelism": "replicas x%d" % world if world > 1 else "single GPU",
                    "l2": "inputs larger than L2: %.0f MB of weights + KV stream per step" % (nbytes / max(steps_done, 1) / 1e6)},
         "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks,
-        "tokens": tokens,
+        "tokens": tokens, "launches_before_timed_region": int(l0),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, budget_steps=args.cpu_steps)

@@ -63,8 +63,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ void trace_mark(unsigned long long *trace, int slot, int which) {
-  if (trace && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+__device__ __forceinline__ void trace_mark(unsigned long long *trace, int slot, int which, int tid = 0) {
+  if (trace && threadIdx.x == tid && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
     trace[8 * slot + which] = global_timer_ns();
 }
 
