@@ -374,9 +374,9 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
 }
 
 // Cluster size for R rows of H heads on n_sm SMs: enough CTAs to cover the GPU about once.
-inline int attention_cluster_size(int R, int H, int n_sm) {
+inline int attention_cluster_size(int R, int H, int n_sm, int fill = 1) {
   int s = 1;
-  while (s < kAttnMaxCluster && R * H * s < n_sm) s *= 2;
+  while (s < kAttnMaxCluster && R * H * s < fill * n_sm) s *= 2;
   return s;
 }
 

@@ -68,6 +68,14 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_kernel(const float *__re
                                                                uint16_t *__restrict__ out, const int *gather,
                                                                const int *out_slot, const StepIO *io) {
   __shared__ float sm[kLnThreads / 32];
+  // gamma and beta do not depend on the kernel in front: fetched ahead of the dependency wait
+  float gg[kLnMaxPerThread], bb[kLnMaxPerThread];
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    gg[i] = c < d ? bf16_bits_to_float(g[c]) : 0.f;
+    bb[i] = c < d ? bf16_bits_to_float(b[c]) : 0.f;
+  }
   pdl_launch_dependents();
   pdl_wait();
   const int j = blockIdx.x;
@@ -95,7 +103,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_kernel(const float *__re
   for (int i = 0; i < kLnMaxPerThread; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     if (c < d) {
-      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * bf16_bits_to_float(g[c]) + bf16_bits_to_float(b[c]));
+      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * gg[i] + bb[i]);
       out[(size_t)j * d + c] = y;
       if (hid) hid[c] = y;
     }
@@ -127,6 +135,15 @@ struct LnTcArgs {
 __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs a) {
   __shared__ float sm[kLnThreads / 32];
   trace_mark(a.trace, a.trace_slot, 0);
+  // gamma, beta and the folded bias do not depend on the kernel in front: fetched ahead of the dependency wait
+  float gg[kLnMaxPerThread], bb[kLnMaxPerThread], bs[kLnMaxPerThread];
+#pragma unroll
+  for (int i = 0; i < kLnMaxPerThread; ++i) {
+    const int c = threadIdx.x + i * kLnThreads;
+    gg[i] = c < a.d ? bf16_bits_to_float(a.g[c]) : 0.f;
+    bb[i] = c < a.d ? bf16_bits_to_float(a.b[c]) : 0.f;
+    bs[i] = (c < a.d && a.n_part > 0 && a.add_bias) ? bf16_bits_to_float(a.add_bias[c]) : 0.f;
+  }
   pdl_launch_dependents();
   pdl_wait();
   trace_mark(a.trace, a.trace_slot, 1);
@@ -136,17 +153,16 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   // all loads of the row (x, bias and up to 4 partial sums per element) are issued before any is
   // used; the sum itself is taken in a fixed order
   constexpr int kMaxPart = 4;
-  float v[kLnMaxPerThread], bs[kLnMaxPerThread], pp[kLnMaxPerThread][kMaxPart];
+  float v[kLnMaxPerThread], pp[kLnMaxPerThread][kMaxPart];
 #pragma unroll
   for (int i = 0; i < kLnMaxPerThread; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
-    v[i] = 0.f; bs[i] = 0.f;
+    v[i] = 0.f;
 #pragma unroll
     for (int p = 0; p < kMaxPart; ++p) pp[i][p] = 0.f;
     if (c < a.d) {
       v[i] = xr[c];
       if (a.n_part > 0) {
-        if (a.add_bias) bs[i] = bf16_bits_to_float(a.add_bias[c]);
 #pragma unroll
         for (int p = 0; p < kMaxPart; ++p)
           if (p < a.n_part) pp[i][p] = __ldcg(a.partials + ((size_t)p * kMaxRows + r) * a.part_cols + c);
@@ -180,7 +196,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   for (int i = 0; i < kLnMaxPerThread; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     if (c < a.d) {
-      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * bf16_bits_to_float(a.g[c]) + bf16_bits_to_float(a.b[c]));
+      const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * gg[i] + bb[i]);
       if (a.out_img) *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset(j, c)) = y;
       if (a.out_plain) a.out_plain[(size_t)j * a.d + c] = y;
       if (hid) hid[c] = y;

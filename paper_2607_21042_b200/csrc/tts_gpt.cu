@@ -77,6 +77,7 @@ struct tts_gpt {
   bool use_pdl;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
   bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
+  int attn_cluster_fill = 1;     // clusters grow until the grid covers the GPU this many times (TTS_GPT_ATTN_CLUSTER_FILL)
   int attn_stream_min_pairs = 0; // (row, head) pairs from which it is used; 0: attention_use_stream decides (TTS_GPT_ATTN_STREAM_MIN)
   int tc_min_rows = 17; // rows from which the tensor-core path is taken (TTS_GPT_TC_MIN_ROWS overrides)
   int n_sm = 148;
@@ -248,7 +249,7 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
   aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
   const bool stream = h->attn_stream_min_pairs > 0 ? R * aa.H >= h->attn_stream_min_pairs : attention_use_stream(R, aa.H, h->n_sm);
   if (h->use_attn_stream && stream) return launch_attention_stream(aa, R, st, pdl);
-  return launch_attention(aa, R, attention_cluster_size(R, aa.H, h->n_sm), st, pdl);
+  return launch_attention(aa, R, attention_cluster_size(R, aa.H, h->n_sm, h->attn_cluster_fill), st, pdl);
 }
 
 // The transformer blocks for R rows already described by the row table, x holding the input rows.
@@ -558,6 +559,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   h->use_tc = !(ntc && ntc[0] == '1');
   const char *nas = getenv("TTS_GPT_NO_ATTN_STREAM");
   h->use_attn_stream = !(nas && nas[0] == '1');
+  const char *acf = getenv("TTS_GPT_ATTN_CLUSTER_FILL");
+  if (acf && atoi(acf) > 0) h->attn_cluster_fill = atoi(acf);
   const char *asm_ = getenv("TTS_GPT_ATTN_STREAM_MIN");
   if (asm_ && atoi(asm_) > 0) h->attn_stream_min_pairs = atoi(asm_);
   if (const char *mr = getenv("TTS_GPT_TC_MIN_ROWS")) { const int v = atoi(mr); if (v >= 1 && v <= kMaxRows) h->tc_min_rows = v; }
