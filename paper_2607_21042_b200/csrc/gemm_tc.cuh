@@ -278,6 +278,15 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       bulk_copy_g2s(ring + (size_t)i * (kTcABytes + kTcBBytes), gA + (size_t)i * kTcABytes, kTcABytes, full + i);
     }
   }
+  // per-row epilogue constants do not depend on the kernel in front either
+  float e_rsc = 1.f, e_bias = 0.f;
+  if (warp >= 2) {
+    const int n = nt * kTcTileM + (warp & 3) * 32 + lane;
+    if (n < a.N) {
+      if (a.wfmt == WF_INT8) e_rsc = bf16_bits_to_float(a.scales[n]);   // per-row scale of the integer codes
+      if (a.bias && (a.mode != EPI_RESID || a.ksplit == 1)) e_bias = bf16_bits_to_float(a.bias[n]);
+    }
+  }
   pdl_launch_dependents();
   pdl_wait();
   trace_mark(a.trace, a.trace_slot, 1);
@@ -356,12 +365,11 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     for (int c = 0; c < 32; ++c) v[c] = 0.f;
   }
   if (n < a.N && !*failed) {
-    if (a.wfmt == WF_INT8) {   // per-row scale of the integer codes
-      const float sc = bf16_bits_to_float(a.scales[n]);
+    if (a.wfmt == WF_INT8) {
 #pragma unroll
-      for (int c = 0; c < 32; ++c) v[c] *= sc;
+      for (int c = 0; c < 32; ++c) v[c] *= e_rsc;
     }
-    const float bias = (a.bias && (a.mode != EPI_RESID || a.ksplit == 1)) ? bf16_bits_to_float(a.bias[n]) : 0.f;
+    const float bias = e_bias;
 #pragma unroll
     for (int c = 0; c < kTcChunkN; ++c) {
       const int b = bc * kTcChunkN + c;

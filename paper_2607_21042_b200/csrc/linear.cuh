@@ -31,6 +31,7 @@ enum { EPI_F32 = 0, EPI_QKV = 1, EPI_RESID = 2, EPI_GELU = 3 };
 
 constexpr int kLinearWarps = 10;  // divides the k-tile counts of K=1280 and K=5120 in every format
 constexpr int kLinearThreads = kLinearWarps * 32;
+constexpr int kSmallKSplit = 4;     // k-ranges of FC2 between 5 and 16 rows (partial sums folded by the next LayerNorm)
 constexpr int kLnFuseMaxRows = 4;   // LayerNorm is fused into the linear up to this batch: every CTA repeats
                                     // it, which beats a separate launch only while the rows are few
 
@@ -144,6 +145,8 @@ struct LinearArgs {
   unsigned long long *trace;  // optional timeline trace (see trace_mark)
   int trace_slot;
   int *err;                   // optional device error word: set to 1 if the weight copy never arrives
+  int ksplit;                 // 0 or 1: whole K per CTA; n > 1 (EPI_RESID only, no fused LN): gridDim.y = n k-ranges,
+                              // out_f32 = partial sums [n][kMaxRows][N] without bias, folded by the next LayerNorm
 };
 
 // exact int8 (biased byte) -> float via the 2^23 magic number
@@ -185,7 +188,9 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
   constexpr int C = 8 * RT;    // output columns (weight rows) of this CTA
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int KB = a.K / KT;
+  const int KBG = a.K / KT;                          // k-tiles of the whole matrix
+  const int KB = KBG / (int)gridDim.y;               // k-tiles of this CTA's k-range
+  const int kb_off = (int)blockIdx.y * KB;           // its first k-tile
   const int tile0 = blockIdx.x * RT, n_rt = row_tiles(a.N);
   trace_mark(a.trace, a.trace_slot, 0);
 
@@ -205,10 +210,20 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
     const uint32_t sbytes = WF == WF_INT4 ? (uint32_t)n_valid * KB * 16u : 0u;
     mbar_init(wbar, 1);
     mbar_expect_tx(wbar, wbytes + sbytes);
-    const unsigned char *gw = reinterpret_cast<const unsigned char *>(a.w) + (size_t)tile0 * KB * 512;
-    for (uint32_t off = 0; off < wbytes; off += 32768u)
-      bulk_copy_g2s(wsm + off, gw + off, min(32768u, wbytes - off), wbar);
-    if (sbytes) bulk_copy_g2s(ssm, a.scales + (size_t)tile0 * KB * 8, sbytes, wbar);
+    if (gridDim.y == 1) {   // all of K: the CTA's tiles are one contiguous range
+      const unsigned char *gw = reinterpret_cast<const unsigned char *>(a.w) + (size_t)tile0 * KB * 512;
+      for (uint32_t off = 0; off < wbytes; off += 32768u)
+        bulk_copy_g2s(wsm + off, gw + off, min(32768u, wbytes - off), wbar);
+      if (sbytes) bulk_copy_g2s(ssm, a.scales + (size_t)tile0 * KB * 8, sbytes, wbar);
+    } else {                // a k-range: one contiguous piece per row tile
+      for (int j = 0; j < n_valid; ++j) {
+        const unsigned char *gw = reinterpret_cast<const unsigned char *>(a.w) + ((size_t)(tile0 + j) * KBG + kb_off) * 512;
+        const uint32_t tb = (uint32_t)KB * 512u;
+        for (uint32_t off = 0; off < tb; off += 32768u)
+          bulk_copy_g2s(wsm + (size_t)j * tb + off, gw + off, min(32768u, tb - off), wbar);
+        if (sbytes) bulk_copy_g2s(ssm + (size_t)j * KB * 8, a.scales + ((size_t)(tile0 + j) * KBG + kb_off) * 8, (uint32_t)KB * 16u, wbar);
+      }
+    }
   }
 
   // ---- everything else that no kernel of the step writes: LN gamma/beta, bias, scales, KV slots ----
@@ -251,7 +266,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
   //      squares of its 4 values; (mean, M2) pairs of equal weight are then merged pairwise
   //      (mean = (ma+mb)/2, M2 = M2a + M2b + (mb-ma)^2 * n/2), first by shuffles, then across the
   //      warps through shared memory: one block barrier, no cancellation.
-  const int stride = ln_stage_stride(WF, a.K);
+  const int stride = ln_stage_stride(WF, KB * KT);   // staged columns: this CTA's k-range
   constexpr int RPR = 4;  // rows per LayerNorm round
   if (LN) {
     float2 *lnred = reinterpret_cast<float2 *>(red);  // [warps][RPR] (mean, M2), reused later for the partial sums
@@ -324,11 +339,12 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       __syncthreads();
     }
   } else if (MODE == ACT_STAGED) {
-    const int k8 = a.K >> 3;
+    const int k8 = (KB * KT) >> 3;
+    const uint16_t *src = a.act + (size_t)kb_off * KT;
     for (int idx = threadIdx.x; idx < a.B * k8; idx += kLinearThreads) {
       const int b = idx / k8, c8 = idx - b * k8;
       *reinterpret_cast<uint4 *>(stage + (size_t)b * stride + 8 * c8) =
-          *reinterpret_cast<const uint4 *>(a.act + (size_t)b * a.K + 8 * c8);
+          *reinterpret_cast<const uint4 *>(src + (size_t)b * a.K + 8 * c8);
     }
     __syncthreads();
   } else {
@@ -354,7 +370,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       e_old[e] = 0.f;
       const int o = threadIdx.x + e * kLinearThreads;
       const int b = m0 + o / C;
-      if (a.mode == EPI_RESID && o < 16 * C && b < a.B && en < a.N) e_old[e] = a.out_f32[(size_t)b * a.out_stride + en];
+      if (a.mode == EPI_RESID && gridDim.y == 1 && o < 16 * C && b < a.B && en < a.N) e_old[e] = a.out_f32[(size_t)b * a.out_stride + en];
     }
     if (NB > 0) {
       // ---- CUDA-core path: lane (g,t) multiplies its 16 bytes of weight row g with the matching
@@ -445,8 +461,8 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
 #pragma unroll
       for (int j = 0; j < RT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
       const int r0 = m0 + g, r1 = m0 + g + 8;
-      const uint16_t *row0 = STAGED ? stage + (size_t)r0 * stride : a.act + (size_t)r0 * a.K;
-      const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K;
+      const uint16_t *row0 = STAGED ? stage + (size_t)r0 * stride : a.act + (size_t)r0 * a.K + (size_t)kb_off * KT;
+      const uint16_t *row1 = STAGED ? stage + (size_t)r1 * stride : a.act + (size_t)r1 * a.K + (size_t)kb_off * KT;
       const bool v0 = r0 < a.B, v1 = r1 < a.B;
       // activation fragments: G k-tiles are fetched together so that their latencies overlap
       constexpr int G = STAGED ? 1 : 8 / AW;   // up to 64 registers of activation fragments in flight
@@ -531,6 +547,10 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
 #pragma unroll
         for (int w = 0; w < kLinearWarps; ++w) v += red[((size_t)w * 16 + bl) * C + ecol];
         if (WF == WF_INT8) v *= e_scale;
+        if (gridDim.y > 1) {   // partial sum of this k-range; bias and residual are added by the folding LayerNorm
+          a.out_f32[((size_t)blockIdx.y * kMaxRows + b) * a.N + n] = v;
+          continue;
+        }
         v += e_bias;
         if (a.mode == EPI_F32) {
           a.out_f32[(size_t)b * a.out_stride + n] = v;
@@ -573,7 +593,7 @@ inline size_t linear_smem_bytes(int wf, int rt, int mode, int B, int K) {
 // byte of the layer is requested before the kernel waits for its predecessor; a CTA's weights and
 // activation rows must fit its share of shared memory.
 struct LinearPlan { int rt, grid; };
-inline LinearPlan plan_linear(int wf, int N, int K, int B, int mode, int max_ctas) {
+inline LinearPlan plan_linear(int wf, int N, int K, int B, int mode, int max_ctas) {   // K, max_ctas: per k-range
   const int tiles = row_tiles(N);
   LinearPlan p;
   p.rt = 1;
@@ -586,13 +606,14 @@ inline LinearPlan plan_linear(int wf, int N, int K, int B, int mode, int max_cta
 
 template <int WF, int RT, int MODE, int NB>
 inline cudaError_t launch_linear_nb(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
-  const size_t smem = linear_smem_bytes(WF, RT, MODE, a.B, a.K);
+  const int ks = a.ksplit > 1 ? a.ksplit : 1;
+  const size_t smem = linear_smem_bytes(WF, RT, MODE, a.B, a.K / ks);
   static bool attr_done = false;  // opt-in to more than 48 KB of dynamic shared memory, once
   if (!attr_done) {
     cudaFuncSetAttribute(linear_kernel<WF, RT, MODE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     attr_done = true;
   }
-  return launch_kernel(linear_kernel<WF, RT, MODE, NB>, dim3(grid), dim3(kLinearThreads), smem, st, pdl, a);
+  return launch_kernel(linear_kernel<WF, RT, MODE, NB>, dim3(grid, ks), dim3(kLinearThreads), smem, st, pdl, a);
 }
 
 template <int WF, int RT, int MODE>
@@ -606,8 +627,9 @@ inline cudaError_t launch_linear_inst(const LinearArgs &a, int grid, cudaStream_
 
 template <int WF, int MODE>
 inline cudaError_t launch_linear_wf(const LinearArgs &a, int max_ctas, cudaStream_t st, bool pdl) {
-  const LinearPlan p = plan_linear(WF, a.N, a.K, a.B, MODE, max_ctas);
-  if (linear_smem_bytes(WF, p.rt, MODE, a.B, a.K) > 200 * 1024) return cudaErrorInvalidValue;
+  const int ks = a.ksplit > 1 ? a.ksplit : 1;
+  const LinearPlan p = plan_linear(WF, a.N, a.K / ks, a.B, MODE, max_ctas / ks);
+  if (linear_smem_bytes(WF, p.rt, MODE, a.B, a.K / ks) > 200 * 1024) return cudaErrorInvalidValue;
   if (p.rt == 1) return launch_linear_inst<WF, 1, MODE>(a, p.grid, st, pdl);
   if (p.rt == 2) return launch_linear_inst<WF, 2, MODE>(a, p.grid, st, pdl);
   return launch_linear_inst<WF, 4, MODE>(a, p.grid, st, pdl);
@@ -622,7 +644,7 @@ inline bool can_fuse_ln(int wf, int B, int K) {
 template <int WF>
 inline cudaError_t launch_linear_mode(const LinearArgs &a, int max_ctas, cudaStream_t st, bool pdl) {
   if (a.ln_x) return launch_linear_wf<WF, ACT_LN>(a, max_ctas, st, pdl);
-  if ((size_t)a.B * ln_stage_stride(WF, a.K) * sizeof(uint16_t) <= (size_t)kStageMaxBytes)
+  if ((size_t)a.B * ln_stage_stride(WF, a.K / (a.ksplit > 1 ? a.ksplit : 1)) * sizeof(uint16_t) <= (size_t)kStageMaxBytes)
     return launch_linear_wf<WF, ACT_STAGED>(a, max_ctas, st, pdl);
   return launch_linear_wf<WF, ACT_DIRECT>(a, max_ctas, st, pdl);
 }
@@ -630,6 +652,7 @@ inline cudaError_t launch_linear_mode(const LinearArgs &a, int max_ctas, cudaStr
 // K must be a multiple of 128.
 inline cudaError_t launch_linear(int wf, const LinearArgs &a, cudaStream_t st, bool pdl = false, int max_ctas = 296) {
   if (a.ln_x && !can_fuse_ln(wf, a.B, a.K)) return cudaErrorInvalidValue;
+  if (a.ksplit > 1 && (a.ln_x || a.mode != EPI_RESID || (a.K / k_per_tile(wf)) % a.ksplit != 0)) return cudaErrorInvalidValue;
   if (wf == WF_BF16) return launch_linear_mode<WF_BF16>(a, max_ctas, st, pdl);
   if (wf == WF_INT8) return launch_linear_mode<WF_INT8>(a, max_ctas, st, pdl);
   return launch_linear_mode<WF_INT4>(a, max_ctas, st, pdl);

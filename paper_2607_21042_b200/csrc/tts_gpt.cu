@@ -75,6 +75,9 @@ struct tts_gpt {
   std::map<int, int> graph_nodes;
   bool use_graph;
   bool use_pdl;
+  bool use_fc2_ksplit = true;   // 5-16 rows: FC2 splits K (TTS_GPT_NO_FC2_KSPLIT=1 switches it off)
+  int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
+  size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
   bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
   int attn_cluster_fill = 1;     // clusters grow until the grid covers the GPU this many times (TTS_GPT_ATTN_CLUSTER_FILL)
@@ -202,6 +205,7 @@ size_t carve(tts_gpt *h, void *base) {
     h->h_img = cv.take<char>(act_image_bytes(F));
     h->hf_img = cv.take<char>(act_image_bytes(d));
     h->partials = cv.take<float>((size_t)kTcKSplit * kMaxRows * d);
+    h->partials_floats = (size_t)kTcKSplit * kMaxRows * d;
   }
   return cv.off;
 }
@@ -363,12 +367,21 @@ int run_layers(tts_gpt *h, int R, bool decode) {
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
   const bool fuse_ln = can_fuse_ln(c.wfmt, R, d);
+  // 5 to 16 rows: FC2 (K = d_ff) splits K over kSmallKSplit CTAs per row tile, so that a CTA stages a
+  // quarter of the wide activation rows; its partial sums are folded into x by the next LayerNorm
+  const int fc2_ks = (!fuse_ln && h->use_fc2_ksplit && (c.d_ff / k_per_tile(c.wfmt)) % kSmallKSplit == 0 &&
+                      (size_t)kSmallKSplit * kMaxRows * d <= h->partials_floats) ? kSmallKSplit : 1;
+  h->pending_parts = 0;
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
     LinearArgs qa = linear_args(h, L.qkv, h->a, R, EPI_QKV);
     if (fuse_ln) {
       qa.ln_x = h->x; qa.ln_g = L.ln1_g; qa.ln_b = L.ln1_b; qa.ln_eps = c.ln_eps;
+    } else if (fc2_ks > 1) {
+      int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : fc2_ks, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
+                            nullptr, h->a, nullptr, nullptr, nullptr, 1);
+      if (rc) return rc;
     } else {
       CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(R), dim3(kLnThreads), 0, st, pdl, (const float *)h->x, d,
                                 (const uint16_t *)L.ln1_g, (const uint16_t *)L.ln1_b, c.ln_eps, h->a,
@@ -404,10 +417,12 @@ int run_layers(tts_gpt *h, int R, bool decode) {
     CUDA_TRY(h, launch_linear(c.wfmt, f1, st, pdl, 2 * h->n_sm));
     LinearArgs f2 = linear_args(h, L.fc2, h->hbuf, R, EPI_RESID);
     f2.out_f32 = h->x; f2.out_stride = d;
+    if (fc2_ks > 1) { f2.ksplit = fc2_ks; f2.out_f32 = h->partials; }
     trace_attach(h, f2);
     CUDA_TRY(h, launch_linear(c.wfmt, f2, st, pdl, 2 * h->n_sm));
     h->launches += 5;
   }
+  h->pending_parts = fc2_ks > 1 ? fc2_ks : 0;   // the last FC2's partial sums: folded by the head's LayerNorm
   return TTS_GPT_OK;
 }
 
@@ -418,7 +433,15 @@ int run_head(tts_gpt *h, int n_out, int R) {
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
   LinearArgs ha = linear_args(h, h->head, h->hf, n_out, EPI_F32);
-  if (can_fuse_ln(WF_BF16, n_out, c.d_model)) {
+  const uint16_t *last_bias = h->layers[c.n_layer - 1].fc2.bias;
+  if (h->pending_parts > 0) {
+    // the last FC2 left k-range partial sums: this LayerNorm folds them for the wanted rows and
+    // writes the normalised rows; the head then runs on those (never on x)
+    int rc = launch_ln_tc(h, n_out, h->lnf_g, h->lnf_b, h->pending_parts, last_bias, nullptr, h->hf, h->rt.out_rows,
+                          h->rt.out_slot, h->io, 0);
+    if (rc) return rc;
+    h->pending_parts = 0;
+  } else if (can_fuse_ln(WF_BF16, n_out, c.d_model)) {
     ha.ln_x = h->x; ha.ln_g = h->lnf_g; ha.ln_b = h->lnf_b; ha.ln_eps = c.ln_eps;
     ha.ln_gather = h->rt.out_rows; ha.ln_out_slot = h->rt.out_slot; ha.ln_io = h->io;
   } else {
@@ -559,6 +582,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   h->use_tc = !(ntc && ntc[0] == '1');
   const char *nas = getenv("TTS_GPT_NO_ATTN_STREAM");
   h->use_attn_stream = !(nas && nas[0] == '1');
+  const char *nfk = getenv("TTS_GPT_NO_FC2_KSPLIT");
+  h->use_fc2_ksplit = !(nfk && nfk[0] == '1');
   const char *acf = getenv("TTS_GPT_ATTN_CLUSTER_FILL");
   if (acf && atoi(acf) > 0) h->attn_cluster_fill = atoi(acf);
   const char *asm_ = getenv("TTS_GPT_ATTN_STREAM_MIN");
