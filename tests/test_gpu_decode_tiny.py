@@ -122,6 +122,26 @@ def test_batch_invariance_page_permutation_and_reuse(tiny_models):
     eng.destroy()
 
 
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
+@pytest.mark.parametrize("S", [5, 16, 40])
+def test_medium_batches_match_oracle(wfmt, S):
+    """Batches of 5..16 rows take the warp-MMA linears with the separate LayerNorm kernels and the
+    k-split FC2 whose partial sums the next LayerNorm folds; 40 rows take the tensor-core path."""
+    cfg = _tiny(wfmt, max_streams=S, n_pages=S * 4)
+    w = C.make_weights(cfg, seed=3)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    lens = [3 + (7 * i) % 90 for i in range(S)]
+    prefixes = C.make_prefixes(cfg, lens, seed=11)
+    n = 6
+    lg, tk = _run_batch(eng, prefixes, n)
+    for s in range(0, S, max(1, S // 6)):
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk[s][:-1])
+        assert_logits_close(lg[s], ref, "batch of %d, stream %d" % (S, s))
+        check_tokens(tk[s], ref, 0, 1.0, None, "batch of %d, stream %d" % (S, s))
+    eng.destroy()
+
+
 def test_prefix_of_one_row_and_pos0(tiny_models):
     cfg, w, model = tiny_models[C.W_INT4_G128]
     eng = B.TtsGpt(cfg, w, DEV)
