@@ -203,12 +203,16 @@ def run_ours(args):
     barrier()
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.profiler_range:
+        torch.cuda.profiler.start()
     with torch.cuda.stream(eng.stream):
         e0.record()
     tokens, nbytes = decode_run(ids, K, True)
     with torch.cuda.stream(eng.stream):
         e1.record()
     barrier()
+    if args.profiler_range:
+        torch.cuda.profiler.stop()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
     launches = eng.kernel_launches() - l0
@@ -378,6 +382,8 @@ def main():
     ap.add_argument("--wfmt", type=int, default=None, help="weight format override for workload 5")
     ap.add_argument("--cpu-steps", type=int, default=150)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profiler-range", action="store_true",
+                    help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

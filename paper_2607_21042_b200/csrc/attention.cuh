@@ -224,8 +224,12 @@ __device__ __forceinline__ void cta_merge(float m, float l, float (&o)[8], int w
 // ------------------------------------------------------------------------------------------
 // cluster variant (the engine's path)
 // ------------------------------------------------------------------------------------------
+// CLUSTER = false: gridDim.x == 1, one CTA per (row, head); the two variants are separate kernels so
+// that each carries only its own code (these kernels run for a few microseconds and mostly execute
+// every instruction once: instruction fetch shows up in their stall reasons)
+template <bool CLUSTER>
 __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnArgs a) {
-  const int S = gridDim.x, c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
+  const int S = CLUSTER ? gridDim.x : 1, c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
   trace_mark(a.trace, a.trace_slot, 0);
   // The row table and page table were written before the first kernel of the step started, so
   // they may be read ahead of the dependency wait.
@@ -249,7 +253,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   // requested before waiting for that kernel; if it covers the new token, that token's 128-byte K
   // and V rows are fetched again after the wait.
   const int tn = (n_tok - 1) & (kPageTokens - 1);   // the new token's slot in the last page
-  if (S > 1) {
+  if (CLUSTER) {
     // ---- cluster: quarter-page units dealt round-robin over all warps of the cluster ----
     const int GW = S * kAttnWarps, gw = c * kAttnWarps + warp;
     const int n_units = (n_tok + 15) >> 4;   // units that hold at least one token
@@ -330,7 +334,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   if (e < kHeadDim)
     out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
                       : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
-  if (S == 1) {
+  if (!CLUSTER) {
     float M, L, O;
     cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
     if (e < kHeadDim) *out = float_to_bf16_bits(O / L);
@@ -400,7 +404,8 @@ inline cudaError_t launch_attention(const AttnArgs &a, int R, int cluster, cudaS
   }
   cfg.attrs = at;
   cfg.numAttrs = n;
-  return cudaLaunchKernelEx(&cfg, attention_kernel, a);
+  if (cluster > 1) return cudaLaunchKernelEx(&cfg, attention_kernel<true>, a);
+  return cudaLaunchKernelEx(&cfg, attention_kernel<false>, a);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -500,9 +505,15 @@ __global__ void __launch_bounds__(kAttnWarps * 32, 3) attention_stream_kernel(co
       vv[i] = *reinterpret_cast<const uint4 *>(stage + kAttnHalfStage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
       if (patch && i == sel) vv[i] = vn;
     }
+    // The stage may be overwritten only after every read of it has returned: the K reads have (the
+    // scores consumed them); one word of every V read is folded into a value that the fence below
+    // takes as an operand, so the copy cannot be issued ahead of those reads either.
+    uint32_t seen = 0u;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) seen ^= vv[i].x;
     __syncwarp();   // every lane has read the stage
     if (page + kAttnWarps < n_pages && lane == 0) {
-      fence_proxy_async_smem();
+      asm volatile("fence.proxy.async.shared::cta; // after %0" ::"r"(seen) : "memory");
       stream_issue(a, pt, h, page + kAttnWarps, n_tok, stage, bar);
     }
     accum_slots<16>(vv, s, pm, vmask, m, l, o);
