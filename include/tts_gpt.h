@@ -124,6 +124,21 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
                             const float *uniforms, int32_t *out_tokens, float *out_logits,
                             void *out_hidden);
 
+/* n_steps successive decode steps for the same n streams, queued in one call (Section II-C: the
+ * later stages consume tokens and hidden states in chunks, so a caller decodes a chunk at a time).
+ * Same result as n_steps calls of tts_gpt_decode_step in which step 1 takes in_tokens (or, if NULL,
+ * each stream's last sample) and every later step the token the stream sampled in the step before,
+ * on the device.  Step k (0-based) writes out_tokens[k*n + i], out_logits[(k*n + i)*vocab ..] and
+ * out_hidden[(k*n + i)*d ..] and draws uniforms[k*n + i]: DEVICE arrays of n_steps*n rows
+ * (out_logits, out_hidden, uniforms may be NULL as in tts_gpt_decode_step).
+ * Errors as tts_gpt_decode_step, checked for the whole chunk before anything is enqueued:
+ * E_CTX_OVERFLOW if a stream lacks room for n_steps more tokens, E_NO_PAGES if the pool cannot
+ * supply every page the chunk will need, E_ARG if n_steps < 1.  All-or-nothing. */
+int32_t tts_gpt_decode_steps(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
+                             const int32_t *in_tokens, int32_t n_steps, int32_t top_k,
+                             float temperature, const float *uniforms, int32_t *out_tokens,
+                             float *out_logits, void *out_hidden);
+
 /* Close a stream and return its pages to the pool.  E_STREAM if the id is not open. */
 int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t stream_id);
 

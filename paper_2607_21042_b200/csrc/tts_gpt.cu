@@ -734,6 +734,42 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   return rc;
 }
 
+int32_t tts_gpt_decode_steps(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, const int32_t *in_tokens,
+                             int32_t n_steps, int32_t top_k, float temperature, const float *uniforms,
+                             int32_t *out_tokens, float *out_logits, void *out_hidden) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  const tts_gpt_config_t &c = h->cfg;
+  if (n_steps < 1) return fail(h, TTS_GPT_E_ARG, "decode_steps: n_steps must be positive");
+  if (n < 1 || n > c.max_streams || !stream_ids || !out_tokens) return fail(h, TTS_GPT_E_ARG, "decode_steps: bad n or null argument");
+  int rc = check_top_k(h, top_k, temperature, uniforms);
+  if (rc) return rc;
+  // the whole chunk is validated first, so that no step of it can be refused once the first is queued
+  long long pages = 0;
+  char seen[kMaxRows];
+  memset(seen, 0, sizeof seen);
+  for (int i = 0; i < n; ++i) {
+    const int s = stream_ids[i];
+    if (s < 0 || s >= c.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "decode_steps: stream %d is not open", s);
+    if (seen[s]) return fail(h, TTS_GPT_E_STREAM, "decode_steps: stream %d listed twice", s);
+    seen[s] = 1;
+    if ((long long)h->ctx[s] + n_steps > c.max_context)
+      return fail(h, TTS_GPT_E_CTX_OVERFLOW, "decode_steps: stream %d has room for %d more tokens, %d asked", s, c.max_context - h->ctx[s], n_steps);
+    if ((long long)h->pos_next[s] + n_steps > c.max_pos)
+      return fail(h, TTS_GPT_E_CTX_OVERFLOW, "decode_steps: stream %d would run past max_pos %d", s, c.max_pos);
+    pages += (h->ctx[s] + n_steps + 63) / 64 - (h->ctx[s] + 63) / 64;
+  }
+  if (pages > h->n_free) return fail(h, TTS_GPT_E_NO_PAGES, "decode_steps: %lld pages needed, %d free", pages, h->n_free);
+  for (int k = 0; k < n_steps; ++k) {
+    const size_t row0 = (size_t)k * n;
+    rc = tts_gpt_decode_step(h, n, stream_ids, k == 0 ? in_tokens : nullptr, top_k, temperature,
+                             uniforms ? uniforms + row0 : nullptr, out_tokens + row0,
+                             out_logits ? out_logits + row0 * c.vocab : nullptr,
+                             out_hidden ? (uint16_t *)out_hidden + row0 * c.d_model : nullptr);
+    if (rc) return rc;   // only a CUDA failure can get here
+  }
+  return TTS_GPT_OK;
+}
+
 int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   if (s < 0 || s >= h->cfg.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "release_stream: stream %d is not open", s);

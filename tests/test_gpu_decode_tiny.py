@@ -142,6 +142,52 @@ def test_medium_batches_match_oracle(wfmt, S):
     eng.destroy()
 
 
+@pytest.mark.parametrize("wfmt,top_k", [(C.W_BF16, 0), (C.W_INT4_G128, 8)])
+def test_decode_steps_equals_single_steps(tiny_models, wfmt, top_k):
+    """A chunk of steps queued by one call gives bit-identical tokens, logits and hidden rows to the
+    same steps issued one by one, and a chunk that does not fit is refused as a whole."""
+    cfg, w, _ = tiny_models[wfmt]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefixes = C.make_prefixes(cfg, [20, 64, 7], seed=21)
+    S, V, d, n = 3, cfg.vocab, cfg.d_model, 9
+    uni = torch.from_numpy(C.make_uniforms(n + 1, S, seed=5)).to(DEV) if top_k > 1 else None
+
+    def opened():
+        t0 = torch.zeros(S, dtype=torch.int32, device=DEV)
+        ids, _ = eng.prefill([bits_dev(p) for p in prefixes], top_k=top_k, uniforms=None if uni is None else uni[0],
+                             out_tokens=t0)
+        return ids
+
+    ids = opened()
+    tk1 = torch.zeros((n, S), dtype=torch.int32, device=DEV)
+    lg1 = torch.zeros((n, S, V), dtype=torch.float32, device=DEV)
+    hd1 = torch.zeros((n, S, d), dtype=torch.int16, device=DEV)
+    for k in range(n):
+        eng.decode_step(ids, tk1[k], top_k=top_k, uniforms=None if uni is None else uni[k + 1],
+                        out_logits=lg1[k], out_hidden=hd1[k])
+    eng.sync()
+    for s in ids:
+        eng.release_stream(s)
+    ids = opened()
+    tk2 = torch.zeros((n, S), dtype=torch.int32, device=DEV)
+    lg2 = torch.zeros((n, S, V), dtype=torch.float32, device=DEV)
+    hd2 = torch.zeros((n, S, d), dtype=torch.int16, device=DEV)
+    eng.decode_steps(ids, n, tk2, top_k=top_k, uniforms=None if uni is None else uni[1:],
+                     out_logits=lg2, out_hidden=hd2)
+    eng.sync()
+    assert torch.equal(tk1, tk2) and torch.equal(lg1, lg2) and torch.equal(hd1, hd2)
+    # a chunk past max_context is refused before anything is queued; state is untouched
+    before = (eng.stats(), [eng.stream_context(s) for s in ids])
+    with pytest.raises(B.TtsGptError) as ei:
+        eng.decode_steps(ids, cfg.max_context, tk2)
+    assert ei.value.code == B.E_CTX_OVERFLOW
+    with pytest.raises(B.TtsGptError) as ei:
+        eng.decode_steps(ids, 0, tk2)
+    assert ei.value.code == B.E_ARG
+    assert (eng.stats(), [eng.stream_context(s) for s in ids]) == before
+    eng.destroy()
+
+
 def test_prefix_of_one_row_and_pos0(tiny_models):
     cfg, w, model = tiny_models[C.W_INT4_G128]
     eng = B.TtsGpt(cfg, w, DEV)
