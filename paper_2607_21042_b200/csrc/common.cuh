@@ -60,11 +60,20 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 // trace[8*slot + 0..7].
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");   // "memory": the read stays where it is written, e.g. behind a barrier
   return t;
 }
 __device__ __forceinline__ void trace_mark(unsigned long long *trace, int slot, int which, int tid = 0) {
+#ifdef TTS_TRACE_GRID_MAX   // experiments: word 7 of the slot = latest end mark over all CTAs of the grid
+  if (trace && threadIdx.x == tid && which == 2) atomicMax(trace + 8 * slot + 7, global_timer_ns());
+#endif
+#ifdef TTS_TRACE_CTA_EIGHTH   // experiments: the CTA at TTS_TRACE_CTA_EIGHTH/8 of the grid marks instead of the first
+  const unsigned lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+  const unsigned tot = gridDim.x * gridDim.y * gridDim.z;
+  if (trace && threadIdx.x == tid && lin == min(tot - 1, tot * TTS_TRACE_CTA_EIGHTH / 8))
+#else
   if (trace && threadIdx.x == tid && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+#endif
     trace[8 * slot + which] = global_timer_ns();
 }
 
@@ -138,10 +147,14 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 0.5 x (1 + tanh(u)) = x / (1 + exp(-2u)), u = sqrt(2/pi) (x + 0.044715 x^3): the same function, written
+// with one exponential and one reciprocal (about 6 instructions; the library tanhf is about 30 with
+// branches, which made the GELU epilogue of the 128-row FC1 the longest part of that kernel).  The
+// quotient form keeps the relative error at a few ulp in the negative tail too, where 1 + tanh cancels.
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   const float k0 = 0.7978845608028654f, k1 = 0.044715f;
-  float u = k0 * (x + k1 * x * x * x);
-  return 0.5f * x * (1.0f + tanhf(u));
+  const float u = k0 * (x + k1 * x * x * x);
+  return __fdividef(x, 1.0f + __expf(-2.0f * u));
 }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f)); }
 

@@ -304,6 +304,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       }
       trace_mark(a.trace, a.trace_slot, 3);   // last copy issued
     }
+    __syncwarp();   // the warp arrives at the final barrier as a whole
   } else if (warp == 1) {
     // ---- MMA issuer ----
     if (lane == 0) {
@@ -327,6 +328,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       }
       if (!GROUPED) tc_commit(acc_done);
     }
+    __syncwarp();   // as above
   }
 
   // ---- epilogue (warps 2-5): a warp may touch the 32 accumulator lanes 32*(warp%4)..+31 = weight
@@ -356,48 +358,68 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     }
   } else {
     tc_wait(acc_done, 0, failed, a.err);
+    trace_mark(a.trace, a.trace_slot, 4, 64);   // accumulator complete
     tc_fence_after_sync();
     __syncwarp();
     tmem_ld32(tmem_d + ((uint32_t)(lw * 32) << 16), v);
+    trace_mark(a.trace, a.trace_slot, 5, 64);   // accumulator in registers
   }
   if (n_it <= 0) {   // an empty k-range contributes nothing (the accumulator was never written)
 #pragma unroll
     for (int c = 0; c < 32; ++c) v[c] = 0.f;
   }
   if (n < a.N && !*failed) {
-    if (a.wfmt == WF_INT8) {
+    // one straight-line store loop per destination kind: a single loop that branches on the epilogue
+    // mode for every batch row compiled into code whose speed varied 2-4x with unrelated edits
+    const int nb = min(kTcChunkN, a.B - bc * kTcChunkN);   // real batch rows of this chunk
 #pragma unroll
-      for (int c = 0; c < 32; ++c) v[c] *= e_rsc;
-    }
-    const float bias = e_bias;
+    for (int c = 0; c < 32; ++c) v[c] = fmaf(v[c], e_rsc, e_bias);   // int8: per-row scale (1 otherwise), then bias
+    if (a.mode == EPI_GELU) {
+      if (a.gelu_tanh) {
 #pragma unroll
-    for (int c = 0; c < kTcChunkN; ++c) {
-      const int b = bc * kTcChunkN + c;
-      if (b >= a.B) break;
-      float r = v[c] + bias;
-      if (a.mode == EPI_F32) {
-        a.out_f32[(size_t)b * a.out_stride + n] = r;
-      } else if (a.mode == EPI_RESID) {
-        if (a.ksplit == 1) a.out_f32[(size_t)b * a.out_stride + n] += r;
-        else a.out_f32[((size_t)ks * kMaxRows + b) * a.N + n] = r;
-      } else if (a.mode == EPI_GELU) {
-        r = a.gelu_tanh ? gelu_tanh_f(r) : gelu_erf_f(r);
-        *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + image_offset(b, n, kMaxRows)) = float_to_bf16_bits(r);
-      } else {  // EPI_QKV
-        if (n < a.d) {
-          a.out_f32[(size_t)b * a.out_stride + n] = r;
-        } else {
-          const int which = n >= 2 * a.d;
-          const int col = n - (which ? 2 * a.d : a.d);
-          kv_base[c][((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63)] = float_to_bf16_bits(r);
-        }
+        for (int c = 0; c < 32; ++c) v[c] = gelu_tanh_f(v[c]);
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) v[c] = gelu_erf_f(v[c]);
+      }
+      // element (b, n) of the next linear's activation image: rows are 128 bytes apart, the 16-byte
+      // unit of column n moves with b % 8 (swizzle)
+      unsigned char *img = reinterpret_cast<unsigned char *>(a.out_img) + (size_t)(n >> 6) * (kMaxRows * 128) + (size_t)(n & 7) * 2;
+      const int u = (n & 63) >> 3;
+#pragma unroll
+      for (int c = 0; c < 32; ++c) {
+        const int b = bc * kTcChunkN + c;
+        if (c < nb) *reinterpret_cast<uint16_t *>(img + (size_t)b * 128 + (size_t)((u ^ (b & 7)) << 4)) = float_to_bf16_bits(v[c]);
+      }
+    } else if (a.mode == EPI_QKV && n >= a.d) {
+      const int which = n >= 2 * a.d;
+      const int col = n - (which ? 2 * a.d : a.d);
+      const size_t off = ((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63);
+#pragma unroll
+      for (int c = 0; c < 32; ++c)
+        if (c < nb) kv_base[c][off] = float_to_bf16_bits(v[c]);
+    } else {
+      // fp32 rows: logits, q, the residual stream, or this k-range's partial sums
+      const bool partial = a.mode == EPI_RESID && a.ksplit > 1;
+      float *dst = partial ? a.out_f32 + ((size_t)ks * kMaxRows + bc * kTcChunkN) * a.N + n
+                           : a.out_f32 + (size_t)(bc * kTcChunkN) * a.out_stride + n;
+      const size_t step = partial ? (size_t)a.N : (size_t)a.out_stride;
+      if (a.mode == EPI_RESID && !partial) {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c < nb) dst[c * step] += v[c];
+      } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c)
+          if (c < nb) dst[c * step] = v[c];
       }
     }
   }
+  trace_mark(a.trace, a.trace_slot, 6, 64);     // this thread's epilogue done
   }
   tc_fence_before_sync();
   __syncthreads();
-  trace_mark(a.trace, a.trace_slot, 2);
+  trace_mark(a.trace, a.trace_slot, 2, 64);   // by an epilogue thread: its own stores precede the mark
   if (warp == 0) tmem_dealloc(tmem_d, GROUPED ? 2 * kTcChunkN : kTcChunkN);
 }
 
