@@ -264,12 +264,11 @@ def run_ours(args):
 
     peak, peak_kind = measured_peaks()
     gbs = nbytes / (ms * 1e-3) / 1e9
-    # DRAM bytes per step from the ncu capture summarised in
-    # profiles/decode_step_cfg2_bf16_b1_launch_list_and_dram_traffic.md: 1022.7 MB read+written for a step
-    # whose algorithmic bytes are 1015.1 MB (context 405); traffic grows with the same KV term as the
-    # algorithmic bytes, so the measured ratio is applied to this run's bytes per step.
-    # Workload 5 (bf16), profiles/decode_step_cfg5_bf16_b128_launch_list_dram_traffic_and_timeline.md:
-    # 12155.3 MB for a step of 11930.8 MB algorithmic bytes.
+    # DRAM bytes per step from ncu captures of one decode step (dram__bytes_read.sum + dram__bytes_write.sum
+    # over its launches; the summaries sit with the other profiles of this repository).  Workload 2:
+    # 1022.7 MB read+written for a step whose algorithmic bytes are 1015.1 MB (context 405).  Workload 5,
+    # bf16: 12155.3 MB for a step of 11930.8 MB.  Traffic grows with the same KV term as the algorithmic
+    # bytes, so the measured ratio is applied to this run's bytes per step.
     traffic = None
     if args.workload == 2:
         traffic = (nbytes / max(steps_done, 1)) * (1022.7 / 1015.1)
