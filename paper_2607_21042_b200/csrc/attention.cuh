@@ -535,11 +535,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32, 3) attention_stream_kernel(co
 inline bool attention_use_stream(int R, int H, int n_sm) { return R * H >= 4 * n_sm; }
 
 inline cudaError_t launch_attention_stream(const AttnArgs &a, int R, cudaStream_t st, bool pdl) {
-  static bool attr_done = false;
+  static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
   const size_t smem = (size_t)kAttnWarps * kAttnStageBytes;
-  if (!attr_done) {
+  if (attr_once.first()) {
     cudaFuncSetAttribute(attention_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_done = true;
   }
   return launch_kernel(attention_stream_kernel, dim3(1, a.H, R), dim3(kAttnWarps * 32), smem, st, pdl, a);
 }

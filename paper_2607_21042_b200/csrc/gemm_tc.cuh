@@ -437,11 +437,10 @@ __global__ void fold_partials_kernel(const float *__restrict__ part, int n_part,
 inline size_t gemm_tc_smem_bytes() { return (size_t)kTcStages * (kTcABytes + kTcBBytes) + 1024 + 512; }
 
 inline cudaError_t launch_gemm_tc(const GemmTcArgs &a, cudaStream_t st, bool pdl) {
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
+  if (attr_once.first()) {
     cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
     cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tc_smem_bytes());
-    attr_done = true;
   }
   dim3 grid((a.N + kTcTileM - 1) / kTcTileM, (a.B + kTcChunkN - 1) / kTcChunkN, a.ksplit);
   if (a.wfmt == WF_INT4)

@@ -608,10 +608,9 @@ template <int WF, int RT, int MODE, int NB>
 inline cudaError_t launch_linear_nb(const LinearArgs &a, int grid, cudaStream_t st, bool pdl) {
   const int ks = a.ksplit > 1 ? a.ksplit : 1;
   const size_t smem = linear_smem_bytes(WF, RT, MODE, a.B, a.K / ks);
-  static bool attr_done = false;  // opt-in to more than 48 KB of dynamic shared memory, once
-  if (!attr_done) {
+  static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
+  if (attr_once.first()) {
     cudaFuncSetAttribute(linear_kernel<WF, RT, MODE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    attr_done = true;
   }
   return launch_kernel(linear_kernel<WF, RT, MODE, NB>, dim3(grid, ks), dim3(kLinearThreads), smem, st, pdl, a);
 }
