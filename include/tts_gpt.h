@@ -173,6 +173,13 @@ int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots);
  * is open).  Results must not depend on which physical pages a stream receives. */
 int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed);
 
+/* Test aid for the device-side error path: enqueues a one-thread kernel that waits, with the same
+ * bounded wait every kernel of the library uses, at most limit_us microseconds (1..100000) on a
+ * barrier that nothing completes, and on expiry sets the engine's error word exactly as a kernel
+ * whose copy never arrived would.  The next tts_gpt_sync then returns TTS_GPT_E_TIMEOUT once and
+ * clears the word; the engine and the CUDA context stay usable.  Nothing hangs or faults. */
+int32_t tts_gpt_debug_expire_wait(tts_gpt_t *h, uint32_t limit_us);
+
 /* ---------------------------------------------------------------------------------------------
  * Single-kernel entry points: the building blocks of the step, callable on their own (unit parity
  * tests, micro-benchmarks).  All pointers DEVICE unless marked HOST; `cuda_stream` as above; each

@@ -24,7 +24,7 @@ EXPORTS = [
     "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_decode_step", "tts_gpt_decode_steps",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
-    "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace",
+    "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace", "tts_gpt_debug_expire_wait",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
     "tts_gpt_op_linear_tc_scratch_bytes", "tts_gpt_op_linear_tc", "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static", "tts_gpt_op_attention_cluster",
     "tts_gpt_op_layernorm",
@@ -245,6 +245,9 @@ class TtsGpt:
 
     def debug_shuffle_free_pages(self, seed):
         return _check(self.lib.tts_gpt_debug_shuffle_free_pages(self.handle, C.c_uint32(seed)), self.handle)
+
+    def debug_expire_wait(self, limit_us):
+        return _check(self.lib.tts_gpt_debug_expire_wait(self.handle, C.c_uint32(limit_us)), self.handle)
 
     def raw_call(self, name, *args):
         """Return the raw status of a C entry point (tests of error behaviour)."""

@@ -831,6 +831,21 @@ int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t s) {
   return h->ctx[s];
 }
 
+// waits on a barrier nothing completes, for at most limit_ns, then reports like any expired wait
+__global__ void expire_wait_kernel(int *err, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  mbar_init(&bar, 1);
+  if (!mbar_wait_bounded(&bar, 0, limit_ns) && err) atomicExch(err, 1);
+}
+
+int32_t tts_gpt_debug_expire_wait(tts_gpt_t *h, uint32_t limit_us) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  if (limit_us < 1 || limit_us > 100000) return fail(h, TTS_GPT_E_ARG, "expire_wait: limit_us must be in 1..100000");
+  expire_wait_kernel<<<1, 1, 0, h->stream>>>(h->dev_err, (unsigned long long)limit_us * 1000ull);
+  CUDA_TRY(h, cudaGetLastError());
+  return TTS_GPT_OK;
+}
+
 int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   for (char o : h->open) if (o) return fail(h, TTS_GPT_E_STREAM, "shuffle: streams are open");

@@ -188,6 +188,28 @@ def test_decode_steps_equals_single_steps(tiny_models, wfmt, top_k):
     eng.destroy()
 
 
+def test_expired_device_wait_is_reported_and_engine_stays_usable(tiny_models):
+    """A bounded wait that runs out (a barrier nothing completes, 2 ms limit) sets the engine's error
+    word; sync reports TTS_GPT_E_TIMEOUT once; afterwards the engine decodes exactly as before."""
+    cfg, w, _ = tiny_models[C.W_BF16]
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefix = C.make_prefixes(cfg, [40], seed=2)[0]
+    toks_a, logits_a, _, sid = gpu_run_stream(eng, bits_dev(prefix), 5)
+    eng.release_stream(sid)
+    eng.sync()
+    eng.debug_expire_wait(2000)
+    with pytest.raises(B.TtsGptError) as ei:
+        eng.sync()
+    assert ei.value.code == B.E_TIMEOUT
+    eng.sync()                                   # reported once, then clear
+    toks_b, logits_b, _, sid = gpu_run_stream(eng, bits_dev(prefix), 5)
+    assert np.array_equal(toks_a, toks_b) and np.array_equal(logits_a, logits_b)
+    with pytest.raises(B.TtsGptError) as ei:
+        eng.debug_expire_wait(0)
+    assert ei.value.code == B.E_ARG
+    eng.destroy()
+
+
 def test_prefix_of_one_row_and_pos0(tiny_models):
     cfg, w, model = tiny_models[C.W_INT4_G128]
     eng = B.TtsGpt(cfg, w, DEV)
