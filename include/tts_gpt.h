@@ -11,6 +11,8 @@
  * top-k sampling, all in hand-written CUDA kernels.
  *
  * General rules
+ *  - Alignment: prefix embeddings and out_hidden 16 bytes (rows are moved with vector loads and
+ *    stores), token / uniform / logit buffers 4 bytes; a misaligned pointer is refused with E_ARG.
  *  - Every function returns an int32 status: TTS_GPT_OK (0) or a negative TTS_GPT_E_* code.
  *    Nothing throws, aborts or traps the device.  tts_gpt_last_error() describes the last failure.
  *  - Memory: the caller owns every buffer, including the workspace given to tts_gpt_create.  The

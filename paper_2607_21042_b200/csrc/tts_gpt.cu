@@ -471,6 +471,16 @@ int run_embed(tts_gpt *h, int R) {
   return TTS_GPT_OK;
 }
 
+// Output rows are written with vector stores: the hidden rows need 16-byte alignment, the rest their
+// element's.  A misaligned pointer is refused here instead of faulting on the device.
+int check_io_alignment(tts_gpt *h, const void *in_tokens, const void *uniforms, const void *out_tokens,
+                       const void *out_logits, const void *out_hidden) {
+  if ((uintptr_t)in_tokens % 4 || (uintptr_t)uniforms % 4 || (uintptr_t)out_tokens % 4 || (uintptr_t)out_logits % 4)
+    return fail(h, TTS_GPT_E_ARG, "token, uniform and logit buffers must be 4-byte aligned");
+  if ((uintptr_t)out_hidden % 16) return fail(h, TTS_GPT_E_ARG, "out_hidden must be 16-byte aligned");
+  return TTS_GPT_OK;
+}
+
 int check_top_k(tts_gpt *h, int top_k, float temperature, const float *uniforms) {
   if (top_k < 0 || top_k > kMaxTopK) return fail(h, TTS_GPT_E_ARG, "top_k must be in 0..%d", kMaxTopK);
   if (top_k > 1 && !(temperature > 0.f)) return fail(h, TTS_GPT_E_ARG, "temperature must be positive");
@@ -604,9 +614,12 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     return fail(h, TTS_GPT_E_ARG, "prefill: bad n or null argument");
   int rc = check_top_k(h, top_k, temperature, uniforms);
   if (rc) return rc;
+  rc = check_io_alignment(h, nullptr, uniforms, out_tokens, out_logits, out_hidden);
+  if (rc) return rc;
   int pages = 0;
   for (int i = 0; i < n; ++i) {
     if (prefix_len[i] < 1 || !prefix_emb[i]) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has an empty prefix", i);
+    if ((uintptr_t)prefix_emb[i] % 16) return fail(h, TTS_GPT_E_ARG, "prefill: prefix %d is not 16-byte aligned", i);
     if (prefix_len[i] > c.max_context) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "prefill: prefix %d exceeds max_context %d", prefix_len[i], c.max_context);
     if (pos0 && (pos0[i] < 0 || pos0[i] >= c.max_pos)) return fail(h, TTS_GPT_E_ARG, "prefill: pos0 out of range");
     pages += (prefix_len[i] + 63) / 64;
@@ -678,6 +691,8 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   const tts_gpt_config_t &c = h->cfg;
   if (n < 1 || n > c.max_streams || !stream_ids || !out_tokens) return fail(h, TTS_GPT_E_ARG, "decode_step: bad n or null argument");
   int rc = check_top_k(h, top_k, temperature, uniforms);
+  if (rc) return rc;
+  rc = check_io_alignment(h, in_tokens, uniforms, out_tokens, out_logits, out_hidden);
   if (rc) return rc;
   int pages = 0;
   char seen[kMaxRows];

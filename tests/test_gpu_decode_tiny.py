@@ -285,6 +285,9 @@ def test_error_behaviour_leaves_state_untouched(tiny_models):
     assert code(lambda: eng.decode_step([1 - a], out)) == B.E_STREAM                 # not open
     assert code(lambda: eng.decode_step([], out)) == B.E_ARG
     assert code(lambda: eng.decode_step([a], out, top_k=30)) == B.E_ARG              # no uniforms
+    odd = torch.zeros(cfg.d_model + 8, dtype=torch.int16, device=DEV)[1:1 + cfg.d_model].view(1, -1)
+    assert code(lambda: eng.decode_step([a], out, out_hidden=odd)) == B.E_ARG        # 2 bytes off a 16-byte boundary
+    assert eng.stream_context(a) == 127
     eng.decode_step([a], out)                                                        # ctx 127 -> 128: allowed
     assert eng.stream_context(a) == 128
     assert code(lambda: eng.decode_step([a], out)) == B.E_CTX_OVERFLOW               # 129
