@@ -185,7 +185,8 @@ int32_t tts_gpt_debug_expire_wait(tts_gpt_t *h, uint32_t limit_us);
 /* ---------------------------------------------------------------------------------------------
  * Single-kernel entry points: the building blocks of the step, callable on their own (unit parity
  * tests, micro-benchmarks).  All pointers DEVICE unless marked HOST; `cuda_stream` as above; each
- * call enqueues and returns.
+ * call enqueues and returns.  Matrices, activation rows, q, the KV pool and fp32 outputs must be 16-byte
+ * aligned (packed weights and scratch as stated per call); misaligned pointers are refused with E_ARG.
  * ------------------------------------------------------------------------------------------- */
 
 /* Bytes of the streaming layout of one [N,K] linear in format wfmt (weights + scales). */

@@ -903,6 +903,8 @@ int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed
   int rc = tts_gpt_op_linear_packed_bytes(wfmt, N, K, &bytes);
   if (rc) return rc;
   if (!packed || !act || !out || B < 1 || B > kMaxRows) return fail(nullptr, TTS_GPT_E_ARG, "op_linear: bad argument");
+  if ((uintptr_t)packed % 256 || (uintptr_t)act % 16 || (uintptr_t)out % 16 || (uintptr_t)bias % 16)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_linear: packed must be 256-byte, act / out / bias 16-byte aligned");
   PackedLinear pl;
   pl.N = N; pl.K = K; pl.w = (void *)packed;
   pl.s = (uint16_t *)((char *)packed + align256(packed_weight_bytes(wfmt, N, K)));
@@ -926,8 +928,9 @@ int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, 
   int rc = tts_gpt_op_linear_tc_scratch_bytes(N, K, &bytes);
   if (rc) return rc;
   if (wfmt < 0 || wfmt > 2 || !w || !act || !out || !scratch || B < 1 || B > kMaxRows || (uintptr_t)scratch % 1024 ||
-      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit || K % 128 || (wfmt != WF_BF16 && !s))
-    return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad argument");
+      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit || K % 128 || (wfmt != WF_BF16 && !s) ||
+      (uintptr_t)w % 16 || (uintptr_t)s % 16 || (uintptr_t)act % 16 || (uintptr_t)out % 16 || (uintptr_t)bias % 16)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad or misaligned argument");
   cudaStream_t st = (cudaStream_t)cuda_stream;
   char *wimg = (char *)scratch;
   char *aimg = wimg + align256(weight_image_bytes(N, K));
@@ -966,6 +969,9 @@ int32_t tts_gpt_op_attention_scratch_bytes(int32_t R, int32_t n_head, size_t *by
 int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
                              const int32_t *page_table, int32_t pages_per_stream, const int32_t *row_stream,
                              const int32_t *row_pos, void *out, void *scratch, void *cuda_stream) {
+  if ((uintptr_t)q % 16 || (uintptr_t)kv_layer % 16 || (uintptr_t)out % 2 || (uintptr_t)page_table % 4 || (uintptr_t)row_stream % 4 ||
+      (uintptr_t)row_pos % 4)
+    return fail(nullptr, TTS_GPT_E_ARG, "attention: q and the KV pool must be 16-byte aligned, index arrays 4-byte");
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out || !scratch ||
       pages_per_stream < 1 || pages_per_stream > kAttnMaxChunks * kAttnWarps || (uintptr_t)scratch % 256)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention: bad argument");
@@ -1005,6 +1011,9 @@ int32_t tts_gpt_op_attention_static(int32_t R, int32_t n_head, const float *q, c
                                     const int32_t *page_table, int32_t pages_per_stream,
                                     const int32_t *row_stream, const int32_t *row_pos, void *out,
                                     void *cuda_stream) {
+  if ((uintptr_t)q % 16 || (uintptr_t)kv_layer % 16 || (uintptr_t)out % 2 || (uintptr_t)page_table % 4 || (uintptr_t)row_stream % 4 ||
+      (uintptr_t)row_pos % 4)
+    return fail(nullptr, TTS_GPT_E_ARG, "attention: q and the KV pool must be 16-byte aligned, index arrays 4-byte");
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1 || pages_per_stream > kAttnMaxChunks * kAttnWarps)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_static: bad argument");
@@ -1040,6 +1049,9 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
                                      const int32_t *page_table, int32_t pages_per_stream,
                                      const int32_t *row_stream, const int32_t *row_pos, void *out,
                                      int32_t cluster_size, void *cuda_stream) {
+  if ((uintptr_t)q % 16 || (uintptr_t)kv_layer % 16 || (uintptr_t)out % 2 || (uintptr_t)page_table % 4 || (uintptr_t)row_stream % 4 ||
+      (uintptr_t)row_pos % 4)
+    return fail(nullptr, TTS_GPT_E_ARG, "attention: q and the KV pool must be 16-byte aligned, index arrays 4-byte");
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
@@ -1059,7 +1071,9 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
 
 int32_t tts_gpt_op_layernorm(int32_t R, int32_t d, const float *x, const void *g, const void *b, float eps,
                              void *out, void *cuda_stream) {
-  if (R < 1 || d < 1 || d > kLnThreads * kLnMaxPerThread || !x || !g || !b || !out) return fail(nullptr, TTS_GPT_E_ARG, "op_layernorm: bad argument");
+  if (R < 1 || d < 1 || d > kLnThreads * kLnMaxPerThread || !x || !g || !b || !out || (uintptr_t)x % 4 || (uintptr_t)g % 2 ||
+      (uintptr_t)b % 2 || (uintptr_t)out % 2)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_layernorm: bad or misaligned argument");
   layernorm_kernel<<<R, kLnThreads, 0, (cudaStream_t)cuda_stream>>>(x, d, (const uint16_t *)g, (const uint16_t *)b, eps,
                                                                     (uint16_t *)out, nullptr, nullptr, nullptr);
   CUDA_TRY(nullptr, cudaGetLastError());
