@@ -17,7 +17,7 @@
 // residual stream, 4 k-ranges, every linear of the block runs on 120-160 CTAs.  Warp 0 produces
 // (bulk copies into a 5-stage ring guarded by full/empty mbarriers; the weight copies of the first
 // stages are issued before the dependency wait), warp 1 issues the MMAs (4 per k-chunk, M=128,
-// N=32, K=16) and commits each stage back to the producer, and warps 2-5 read the 128x32 fp32
+// N=32, K=16) and commits each stage back to the producer, and warps 2-9 read the 128x32 fp32
 // accumulator out of tensor memory and run the epilogue.  K-split partial sums go to a scratch
 // array that the following LayerNorm kernel folds into the residual stream in a fixed order.
 // Every wait is bounded; on expiry the CTA sets the error word, stops waiting and still releases
@@ -38,8 +38,9 @@ constexpr int kTcKChunk = 64;          // columns per pipeline stage (128 bytes 
 constexpr uint32_t kTcABytes = kTcTileM * 128;   // 16 KB
 constexpr uint32_t kTcBBytes = kTcChunkN * 128;  // 4 KB
 static_assert(kTcChunkN == 32, "the epilogue reads one 32-column accumulator slice per thread");
-constexpr int kTcThreads = 192;          // warp 0: producer, warp 1: MMA issuer, warps 2-5: epilogue
-constexpr int kTcEpiThreads = 128;
+constexpr int kTcThreads = 320;          // warp 0: producer, warp 1: MMA issuer, warps 2-9: epilogue
+constexpr int kTcEpiThreads = 256;
+constexpr int kTcEpiCols = 16;           // accumulator columns (batch rows) per epilogue thread: two warps share a lane quarter
 constexpr int kTcKSplit = 4;            // k-ranges of the two linears that feed the residual stream
 constexpr unsigned long long kTcWaitNs = 2000000000ull;
 
@@ -183,6 +184,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 32 lanes x 16 columns of 32-bit
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 struct GemmTcArgs {
   const void *w_img;        // weight image [N/128][K/64] blocks
   const void *act_img;      // activation image [K/64] blocks of 128 rows
@@ -217,7 +232,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 }
 
 // GROUPED (int4 weights): the MMAs of each 128-column group accumulate into one of two 32-column
-// tensor-memory buffers; while the next group runs in the other buffer, the four warps read the
+// tensor-memory buffers; while the next group runs in the other buffer, the epilogue warps read the
 // finished group out, multiply it by the group's scale of their weight row and add it to fp32
 // registers.  Otherwise one 32-column accumulator collects the whole k-range.
 template <bool GROUPED>
@@ -230,7 +245,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   uint64_t *empty = full + kTcStages;
   uint64_t *acc_done = empty + kTcStages;
   uint64_t *grp_done = acc_done + 1;   // [2] group buffer filled (MMA warp -> all)
-  uint64_t *grp_free = grp_done + 2;   // [2] group buffer read out (all 128 threads -> MMA warp)
+  uint64_t *grp_free = grp_done + 2;   // [2] group buffer read out (all epilogue threads -> MMA warp)
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(grp_free + 2);
   volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
   uint16_t **kv_base = reinterpret_cast<uint16_t **>(tmem_slot + 4);   // [32] EPI_QKV: page slot of each batch row
@@ -331,15 +346,16 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     __syncwarp();   // as above
   }
 
-  // ---- epilogue (warps 2-5): a warp may touch the 32 accumulator lanes 32*(warp%4)..+31 = weight
+  // ---- epilogue (warps 2-9; warps w and w+4 share a lane quarter and take 16 columns each): a warp may touch the 32 accumulator lanes 32*(warp%4)..+31 = weight
   //      rows n; columns = batch rows ----
   if (warp >= 2) {
   const int lw = warp & 3;
+  const int c0 = ((warp - 2) >> 2) * kTcEpiCols;   // this thread's first accumulator column
   const int n = nt * kTcTileM + lw * 32 + lane;
-  float v[32];
+  float v[kTcEpiCols];
   if (GROUPED) {
 #pragma unroll
-    for (int c = 0; c < 32; ++c) v[c] = 0.f;
+    for (int c = 0; c < kTcEpiCols; ++c) v[c] = 0.f;
     const int n_groups = (n_it + 1) >> 1;
     const int KG = a.K / 128;
     for (int g = 0; g < n_groups; ++g) {
@@ -349,46 +365,46 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       tc_wait(grp_done + (g & 1), (g >> 1) & 1, failed, a.err);
       tc_fence_after_sync();
       __syncwarp();
-      float t[32];
-      tmem_ld32(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)(g & 1) * 32u, t);
+      float t[kTcEpiCols];
+      tmem_ld16(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)(g & 1) * 32u + (uint32_t)c0, t);
       tc_fence_before_sync();
       mbar_arrive(grp_free + (g & 1));   // the buffer may take the group after next
 #pragma unroll
-      for (int c = 0; c < 32; ++c) v[c] = fmaf(sc, t[c], v[c]);
+      for (int c = 0; c < kTcEpiCols; ++c) v[c] = fmaf(sc, t[c], v[c]);
     }
   } else {
     tc_wait(acc_done, 0, failed, a.err);
     trace_mark(a.trace, a.trace_slot, 4, 64);   // accumulator complete
     tc_fence_after_sync();
     __syncwarp();
-    tmem_ld32(tmem_d + ((uint32_t)(lw * 32) << 16), v);
+    tmem_ld16(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)c0, v);
     trace_mark(a.trace, a.trace_slot, 5, 64);   // accumulator in registers
   }
   if (n_it <= 0) {   // an empty k-range contributes nothing (the accumulator was never written)
 #pragma unroll
-    for (int c = 0; c < 32; ++c) v[c] = 0.f;
+    for (int c = 0; c < kTcEpiCols; ++c) v[c] = 0.f;
   }
   if (n < a.N && !*failed) {
     // one straight-line store loop per destination kind: a single loop that branches on the epilogue
     // mode for every batch row compiled into code whose speed varied 2-4x with unrelated edits
-    const int nb = min(kTcChunkN, a.B - bc * kTcChunkN);   // real batch rows of this chunk
+    const int nb = min(kTcEpiCols, a.B - bc * kTcChunkN - c0);   // real batch rows among this thread's columns
 #pragma unroll
-    for (int c = 0; c < 32; ++c) v[c] = fmaf(v[c], e_rsc, e_bias);   // int8: per-row scale (1 otherwise), then bias
+    for (int c = 0; c < kTcEpiCols; ++c) v[c] = fmaf(v[c], e_rsc, e_bias);   // int8: per-row scale (1 otherwise), then bias
     if (a.mode == EPI_GELU) {
       if (a.gelu_tanh) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = gelu_tanh_f(v[c]);
+        for (int c = 0; c < kTcEpiCols; ++c) v[c] = gelu_tanh_f(v[c]);
       } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) v[c] = gelu_erf_f(v[c]);
+        for (int c = 0; c < kTcEpiCols; ++c) v[c] = gelu_erf_f(v[c]);
       }
       // element (b, n) of the next linear's activation image: rows are 128 bytes apart, the 16-byte
       // unit of column n moves with b % 8 (swizzle)
       unsigned char *img = reinterpret_cast<unsigned char *>(a.out_img) + (size_t)(n >> 6) * (kMaxRows * 128) + (size_t)(n & 7) * 2;
       const int u = (n & 63) >> 3;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const int b = bc * kTcChunkN + c;
+      for (int c = 0; c < kTcEpiCols; ++c) {
+        const int b = bc * kTcChunkN + c0 + c;
         if (c < nb) *reinterpret_cast<uint16_t *>(img + (size_t)b * 128 + (size_t)((u ^ (b & 7)) << 4)) = float_to_bf16_bits(v[c]);
       }
     } else if (a.mode == EPI_QKV && n >= a.d) {
@@ -396,21 +412,21 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       const int col = n - (which ? 2 * a.d : a.d);
       const size_t off = ((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63);
 #pragma unroll
-      for (int c = 0; c < 32; ++c)
-        if (c < nb) kv_base[c][off] = float_to_bf16_bits(v[c]);
+      for (int c = 0; c < kTcEpiCols; ++c)
+        if (c < nb) kv_base[c0 + c][off] = float_to_bf16_bits(v[c]);
     } else {
       // fp32 rows: logits, q, the residual stream, or this k-range's partial sums
       const bool partial = a.mode == EPI_RESID && a.ksplit > 1;
-      float *dst = partial ? a.out_f32 + ((size_t)ks * kMaxRows + bc * kTcChunkN) * a.N + n
-                           : a.out_f32 + (size_t)(bc * kTcChunkN) * a.out_stride + n;
+      float *dst = partial ? a.out_f32 + ((size_t)ks * kMaxRows + bc * kTcChunkN + c0) * a.N + n
+                           : a.out_f32 + (size_t)(bc * kTcChunkN + c0) * a.out_stride + n;
       const size_t step = partial ? (size_t)a.N : (size_t)a.out_stride;
       if (a.mode == EPI_RESID && !partial) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c)
+        for (int c = 0; c < kTcEpiCols; ++c)
           if (c < nb) dst[c * step] += v[c];
       } else {
 #pragma unroll
-        for (int c = 0; c < 32; ++c)
+        for (int c = 0; c < kTcEpiCols; ++c)
           if (c < nb) dst[c * step] = v[c];
       }
     }
