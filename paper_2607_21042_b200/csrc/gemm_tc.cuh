@@ -15,9 +15,9 @@
 // A CTA owns a 128-row weight tile (the M operand), one chunk of 32 batch rows (the N operand) and
 // a contiguous range of k-chunks; with 4 batch chunks of 32 and, for the two linears that feed the
 // residual stream, 4 k-ranges, every linear of the block runs on 120-160 CTAs.  Warp 0 produces
-// (bulk copies into a 5-stage ring guarded by full/empty mbarriers; the weight copies of the first
-// stages are issued before the dependency wait), warp 1 issues the MMAs (4 per k-chunk, M=128,
-// N=32, K=16) and commits each stage back to the producer, and warps 2-9 read the 128x32 fp32
+// (bulk copies into a 4-stage ring guarded by full/empty mbarriers; the weight copies of the first
+// stages are issued before the dependency wait), warps 1 and 10 issue the MMAs (4 per k-chunk, M=128,
+// N=32, K=16; even and odd k-chunks into two accumulators) and commit each stage back to the producer, and warps 2-9 read the 128x32 fp32
 // accumulator out of tensor memory and run the epilogue.  K-split partial sums go to a scratch
 // array that the following LayerNorm kernel folds into the residual stream in a fixed order.
 // Every wait is bounded; on expiry the CTA sets the error word, stops waiting and still releases
@@ -31,14 +31,14 @@ namespace ttsgpt {
 // Measured on B200 (FC1 shape, 128 rows): chunks of 32 rows with a 5-stage ring (160 CTAs, two per
 // SM) beat chunks of 64 rows with 4 or 8 stages by 6-13 us per linear although the latter re-read
 // the weights from L2 only twice: more CTAs keep more copies in flight and overlap their epilogues.
-constexpr int kTcStages = 5;            // 5 x 20 KB: two CTAs fit one SM
+constexpr int kTcStages = 4;            // even: a stage is always consumed by the same MMA issuer (see the issuers); 4 x 20 KB
 constexpr int kTcTileM = 128;          // weight rows per CTA
 constexpr int kTcChunkN = 32;          // batch rows per CTA (the N operand; weights are re-read once per chunk)
 constexpr int kTcKChunk = 64;          // columns per pipeline stage (128 bytes of bf16)
 constexpr uint32_t kTcABytes = kTcTileM * 128;   // 16 KB
 constexpr uint32_t kTcBBytes = kTcChunkN * 128;  // 4 KB
 static_assert(kTcChunkN == 32, "the epilogue reads one 32-column accumulator slice per thread");
-constexpr int kTcThreads = 320;          // warp 0: producer, warp 1: MMA issuer, warps 2-9: epilogue
+constexpr int kTcThreads = 352;          // warp 0: producer, warp 1: MMA issuer, warps 2-9: epilogue
 constexpr int kTcEpiThreads = 256;
 constexpr int kTcEpiCols = 16;           // accumulator columns (batch rows) per epilogue thread: two warps share a lane quarter
 constexpr int kTcKSplit = 4;            // k-ranges of the two linears that feed the residual stream
@@ -261,12 +261,12 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kTcStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-    mbar_init(acc_done, 1);
+    mbar_init(acc_done, GROUPED ? 1 : 2);   // both MMA issuers commit to it
     mbar_init(grp_done, 1); mbar_init(grp_done + 1, 1);
     mbar_init(grp_free, kTcEpiThreads); mbar_init(grp_free + 1, kTcEpiThreads);
     *failed = 0;
   }
-  if (warp == 0) tmem_alloc(tmem_slot, GROUPED ? 2 * kTcChunkN : kTcChunkN);
+  if (warp == 0) tmem_alloc(tmem_slot, 2 * kTcChunkN);
   if (a.mode == EPI_QKV && threadIdx.x >= 64 && threadIdx.x < 64 + kTcChunkN) {   // page slots of this chunk's batch rows
     const int bl = threadIdx.x - 64;
     const int b = bc * kTcChunkN + bl;
@@ -320,11 +320,20 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
       trace_mark(a.trace, a.trace_slot, 3);   // last copy issued
     }
     __syncwarp();   // the warp arrives at the final barrier as a whole
-  } else if (warp == 1) {
-    // ---- MMA issuer ----
-    if (lane == 0) {
+  } else if (warp == 1 || warp == 10) {
+    // ---- MMA issuers: two threads of different warps, each with its own accumulator.  Ungrouped:
+    //      warp 1 takes the even k-chunks into accumulator 0, warp 10 the odd ones into accumulator 1; the
+    //      epilogue adds the two.  Measured: the rate of the chain stays what it is (about 0.33 us per
+    //      k-chunk and CTA), but the accumulators are complete 0.8 us after the last stage is handed over
+    //      instead of 1.35 us.  The ring has an even number of stages so that a stage is always consumed
+    //      by the same issuer: a thread may wait on an mbarrier at most one phase ahead, and with an odd
+    //      ring the issuer that runs ahead would ask for a phase whose predecessor is still pending and
+    //      be told it is complete ----
+    const int par = GROUPED ? 0 : (warp == 10 ? 1 : 0);
+    const int stride = GROUPED ? 1 : 2;
+    if (lane == 0 && !(GROUPED && warp == 10)) {
       const uint32_t idesc = tc_instr_desc(kTcTileM, kTcChunkN);
-      for (int i = 0; i < n_it; ++i) {
+      for (int i = par; i < n_it; i += stride) {
         const int s = i % kTcStages;
         tc_wait(full + s, (i / kTcStages) & 1, failed, a.err);
         const int g = i >> 1;   // group of this k-chunk inside the k-range
@@ -332,10 +341,10 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
         tc_fence_after_sync();
         const unsigned char *sa = ring + (size_t)s * (kTcABytes + kTcBBytes);
         const uint64_t da = tc_smem_desc(sa), db = tc_smem_desc(sa + kTcABytes);
-        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * kTcChunkN : tmem_d;
+        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * kTcChunkN : tmem_d + (uint32_t)par * kTcChunkN;
 #pragma unroll
         for (int j = 0; j < kTcKChunk / 16; ++j) {  // 32 bytes further along K per step: +2 in 16-byte units
-          const bool fresh = GROUPED ? ((i & 1) == 0 && j == 0) : (i == 0 && j == 0);
+          const bool fresh = GROUPED ? ((i & 1) == 0 && j == 0) : (i == par && j == 0);
           tc_mma(dst, da + 2 * j, db + 2 * j, idesc, fresh ? 0u : 1u);
         }
         tc_commit(empty + s);   // the stage may be refilled once these MMAs have read it
@@ -348,7 +357,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
 
   // ---- epilogue (warps 2-9; warps w and w+4 share a lane quarter and take 16 columns each): a warp may touch the 32 accumulator lanes 32*(warp%4)..+31 = weight
   //      rows n; columns = batch rows ----
-  if (warp >= 2) {
+  if (warp >= 2 && warp < 10) {
   const int lw = warp & 3;
   const int c0 = ((warp - 2) >> 2) * kTcEpiCols;   // this thread's first accumulator column
   const int n = nt * kTcTileM + lw * 32 + lane;
@@ -378,6 +387,12 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     tc_fence_after_sync();
     __syncwarp();
     tmem_ld16(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)c0, v);
+    if (n_it >= 2) {   // the odd k-chunks' accumulator
+      float t2[kTcEpiCols];
+      tmem_ld16(tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)kTcChunkN + (uint32_t)c0, t2);
+#pragma unroll
+      for (int c = 0; c < kTcEpiCols; ++c) v[c] += t2[c];
+    }
     trace_mark(a.trace, a.trace_slot, 5, 64);   // accumulator in registers
   }
   if (n_it <= 0) {   // an empty k-range contributes nothing (the accumulator was never written)
@@ -436,7 +451,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   tc_fence_before_sync();
   __syncthreads();
   trace_mark(a.trace, a.trace_slot, 2, 64);   // by an epilogue thread: its own stores precede the mark
-  if (warp == 0) tmem_dealloc(tmem_d, GROUPED ? 2 * kTcChunkN : kTcChunkN);
+  if (warp == 0) tmem_dealloc(tmem_d, 2 * kTcChunkN);
 }
 
 // out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)
