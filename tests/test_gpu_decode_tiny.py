@@ -210,6 +210,36 @@ def test_expired_device_wait_is_reported_and_engine_stays_usable(tiny_models):
     eng.destroy()
 
 
+def test_two_engines_interleaved(tiny_models):
+    """Two engines (different weight formats, own workspaces and streams) used alternately in one process
+    give what each gives alone: the library keeps no per-process state between them."""
+    cfg_a, w_a, _ = tiny_models[C.W_BF16]
+    cfg_b, w_b, _ = tiny_models[C.W_INT4_G128]
+    pre_a = C.make_prefixes(cfg_a, [33], seed=4)[0]
+    pre_b = C.make_prefixes(cfg_b, [70], seed=5)[0]
+    n = 6
+    solo = []
+    for cfg, w, pre in ((cfg_a, w_a, pre_a), (cfg_b, w_b, pre_b)):
+        eng = B.TtsGpt(cfg, w, DEV)
+        toks, logits, _, _ = gpu_run_stream(eng, bits_dev(pre), n)
+        solo.append((toks, logits))
+        eng.destroy()
+    ea, eb = B.TtsGpt(cfg_a, w_a, DEV), B.TtsGpt(cfg_b, w_b, DEV)
+    V = cfg_a.vocab
+    ta = torch.zeros(n + 1, dtype=torch.int32, device=DEV); la = torch.zeros((n + 1, V), dtype=torch.float32, device=DEV)
+    tb = torch.zeros(n + 1, dtype=torch.int32, device=DEV); lb = torch.zeros((n + 1, V), dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    ia, _ = ea.prefill([bits_dev(pre_a)], out_tokens=ta[0:1], out_logits=la[0:1])
+    ib, _ = eb.prefill([bits_dev(pre_b)], out_tokens=tb[0:1], out_logits=lb[0:1])
+    for k in range(1, n + 1):
+        ea.decode_step(ia, ta[k:k + 1], out_logits=la[k:k + 1])
+        eb.decode_step(ib, tb[k:k + 1], out_logits=lb[k:k + 1])
+    ea.sync(); eb.sync()
+    assert np.array_equal(ta.cpu().numpy(), solo[0][0]) and np.array_equal(la.cpu().numpy(), solo[0][1])
+    assert np.array_equal(tb.cpu().numpy(), solo[1][0]) and np.array_equal(lb.cpu().numpy(), solo[1][1])
+    ea.destroy(); eb.destroy()
+
+
 def test_prefix_of_one_row_and_pos0(tiny_models):
     cfg, w, model = tiny_models[C.W_INT4_G128]
     eng = B.TtsGpt(cfg, w, DEV)
