@@ -544,6 +544,133 @@ inline cudaError_t launch_attention_stream(const AttnArgs &a, int R, cudaStream_
 }
 
 // ------------------------------------------------------------------------------------------
+// prefill variant: the rows of a prefill pass are consecutive positions of a few streams, so rows
+// of one stream read the same K/V pages.  A CTA takes 8 consecutive rows of the pass for one head,
+// one row per warp; it walks the pages of each stream its rows belong to (rows of a pass are
+// stream-major, so a CTA's rows split into at most 8 runs of one stream each), brings a page's K and
+// V blocks into shared memory once by bulk asynchronous copies, and every warp whose row belongs
+// to that stream and reaches into that page folds it into its own running softmax.  The page
+// traffic from L2 drops eightfold against one CTA per row; no merge between warps is needed.
+// ------------------------------------------------------------------------------------------
+constexpr int kAttnPrefillRows = 8;   // rows (= warps) per CTA
+
+__global__ void __launch_bounds__(kAttnPrefillRows * 32) attention_prefill_kernel(const AttnArgs a, int R) {
+  __shared__ __align__(128) unsigned char stages[2][kAttnStageBytes];   // two pages: K 8 KB | V 8 KB each
+  __shared__ __align__(8) uint64_t bars[2];
+  __shared__ int seg_stream[kAttnPrefillRows], seg_i0[kAttnPrefillRows], seg_i1[kAttnPrefillRows], seg_last[kAttnPrefillRows];
+  __shared__ int n_seg_s;
+  const int h = blockIdx.y, r0 = blockIdx.z * kAttnPrefillRows;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tg = lane >> 3, sub = lane & 7;
+  const int r = r0 + warp;
+  const bool have_row = r < R;
+  trace_mark(a.trace, a.trace_slot, 0);
+  if (threadIdx.x == 0) {
+    mbar_init(bars, 1); mbar_init(bars + 1, 1);
+    // runs of rows of one stream (the row table is final before the pass's first kernel starts)
+    const int r_end = min(R, r0 + kAttnPrefillRows);
+    int n = 0, i0 = r0;
+    while (i0 < r_end) {
+      const int s = a.row_stream[i0];
+      int i1 = i0 + 1;
+      while (i1 < r_end && a.row_stream[i1] == s) ++i1;
+      seg_stream[n] = s; seg_i0[n] = i0; seg_i1[n] = i1; seg_last[n] = a.row_pos[i1 - 1];
+      ++n; i0 = i1;
+    }
+    n_seg_s = n;
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  pdl_wait();     // the K/V rows of this pass were written by the QKV kernel in front: nothing is read before
+  trace_mark(a.trace, a.trace_slot, 1);
+  const int n_seg = n_seg_s;
+  const int my_pos = have_row ? a.row_pos[r] : -1;
+  float m = -INFINITY, l = 0.f;
+  float o[8], qv[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) { o[e] = 0.f; qv[e] = 0.f; }
+  if (have_row) load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
+
+  // page jobs in order: for each run, pages 0 .. last_pos/64.  Thread 0 requests job j+1 into the other
+  // stage before the warps fold job j.
+  auto issue = [&](int seg, int p, int slot) {
+    const int last_pos = seg_last[seg];
+    const int n_here = min(kPageTokens, last_pos + 1 - p * kPageTokens);
+    const uint32_t bytes = (uint32_t)n_here * kHeadDim * 2;
+    const int phys = a.page_table[(size_t)seg_stream[seg] * a.pps + p];
+    const uint16_t *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
+    mbar_expect_tx(bars + slot, 2 * bytes);
+    bulk_copy_g2s(stages[slot], K, bytes, bars + slot);
+    bulk_copy_g2s(stages[slot] + kAttnHalfStage, K + (size_t)a.H * kPageElems, bytes, bars + slot);
+  };
+  int iseg = 0, ip = 0;          // thread 0: the next job to request
+  if (threadIdx.x == 0 && n_seg > 0) {
+    issue(0, 0, 0);
+    ip = 1;
+    if (ip > seg_last[0] / kPageTokens) { iseg = 1; ip = 0; }
+  }
+  bool dead = false;   // a copy did not arrive in time: stop folding, keep walking the barriers
+  int j = 0;
+  for (int seg = 0; seg < n_seg; ++seg) {
+    const int n_pages = seg_last[seg] / kPageTokens + 1;
+    const bool mine = have_row && r >= seg_i0[seg] && r < seg_i1[seg];
+    for (int p = 0; p < n_pages; ++p, ++j) {
+      const int slot = j & 1;
+      if (threadIdx.x == 0 && iseg < n_seg) {   // job j+1 into the stage that job j-1 used (free since the barrier below)
+        issue(iseg, ip, slot ^ 1);
+        if (++ip > seg_last[iseg] / kPageTokens) { ++iseg; ip = 0; }
+      }
+      if (!dead && !mbar_wait_bounded(bars + slot, (uint32_t)(j >> 1) & 1u, kAttnWaitNs)) {
+        if (a.err) atomicExch(a.err, 1);
+        mbar_wait_bounded(bars + slot, (uint32_t)(j >> 1) & 1u, kAttnWaitNs);   // a last chance for the copy in flight
+        dead = true;
+      }
+      const unsigned char *stage = stages[slot];
+      const int n_mine = mine ? min(kPageTokens, my_pos + 1 - p * kPageTokens) : 0;   // tokens of this page the row sees
+      if (!dead && n_mine > 0) {   // warp-uniform
+        uint32_t vmask = 0u;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) vmask |= (tg + 4 * i < n_mine) ? (1u << i) : 0u;
+        uint4 kk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          kk[i] = *reinterpret_cast<const uint4 *>(stage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
+        float sc[16];
+        const float pm = score_slots<16>(kk, qv, vmask, sc);
+        uint4 vv[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          vv[i] = *reinterpret_cast<const uint4 *>(stage + kAttnHalfStage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
+        accum_slots<16>(vv, sc, pm, vmask, m, l, o);
+      }
+      __syncthreads();   // every warp is done with this stage (all reads consumed): it may be refilled
+      if (threadIdx.x == 0) fence_proxy_async_smem();
+    }
+  }
+  trace_mark(a.trace, a.trace_slot, 3);
+  // the warp's result: sum the partial outputs over the 4 token groups, then lanes tg == 0 write 8 values each
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 8);
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 16);
+  }
+  if (have_row && tg == 0 && !dead) {
+    const float inv = 1.0f / l;
+    const uint4 y = make_uint4(pack_bf16x2(o[0] * inv, o[1] * inv), pack_bf16x2(o[2] * inv, o[3] * inv),
+                               pack_bf16x2(o[4] * inv, o[5] * inv), pack_bf16x2(o[6] * inv, o[7] * inv));
+    const int col = h * kHeadDim + 8 * sub;
+    if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, col)) = y;
+    else *reinterpret_cast<uint4 *>(a.out + (size_t)r * a.H * kHeadDim + col) = y;
+  }
+  trace_mark(a.trace, a.trace_slot, 2);
+}
+
+inline cudaError_t launch_attention_prefill(const AttnArgs &a, int R, cudaStream_t st, bool pdl) {
+  const int groups = (R + kAttnPrefillRows - 1) / kAttnPrefillRows;
+  return launch_kernel(attention_prefill_kernel, dim3(1, a.H, groups), dim3(kAttnPrefillRows * 32), 0, st, pdl, a, R);
+}
+
+// ------------------------------------------------------------------------------------------
 // ticket variant: chunks of 4 pages per CTA, partial results through global scratch, merged by
 // the CTA that arrives last at the row's ticket counter (no spinning)
 // ------------------------------------------------------------------------------------------

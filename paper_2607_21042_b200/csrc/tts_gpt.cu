@@ -79,6 +79,7 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
+  bool use_attn_prefill = true;  // shared-page attention in prefill passes (TTS_GPT_NO_ATTN_PREFILL=1 switches it off)
   bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
   int attn_cluster_fill = 1;     // clusters grow until the grid covers the GPU this many times (TTS_GPT_ATTN_CLUSTER_FILL)
   int attn_stream_min_pairs = 0; // (row, head) pairs from which it is used; 0: attention_use_stream decides (TTS_GPT_ATTN_STREAM_MIN)
@@ -251,6 +252,8 @@ void trace_attach(tts_gpt *h, Args &a) {
 cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool pdl) {
   aa.err = h->dev_err;
   aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
+  // prefill passes: rows of one stream share their pages (one CTA per 8 rows and head)
+  if (!aa.old_pages_final && h->use_attn_prefill && R >= kAttnPrefillRows) return launch_attention_prefill(aa, R, st, pdl);
   const bool stream = h->attn_stream_min_pairs > 0 ? R * aa.H >= h->attn_stream_min_pairs : attention_use_stream(R, aa.H, h->n_sm);
   if (h->use_attn_stream && stream) return launch_attention_stream(aa, R, st, pdl);
   return launch_attention(aa, R, attention_cluster_size(R, aa.H, h->n_sm, h->attn_cluster_fill), st, pdl);
@@ -590,6 +593,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   }
   const char *ntc = getenv("TTS_GPT_NO_TC");
   h->use_tc = !(ntc && ntc[0] == '1');
+  const char *nap = getenv("TTS_GPT_NO_ATTN_PREFILL");
+  h->use_attn_prefill = !(nap && nap[0] == '1');
   const char *nas = getenv("TTS_GPT_NO_ATTN_STREAM");
   h->use_attn_stream = !(nas && nas[0] == '1');
   const char *nfk = getenv("TTS_GPT_NO_FC2_KSPLIT");
