@@ -231,8 +231,10 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
  * cluster_size 1, 2, 4 or 8: each (row, head) is split over a thread-block cluster of that many
  * CTAs that merge their partial results through distributed shared memory (small batches).
  * cluster_size 0: the streaming variant the engine uses for large batches, one CTA per (row, head)
- * whose warps pull whole K/V pages into shared memory with bulk asynchronous copies.  Its waits on
- * those copies are bounded; this stand-alone entry does not report an expired wait (the engine
+ * whose warps pull whole K/V pages into shared memory with bulk asynchronous copies.
+ * cluster_size -1: the prefill variant (rows must be ordered as in a prefill pass: grouped by stream,
+ * positions ascending inside a stream): 8 consecutive rows per CTA share each K/V page.  The waits on
+ * the copies of both are bounded; this stand-alone entry does not report an expired wait (the engine
  * does, as TTS_GPT_E_TIMEOUT). */
 int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
                                      const int32_t *page_table, int32_t pages_per_stream,

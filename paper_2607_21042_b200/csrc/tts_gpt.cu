@@ -1060,14 +1060,18 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
-  if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
-    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be 0, 1, 2, 4 or 8");
+  if (cluster_size != -1 && cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be -1, 0, 1, 2, 4 or 8");
   AttnArgs a;
   memset(&a, 0, sizeof a);
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
   a.row_pos = row_pos; a.out = (uint16_t *)out; a.H = n_head; a.pps = pages_per_stream;
   if (cluster_size == 0) {
     CUDA_TRY(nullptr, launch_attention_stream(a, R, (cudaStream_t)cuda_stream, false));
+    return TTS_GPT_OK;
+  }
+  if (cluster_size == -1) {   // rows must be stream-major with ascending positions, as in a prefill pass
+    CUDA_TRY(nullptr, launch_attention_prefill(a, R, (cudaStream_t)cuda_stream, false));
     return TTS_GPT_OK;
   }
   CUDA_TRY(nullptr, launch_attention(a, R, cluster_size, (cudaStream_t)cuda_stream, false));
