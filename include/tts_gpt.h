@@ -233,9 +233,12 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
  * cluster_size 0: the streaming variant the engine uses for large batches, one CTA per (row, head)
  * whose warps pull whole K/V pages into shared memory with bulk asynchronous copies.
  * cluster_size -1: the prefill variant (rows must be ordered as in a prefill pass: grouped by stream,
- * positions ascending inside a stream): 8 consecutive rows per CTA share each K/V page.  The waits on
- * the copies of both are bounded; this stand-alone entry does not report an expired wait (the engine
- * does, as TTS_GPT_E_TIMEOUT). */
+ * positions ascending inside a stream): 8 consecutive rows per CTA share each K/V page.
+ * cluster_size -2: the prefill variant the engine uses, same requirement on the rows: 16 consecutive rows
+ * per CTA, Q K^T and P V on the tensor cores (bf16 operands: Q and the softmax weights are rounded to
+ * bf16, sums and accumulators stay fp32).  It has no waits.
+ * The waits on the copies of variants 0 and -1 are bounded; this stand-alone entry does not report an
+ * expired wait (the engine does, as TTS_GPT_E_TIMEOUT).  q, out and kv_layer must be 16-byte aligned. */
 int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, const void *kv_layer,
                                      const int32_t *page_table, int32_t pages_per_stream,
                                      const int32_t *row_stream, const int32_t *row_pos, void *out,

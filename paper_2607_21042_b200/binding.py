@@ -327,8 +327,8 @@ def op_attention(q, kv_layer, page_table, row_stream, row_pos, scratch=None, str
 
 
 def op_attention_cluster(q, kv_layer, page_table, row_stream, row_pos, cluster_size, stream=None):
-    """cluster_size 1, 2, 4, 8: cluster variant; 0: streaming variant; -1: prefill variant (rows grouped by
-    stream with ascending positions)."""
+    """cluster_size 1, 2, 4, 8: cluster variant; 0: streaming variant; -1: prefill variant on the CUDA cores,
+    -2: prefill variant on the tensor cores (both: rows grouped by stream with ascending positions)."""
     R, dm = q.shape
     H = dm // 64
     out = torch.empty((R, dm), dtype=torch.int16, device=q.device)

@@ -552,11 +552,30 @@ inline cudaError_t launch_attention_stream(const AttnArgs &a, int R, cudaStream_
 // to that stream and reaches into that page folds it into its own running softmax.  The page
 // traffic from L2 drops eightfold against one CTA per row; no merge between warps is needed.
 // ------------------------------------------------------------------------------------------
-constexpr int kAttnPrefillRows = 8;   // rows (= warps) per CTA
+constexpr int kAttnPrefillRows = 8;     // rows (= warps) per CTA
+constexpr int kAttnPrefillStages = 4;   // pages in flight or in use per CTA (a ring of 16 KB stages)
 
-__global__ void __launch_bounds__(kAttnPrefillRows * 32) attention_prefill_kernel(const AttnArgs a, int R) {
-  __shared__ __align__(128) unsigned char stages[2][kAttnStageBytes];   // two pages: K 8 KB | V 8 KB each
-  __shared__ __align__(8) uint64_t bars[2];
+// one half page (32 tokens: slots 0..7 of every lane) from a stage into the warp's running softmax
+__device__ __forceinline__ void prefill_fold_half(const unsigned char *stage, int half, int n_mine, int tg, int sub,
+                                                  const float (&qv)[8], float &m, float &l, float (&o)[8]) {
+  uint32_t vmask = 0u;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) vmask |= (32 * half + tg + 4 * i < n_mine) ? (1u << i) : 0u;
+  const unsigned char *base = stage + (size_t)(32 * half + tg) * (kHeadDim * 2) + 16 * sub;
+  uint4 kk[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) kk[i] = *reinterpret_cast<const uint4 *>(base + (size_t)(4 * i) * (kHeadDim * 2));
+  float sc[16];
+  const float pm = score_slots<8>(kk, qv, vmask, sc);
+  uint4 vv[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) vv[i] = *reinterpret_cast<const uint4 *>(base + kAttnHalfStage + (size_t)(4 * i) * (kHeadDim * 2));
+  accum_slots<8>(vv, sc, pm, vmask, m, l, o);
+}
+
+__global__ void __launch_bounds__(kAttnPrefillRows * 32, 3) attention_prefill_kernel(const AttnArgs a, int R) {
+  extern __shared__ __align__(128) unsigned char prefill_stages[];   // [stage][K 8 KB | V 8 KB]
+  __shared__ __align__(8) uint64_t bars[kAttnPrefillStages];
   __shared__ int seg_stream[kAttnPrefillRows], seg_i0[kAttnPrefillRows], seg_i1[kAttnPrefillRows], seg_last[kAttnPrefillRows];
   __shared__ int n_seg_s;
   const int h = blockIdx.y, r0 = blockIdx.z * kAttnPrefillRows;
@@ -566,7 +585,7 @@ __global__ void __launch_bounds__(kAttnPrefillRows * 32) attention_prefill_kerne
   const bool have_row = r < R;
   trace_mark(a.trace, a.trace_slot, 0);
   if (threadIdx.x == 0) {
-    mbar_init(bars, 1); mbar_init(bars + 1, 1);
+    for (int i = 0; i < kAttnPrefillStages; ++i) mbar_init(bars + i, 1);
     // runs of rows of one stream (the row table is final before the pass's first kernel starts)
     const int r_end = min(R, r0 + kAttnPrefillRows);
     int n = 0, i0 = r0;
@@ -591,57 +610,44 @@ __global__ void __launch_bounds__(kAttnPrefillRows * 32) attention_prefill_kerne
   for (int e = 0; e < 8; ++e) { o[e] = 0.f; qv[e] = 0.f; }
   if (have_row) load_q(qv, a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 8 * sub);
 
-  // page jobs in order: for each run, pages 0 .. last_pos/64.  Thread 0 requests job j+1 into the other
-  // stage before the warps fold job j.
-  auto issue = [&](int seg, int p, int slot) {
-    const int last_pos = seg_last[seg];
-    const int n_here = min(kPageTokens, last_pos + 1 - p * kPageTokens);
-    const uint32_t bytes = (uint32_t)n_here * kHeadDim * 2;
-    const int phys = a.page_table[(size_t)seg_stream[seg] * a.pps + p];
-    const uint16_t *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
-    mbar_expect_tx(bars + slot, 2 * bytes);
-    bulk_copy_g2s(stages[slot], K, bytes, bars + slot);
-    bulk_copy_g2s(stages[slot] + kAttnHalfStage, K + (size_t)a.H * kPageElems, bytes, bars + slot);
-  };
+  // page jobs in order: for each run, pages 0 .. last_pos/64.  Thread 0 keeps kAttnPrefillStages - 1
+  // jobs requested ahead of the one the warps fold.
   int iseg = 0, ip = 0;          // thread 0: the next job to request
-  if (threadIdx.x == 0 && n_seg > 0) {
-    issue(0, 0, 0);
-    ip = 1;
-    if (ip > seg_last[0] / kPageTokens) { iseg = 1; ip = 0; }
-  }
+  auto issue_next = [&](int slot) {
+    if (iseg >= n_seg) return;
+    const int last_pos = seg_last[iseg];
+    const int n_here = min(kPageTokens, last_pos + 1 - ip * kPageTokens);
+    const uint32_t bytes = (uint32_t)n_here * kHeadDim * 2;
+    const int phys = a.page_table[(size_t)seg_stream[iseg] * a.pps + ip];
+    const uint16_t *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kPageElems;
+    unsigned char *stage = prefill_stages + (size_t)slot * kAttnStageBytes;
+    mbar_expect_tx(bars + slot, 2 * bytes);
+    bulk_copy_g2s(stage, K, bytes, bars + slot);
+    bulk_copy_g2s(stage + kAttnHalfStage, K + (size_t)a.H * kPageElems, bytes, bars + slot);
+    if (++ip > last_pos / kPageTokens) { ++iseg; ip = 0; }
+  };
+  if (threadIdx.x == 0)
+    for (int i = 0; i < kAttnPrefillStages - 1; ++i) issue_next(i);
   bool dead = false;   // a copy did not arrive in time: stop folding, keep walking the barriers
   int j = 0;
   for (int seg = 0; seg < n_seg; ++seg) {
     const int n_pages = seg_last[seg] / kPageTokens + 1;
     const bool mine = have_row && r >= seg_i0[seg] && r < seg_i1[seg];
     for (int p = 0; p < n_pages; ++p, ++j) {
-      const int slot = j & 1;
-      if (threadIdx.x == 0 && iseg < n_seg) {   // job j+1 into the stage that job j-1 used (free since the barrier below)
-        issue(iseg, ip, slot ^ 1);
-        if (++ip > seg_last[iseg] / kPageTokens) { ++iseg; ip = 0; }
-      }
-      if (!dead && !mbar_wait_bounded(bars + slot, (uint32_t)(j >> 1) & 1u, kAttnWaitNs)) {
+      const int slot = j % kAttnPrefillStages;
+      // the stage job j-1 used is free since the barrier that ended its iteration
+      if (threadIdx.x == 0) issue_next((j + kAttnPrefillStages - 1) % kAttnPrefillStages);
+      const uint32_t parity = (uint32_t)(j / kAttnPrefillStages) & 1u;
+      if (!dead && !mbar_wait_bounded(bars + slot, parity, kAttnWaitNs)) {
         if (a.err) atomicExch(a.err, 1);
-        mbar_wait_bounded(bars + slot, (uint32_t)(j >> 1) & 1u, kAttnWaitNs);   // a last chance for the copy in flight
+        mbar_wait_bounded(bars + slot, parity, kAttnWaitNs);   // a last chance for the copy in flight
         dead = true;
       }
-      const unsigned char *stage = stages[slot];
+      const unsigned char *stage = prefill_stages + (size_t)slot * kAttnStageBytes;
       const int n_mine = mine ? min(kPageTokens, my_pos + 1 - p * kPageTokens) : 0;   // tokens of this page the row sees
       if (!dead && n_mine > 0) {   // warp-uniform
-        uint32_t vmask = 0u;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) vmask |= (tg + 4 * i < n_mine) ? (1u << i) : 0u;
-        uint4 kk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          kk[i] = *reinterpret_cast<const uint4 *>(stage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
-        float sc[16];
-        const float pm = score_slots<16>(kk, qv, vmask, sc);
-        uint4 vv[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          vv[i] = *reinterpret_cast<const uint4 *>(stage + kAttnHalfStage + (size_t)(tg + 4 * i) * (kHeadDim * 2) + 16 * sub);
-        accum_slots<16>(vv, sc, pm, vmask, m, l, o);
+        prefill_fold_half(stage, 0, n_mine, tg, sub, qv, m, l, o);
+        if (n_mine > 32) prefill_fold_half(stage, 1, n_mine, tg, sub, qv, m, l, o);
       }
       __syncthreads();   // every warp is done with this stage (all reads consumed): it may be refilled
       if (threadIdx.x == 0) fence_proxy_async_smem();
@@ -666,8 +672,13 @@ __global__ void __launch_bounds__(kAttnPrefillRows * 32) attention_prefill_kerne
 }
 
 inline cudaError_t launch_attention_prefill(const AttnArgs &a, int R, cudaStream_t st, bool pdl) {
+  static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
+  const size_t smem = (size_t)kAttnPrefillStages * kAttnStageBytes;
+  if (attr_once.first()) {
+    cudaFuncSetAttribute(attention_prefill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  }
   const int groups = (R + kAttnPrefillRows - 1) / kAttnPrefillRows;
-  return launch_kernel(attention_prefill_kernel, dim3(1, a.H, groups), dim3(kAttnPrefillRows * 32), 0, st, pdl, a, R);
+  return launch_kernel(attention_prefill_kernel, dim3(1, a.H, groups), dim3(kAttnPrefillRows * 32), smem, st, pdl, a, R);
 }
 
 // ------------------------------------------------------------------------------------------

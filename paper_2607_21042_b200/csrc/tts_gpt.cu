@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "linear.cuh"
 #include "attention.cuh"
+#include "attention_prefill.cuh"
 #include "gemm_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
@@ -79,6 +80,7 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
+  bool use_attn_mma = true;      // tensor-core attention in prefill passes (TTS_GPT_NO_ATTN_MMA=1 switches it off)
   bool use_attn_prefill = true;  // shared-page attention in prefill passes (TTS_GPT_NO_ATTN_PREFILL=1 switches it off)
   bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
   int attn_cluster_fill = 1;     // clusters grow until the grid covers the GPU this many times (TTS_GPT_ATTN_CLUSTER_FILL)
@@ -252,7 +254,9 @@ void trace_attach(tts_gpt *h, Args &a) {
 cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool pdl) {
   aa.err = h->dev_err;
   aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
-  // prefill passes: rows of one stream share their pages (one CTA per 8 rows and head)
+  // prefill passes: rows of one stream share their pages (one CTA per 16 rows and head on the tensor cores;
+  // the CUDA-core variant with 8 rows per CTA stays selectable)
+  if (!aa.old_pages_final && h->use_attn_mma && R >= kAttnPrefillRows) return launch_attention_prefill_mma(aa, R, st, pdl);
   if (!aa.old_pages_final && h->use_attn_prefill && R >= kAttnPrefillRows) return launch_attention_prefill(aa, R, st, pdl);
   const bool stream = h->attn_stream_min_pairs > 0 ? R * aa.H >= h->attn_stream_min_pairs : attention_use_stream(R, aa.H, h->n_sm);
   if (h->use_attn_stream && stream) return launch_attention_stream(aa, R, st, pdl);
@@ -593,6 +597,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   }
   const char *ntc = getenv("TTS_GPT_NO_TC");
   h->use_tc = !(ntc && ntc[0] == '1');
+  const char *nam = getenv("TTS_GPT_NO_ATTN_MMA");
+  h->use_attn_mma = !(nam && nam[0] == '1');
   const char *nap = getenv("TTS_GPT_NO_ATTN_PREFILL");
   h->use_attn_prefill = !(nap && nap[0] == '1');
   const char *nas = getenv("TTS_GPT_NO_ATTN_STREAM");
@@ -1054,14 +1060,14 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
                                      const int32_t *page_table, int32_t pages_per_stream,
                                      const int32_t *row_stream, const int32_t *row_pos, void *out,
                                      int32_t cluster_size, void *cuda_stream) {
-  if ((uintptr_t)q % 16 || (uintptr_t)kv_layer % 16 || (uintptr_t)out % 2 || (uintptr_t)page_table % 4 || (uintptr_t)row_stream % 4 ||
+  if ((uintptr_t)q % 16 || (uintptr_t)kv_layer % 16 || (uintptr_t)out % 16 || (uintptr_t)page_table % 4 || (uintptr_t)row_stream % 4 ||
       (uintptr_t)row_pos % 4)
-    return fail(nullptr, TTS_GPT_E_ARG, "attention: q and the KV pool must be 16-byte aligned, index arrays 4-byte");
+    return fail(nullptr, TTS_GPT_E_ARG, "attention: q, out and the KV pool must be 16-byte aligned, index arrays 4-byte");
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
-  if (cluster_size != -1 && cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
-    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be -1, 0, 1, 2, 4 or 8");
+  if (cluster_size != -2 && cluster_size != -1 && cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be -2, -1, 0, 1, 2, 4 or 8");
   AttnArgs a;
   memset(&a, 0, sizeof a);
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
@@ -1070,7 +1076,11 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
     CUDA_TRY(nullptr, launch_attention_stream(a, R, (cudaStream_t)cuda_stream, false));
     return TTS_GPT_OK;
   }
-  if (cluster_size == -1) {   // rows must be stream-major with ascending positions, as in a prefill pass
+  if (cluster_size == -2) {   // rows must be stream-major with ascending positions, as in a prefill pass
+    CUDA_TRY(nullptr, launch_attention_prefill_mma(a, R, (cudaStream_t)cuda_stream, false));
+    return TTS_GPT_OK;
+  }
+  if (cluster_size == -1) {   // same requirement on the rows
     CUDA_TRY(nullptr, launch_attention_prefill(a, R, (cudaStream_t)cuda_stream, false));
     return TTS_GPT_OK;
   }

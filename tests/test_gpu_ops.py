@@ -201,9 +201,10 @@ def test_attention_streaming_variant_rows_of_one_stream():
         assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5
 
 
-def test_attention_prefill_variant_mixed_streams():
+@pytest.mark.parametrize("variant", [-1, -2])
+def test_attention_prefill_variant_mixed_streams(variant):
     # rows as a prefill pass orders them: stream-major, positions ascending; runs of 5, 11, 1 and 40 rows so
-    # that CTAs of 8 rows hold one, two and three streams, starting inside a context
+    # that CTAs of 8 (variant -1) or 16 rows (variant -2) hold one, two and three streams, starting inside a context
     rng = np.random.default_rng(79)
     H = 3
     ctxs = [70, 200, 1, 333]
@@ -213,12 +214,14 @@ def test_attention_prefill_variant_mixed_streams():
     q = rng.standard_normal(size=(R, H * 64)).astype(np.float32)
     out = B.op_attention_cluster(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
                                  torch.tensor([s for s, _ in rows], dtype=torch.int32, device=DEV),
-                                 torch.tensor([p for _, p in rows], dtype=torch.int32, device=DEV), -1)
+                                 torch.tensor([p for _, p in rows], dtype=torch.int32, device=DEV), variant)
     torch.cuda.synchronize()
     got = bits_to_f64(out)
+    # variant -2 rounds Q and the softmax weights to bf16 on top of the bf16 output: one more unit of 2^-9 each
+    tol = 2.0 ** -8 if variant == -1 else 2.0 ** -7
     for r, (s_, p_) in enumerate(rows):
         ref = _attention_ref(q[r].astype(np.float64), Ks[s_][:p_ + 1], Vs[s_][:p_ + 1], H)
-        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, (r, s_, p_)
+        assert np.max(np.abs(got[r] - ref)) <= tol * np.abs(ref).max() + 1e-5, (r, s_, p_)
 
 
 @pytest.mark.parametrize("R,d", [(1, 256), (5, 1280), (128, 1280), (3, 2048), (2, 128)])
