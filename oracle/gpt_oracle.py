@@ -16,7 +16,8 @@ causal mask, untied LM head, hidden = output of the final LayerNorm).
 
 Pins (tests/test_oracle_pins.py): cached decode == full causal recompute; whole forward == a
 composition of torch float64 library routines; closed forms and invariants of LayerNorm, GELU,
-softmax/attention; exact int8/int4 round trips; sampling special cases and frequencies.
+softmax/attention; exact int8/int4 round trips; sampling special cases and frequencies; prefix
+assembly against a worked example with hand-made tables and its invariants.
 Parity with the paper's trained model itself is unpinned: the paper prints no value to pin to.
 
 Every function works on float64 numpy arrays.  bf16 inputs arrive as uint16 bit patterns and are
@@ -148,6 +149,21 @@ class OracleModel:
         """Input row of a generated token: its embedding plus the positional embedding of its
         index in the semantic-token range (Section II-C)."""
         return self.tok_emb[int(token)] + self.pos_emb[int(pos)]
+
+
+def assemble_prefix(model: OracleModel, cond_rows: np.ndarray, text_ids, text_shift: int,
+                    text_pos0: int) -> np.ndarray:
+    """Prefix rows of one utterance (Section II-C, the three input adaptations): the conditioning
+    embeddings come first and are used as given, with no positional embedding; text token j follows
+    as row ``text_ids[j] + text_shift`` of the merged embedding table (the text region of the table
+    starts after the semantic codes, so the shift is their number) plus row ``text_pos0 + j`` of the
+    position table (text tokens count positions in a range of their own).  Returns
+    [n_cond + n_text, d] float64."""
+    cond_rows = np.asarray(cond_rows, dtype=np.float64).reshape(-1, model.d)
+    rows = [cond_rows[i].copy() for i in range(cond_rows.shape[0])]
+    for j, t in enumerate(text_ids):
+        rows.append(model.tok_emb[int(t) + int(text_shift)] + model.pos_emb[int(text_pos0) + j])
+    return np.stack(rows) if rows else np.zeros((0, model.d))
 
 
 class OracleStream:

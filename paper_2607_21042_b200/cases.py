@@ -41,6 +41,11 @@ class GPTConfig:
     gelu_tanh: int = 1
     stop_token: int = -1
     ln_eps: float = 1e-5
+    emb_rows: int = 0       # rows of the merged embedding table (semantic codes, then text ids); 0 = vocab
+
+    @property
+    def n_emb_rows(self) -> int:
+        return self.emb_rows if self.emb_rows > 0 else self.vocab
 
     def as_dict(self):
         return asdict(self)
@@ -173,7 +178,7 @@ def make_weights(cfg: GPTConfig, seed: int = 0) -> dict:
     for lin in LINEARS:
         for suf in ("_w", "_s", "_b"):
             w[lin + suf] = []
-    w["tok_emb"] = _normal_bf16(rng, (v, d), 0.02)
+    w["tok_emb"] = _normal_bf16(rng, (cfg.n_emb_rows, d), 0.02)
     w["pos_emb"] = _normal_bf16(rng, (cfg.max_pos, d), 0.02)
 
     def put_linear(name):

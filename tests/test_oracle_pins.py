@@ -433,3 +433,62 @@ def test_topk_frequencies_chi_square():
     chi2 = ((counts - p * len(us)) ** 2 / (p * len(us))).sum()
     assert chi2 < 18.47         # 99.9 % quantile of chi-square with 4 degrees of freedom
     assert set(pos) == {4, 0, 1, 6, 2}
+
+
+def _table_model(d=4, emb_rows=12, max_pos=20):
+    # hand-made tables: element e of table row i is 10*i + e, of position row p is 1000*p + 100*e
+    m = O.OracleModel.__new__(O.OracleModel)
+    m.d = d
+    m.tok_emb = 10.0 * np.arange(emb_rows)[:, None] + np.arange(d)[None, :]
+    m.pos_emb = 1000.0 * np.arange(max_pos)[:, None] + 100.0 * np.arange(d)[None, :]
+    return m
+
+
+def test_assemble_prefix_worked_example():
+    # Section II-C: 2 conditioning rows as given, then text ids (3, 0, 1) in a table whose text region
+    # starts at row 7, text positions counted from row 5 of the position table
+    m = _table_model()
+    cond = np.array([[0.5, -1.0, 2.0, 4.0], [9.0, 8.0, 7.0, 6.0]])
+    got = O.assemble_prefix(m, cond, [3, 0, 1], text_shift=7, text_pos0=5)
+    want = np.array([
+        [0.5, -1.0, 2.0, 4.0],
+        [9.0, 8.0, 7.0, 6.0],
+        [5100.0, 5201.0, 5302.0, 5403.0],     # table row 10 (100..103) + position row 5 (5000, 5100, 5200, 5300)
+        [6070.0, 6171.0, 6272.0, 6373.0],     # table row 7 (70..73)    + position row 6
+        [7080.0, 7181.0, 7282.0, 7383.0],     # table row 8 (80..83)    + position row 7
+    ])
+    assert got.shape == (5, 4) and np.array_equal(got, want)
+
+
+def test_assemble_prefix_invariants():
+    m = _table_model()
+    rng = np.random.default_rng(3)
+    cond = rng.normal(size=(3, 4))
+    # no text: the conditioning rows come back untouched, whatever the position table holds
+    assert np.array_equal(O.assemble_prefix(m, cond, [], 7, 5), cond)
+    a = O.assemble_prefix(m, cond, [2, 4], 7, 5)
+    m2 = _table_model(); m2.pos_emb = m2.pos_emb * 0.0
+    b = O.assemble_prefix(m2, cond, [2, 4], 7, 5)
+    assert np.array_equal(a[:3], b[:3]) and np.array_equal(a[:3], cond)      # no positional term on conditioning rows
+    assert np.array_equal(a[3:] - b[3:], m.pos_emb[5:7])                     # text rows carry rows 5, 6 of the position table
+    assert np.array_equal(b[3:], m.tok_emb[[9, 11]])                         # and rows id + shift of the merged table
+    # the shift only relabels: ids + 1 with shift - 1 is the same prefix; so is a text range moved with the table
+    assert np.array_equal(O.assemble_prefix(m, cond, [3, 5], 6, 5), a)
+    m3 = _table_model(); m3.pos_emb = np.roll(m.pos_emb, 2, axis=0)
+    assert np.array_equal(O.assemble_prefix(m3, cond, [2, 4], 7, 7), a)
+
+
+def test_assembled_prefix_feeds_the_decoder_like_given_rows():
+    # a stream opened from (conditioning rows, text ids) equals one opened from the assembled rows
+    cfg = _toy_cfg(emb_rows=43)
+    w = C.make_weights(cfg, seed=4)
+    m = O.OracleModel(cfg, w)
+    rng = np.random.default_rng(5)
+    cond = rng.normal(size=(3, cfg.d_model)) * 0.02
+    shift = m.tok_emb.shape[0] - 6
+    rows = O.assemble_prefix(m, cond, [1, 5, 0, 2], shift, 9)
+    assert rows.shape == (7, cfg.d_model)
+    run = O.run_stream(m, rows, 3, pos0=2)
+    # position matters: the same ids counted from another text position give other logits
+    other = O.run_stream(m, O.assemble_prefix(m, cond, [1, 5, 0, 2], shift, 10), 3, pos0=2)
+    assert np.abs(run["logits"] - other["logits"]).max() > 1e-6
