@@ -68,11 +68,13 @@ typedef struct {
   int32_t gelu_tanh;     /* 1: tanh-form GELU (GPT-2), 0: erf form */
   int32_t stop_token;    /* -1: none */
   float ln_eps;          /* LayerNorm epsilon (inside the square root) */
+  int32_t emb_rows;      /* rows of tok_emb: the merged embedding table of Section II-C holds the semantic
+                            codes first and the text ids after them; 0 = vocab (no text region) */
 } tts_gpt_config_t;
 
 /* All DEVICE pointers, read only during tts_gpt_create (the library keeps its own re-laid-out
  * copy in the workspace; the caller may free these afterwards).  Per-layer entries are HOST arrays
- * of n_layer device pointers.  Shapes: tok_emb [vocab,d]; pos_emb [max_pos,d]; ln*_g/_b [d];
+ * of n_layer device pointers.  Shapes: tok_emb [emb_rows (vocab if 0),d]; pos_emb [max_pos,d]; ln*_g/_b [d];
  * head_w [vocab,d]; head_b [vocab] or NULL; qkv_w [3d,d] with rows ordered Q,K,V and head h owning
  * columns 64h..64h+63 of each; o_w [d,d]; fc1_w [d_ff,d]; fc2_w [d,d_ff]; *_b bf16 [N];
  * *_s bf16 scales (NULL array or NULL entries for bf16 weights). */
@@ -111,6 +113,25 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb,
                         const int32_t *prefix_len, const int32_t *pos0, int32_t top_k,
                         float temperature, const float *uniforms, int32_t *out_stream_ids,
                         int32_t *out_tokens, float *out_logits, void *out_hidden);
+
+/* Context phase with the prefix assembled on the device (Section II-C: conditioning embeddings
+ * retrieved in front of the sequence, one merged embedding table with text ids shifted past the
+ * semantic codes, position ids of the library's own making).  Stream i's prefix is
+ *   rows 0 .. n_cond[i]-1:  cond_emb[i] (DEVICE bf16 [n_cond[i], d]) used as given, no positional
+ *                           embedding;
+ *   then text token j:      tok_emb[text_ids[i][j] + text_shift] + pos_emb[text_pos0 + j]
+ * (bf16 rows widened and added in fp32).  cond_emb, text_ids: HOST arrays of n DEVICE pointers
+ * (cond_emb[i] 16-byte, text_ids[i] 4-byte aligned; either may be NULL when its count is 0);
+ * n_cond, n_text: HOST int32 [n], n_cond[i] + n_text[i] >= 1.  text_shift is the number of semantic
+ * codes in front of the text region; a shifted id outside 0..emb_rows-1 is clamped into that range
+ * (the ids live on the device and are not inspected by the host).  text_pos0 + n_text[i] must not
+ * exceed max_pos.  pos0 and everything after it: as for tts_gpt_prefill, whose errors also apply
+ * (with prefix_len = n_cond + n_text). */
+int32_t tts_gpt_prefill_tokens(tts_gpt_t *h, int32_t n, const void *const *cond_emb, const int32_t *n_cond,
+                               const int32_t *const *text_ids, const int32_t *n_text, int32_t text_shift,
+                               int32_t text_pos0, const int32_t *pos0, int32_t top_k, float temperature,
+                               const float *uniforms, int32_t *out_stream_ids, int32_t *out_tokens,
+                               float *out_logits, void *out_hidden);
 
 /* One incremental decode step (Sections I, II-C) for n distinct open streams (stream_ids: HOST).
  * Stream i consumes one input token — in_tokens[i] (DEVICE int32 [n]) or, if in_tokens is NULL,

@@ -21,7 +21,7 @@ OK, E_ARG, E_NO_PAGES, E_STREAM, E_CTX_OVERFLOW, E_CUDA, E_TIMEOUT, E_WORKSPACE,
     0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
-    "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_decode_step", "tts_gpt_decode_steps",
+    "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_prefill_tokens", "tts_gpt_decode_step", "tts_gpt_decode_steps",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
     "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace", "tts_gpt_debug_expire_wait",
@@ -42,7 +42,7 @@ class ConfigStruct(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layer", "d_model", "n_head", "head_dim", "d_ff", "vocab", "wfmt", "max_streams",
                  "max_context", "page_tokens", "n_pages", "max_pos", "gelu_tanh", "stop_token")] + \
-               [("ln_eps", C.c_float)]
+               [("ln_eps", C.c_float), ("emb_rows", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)
@@ -187,6 +187,28 @@ class TtsGpt:
         _check(self.lib.tts_gpt_prefill(self.handle, C.c_int32(n), ptrs, lens, p0, C.c_int32(top_k),
                                         C.c_float(temperature), _ptr(uniforms), ids, _ptr(out_tokens),
                                         _ptr(out_logits), _ptr(out_hidden)), self.handle)
+        return list(ids), out_tokens
+
+    def prefill_tokens(self, cond, text_ids, text_shift, text_pos0, top_k=0, temperature=1.0, uniforms=None,
+                       pos0=None, out_tokens=None, out_logits=None, out_hidden=None):
+        """Prefixes assembled on the device: cond[i] a device tensor of bf16 bits [n_cond_i, d] (or None),
+        text_ids[i] a device int32 tensor [n_text_i] (or None).  Returns (stream_ids list, out_tokens tensor)."""
+        n = len(cond)
+        self.wait_for_caller()
+        self._live_prefixes = [None if p is None else p.contiguous() for p in cond]
+        self._live_text = [None if t is None else t.contiguous() for t in text_ids]
+        cptrs = (C.c_void_p * n)(*[None if p is None else p.data_ptr() for p in self._live_prefixes])
+        tptrs = (C.c_void_p * n)(*[None if t is None else t.data_ptr() for t in self._live_text])
+        ncond = _i32_array([0 if p is None else p.shape[0] for p in self._live_prefixes])
+        ntext = _i32_array([0 if t is None else t.shape[0] for t in self._live_text])
+        ids = (C.c_int32 * n)()
+        if out_tokens is None:
+            out_tokens = torch.empty(n, dtype=torch.int32, device=self.device)
+        p0 = _i32_array(pos0) if pos0 is not None else None
+        _check(self.lib.tts_gpt_prefill_tokens(self.handle, C.c_int32(n), cptrs, ncond, tptrs, ntext,
+                                               C.c_int32(text_shift), C.c_int32(text_pos0), p0, C.c_int32(top_k),
+                                               C.c_float(temperature), _ptr(uniforms), ids, _ptr(out_tokens),
+                                               _ptr(out_logits), _ptr(out_hidden)), self.handle)
         return list(ids), out_tokens
 
     def decode_step(self, stream_ids, out_tokens, in_tokens=None, top_k=0, temperature=1.0,

@@ -19,6 +19,8 @@ struct PageState {
   int *pos_next;    // [max_streams] pos_emb index of the next generated token
   int *stop_flag;   // [max_streams]
   const uint16_t **stream_emb;  // [max_streams] prefix base pointer during prefill
+  const int **stream_text;      // [max_streams] text ids behind the given rows (null: none)
+  int *stream_ncond;            // [max_streams] rows of the prefix that are given embeddings
   int pps, n_pages, max_streams;
 };
 
@@ -109,15 +111,36 @@ __global__ void __launch_bounds__(kMaxRows) prefill_open_kernel(const PrefillPar
     ps.pos_next[s] = p.pos0[i];
     ps.stop_flag[s] = 0;
     ps.stream_emb[s] = p.emb[i];
+    ps.stream_text[s] = nullptr;            // the whole prefix is given as embeddings unless
+    ps.stream_ncond[s] = p.prefix_len[i];   // prefill_text_kernel says otherwise
   }
   __syncthreads();
   if (i == 0) *ps.free_top = top - total;
+}
+
+// Prefixes assembled on the device (Section II-C): the first n_cond rows of a stream's prefix are the
+// given conditioning embeddings, the rest are text tokens looked up in the merged embedding table.
+struct TextParams {
+  int n;
+  int stream_ids[kMaxRows];
+  int n_cond[kMaxRows];
+  const int *text[kMaxRows];
+};
+
+__global__ void __launch_bounds__(kMaxRows) prefill_text_kernel(const TextParams p, PageState ps) {
+  const int i = threadIdx.x;
+  if (i < p.n) {
+    const int s = p.stream_ids[i];
+    ps.stream_text[s] = p.text[i];
+    ps.stream_ncond[s] = p.n_cond[i];
+  }
 }
 
 struct PassParams {
   int n_rows, n_out;
   short row_stream[kMaxRows], row_pos[kMaxRows], out_rows[kMaxRows], out_slot[kMaxRows];
   StepIO io;
+  int text_shift, text_pos0, emb_rows;   // text rows: table row = id + text_shift (clamped), position row = text_pos0 + j
 };
 
 // Row table of one prefill pass: up to 128 (stream, position) rows taken from the prefixes.
@@ -127,9 +150,17 @@ __global__ void __launch_bounds__(kMaxRows) prefill_pass_kernel(const PassParams
     const int s = p.row_stream[i], t = p.row_pos[i];
     rt.row_stream[i] = s;
     rt.row_pos[i] = t;
-    rt.row_token[i] = -1;
-    rt.row_posidx[i] = 0;
-    rt.row_emb[i] = ps.stream_emb[s] + (size_t)t * d;
+    const int nc = ps.stream_ncond[s];
+    if (t < nc) {     // a given embedding row, used as it is
+      rt.row_token[i] = -1;
+      rt.row_posidx[i] = 0;
+      rt.row_emb[i] = ps.stream_emb[s] + (size_t)t * d;
+    } else {          // text token j of the stream
+      const int j = t - nc;
+      rt.row_token[i] = min(max(ps.stream_text[s][j] + p.text_shift, 0), p.emb_rows - 1);
+      rt.row_posidx[i] = p.text_pos0 + j;
+      rt.row_emb[i] = nullptr;
+    }
   }
   if (i < p.n_out) { rt.out_rows[i] = p.out_rows[i]; rt.out_slot[i] = p.out_slot[i]; }
   if (i == 0) *io = p.io;

@@ -126,8 +126,12 @@ int check_config(const tts_gpt_config_t *c) {
     return fail(nullptr, TTS_GPT_E_ARG, "max_context must be a multiple of 64 in 64..2048");
   if (c->n_pages < 1 || c->max_pos < 1) return fail(nullptr, TTS_GPT_E_ARG, "n_pages and max_pos must be positive");
   if (!(c->ln_eps > 0.f)) return fail(nullptr, TTS_GPT_E_ARG, "ln_eps must be positive");
+  if (c->emb_rows != 0 && c->emb_rows < c->vocab) return fail(nullptr, TTS_GPT_E_ARG, "emb_rows must be 0 or at least vocab");
   return TTS_GPT_OK;
 }
+
+// rows of the embedding table: the semantic codes and specials the head predicts, then the text region if any
+inline int emb_rows_of(const tts_gpt_config_t &c) { return c.emb_rows > 0 ? c.emb_rows : c.vocab; }
 
 // Walks the workspace; with base == nullptr only measures.
 struct Carver {
@@ -156,7 +160,7 @@ size_t carve(tts_gpt *h, void *base) {
   const int d = c.d_model, F = c.d_ff, V = c.vocab, S = c.max_streams;
   h->pps = c.max_context / 64;
   Carver cv(base);
-  h->tok_emb = cv.take<uint16_t>((size_t)V * d);
+  h->tok_emb = cv.take<uint16_t>((size_t)emb_rows_of(c) * d);
   h->pos_emb = cv.take<uint16_t>((size_t)c.max_pos * d);
   h->lnf_g = cv.take<uint16_t>(d);
   h->lnf_b = cv.take<uint16_t>(d);
@@ -182,6 +186,8 @@ size_t carve(tts_gpt *h, void *base) {
   ps.pos_next = cv.take<int>(S);
   ps.stop_flag = cv.take<int>(S);
   ps.stream_emb = cv.take<const uint16_t *>(S);
+  ps.stream_text = cv.take<const int *>(S);
+  ps.stream_ncond = cv.take<int>(S);
   RowTable &rt = h->rt;
   rt.row_stream = cv.take<int>(kMaxRows);
   rt.row_pos = cv.take<int>(kMaxRows);
@@ -472,7 +478,7 @@ int run_head(tts_gpt *h, int n_out, int R) {
 
 int run_embed(tts_gpt *h, int R) {
   const tts_gpt_config_t &c = h->cfg;
-  embed_kernel<<<R, 256, 0, h->stream>>>(h->rt, h->tok_emb, h->pos_emb, c.d_model, c.vocab, c.max_pos, h->x);
+  embed_kernel<<<R, 256, 0, h->stream>>>(h->rt, h->tok_emb, h->pos_emb, c.d_model, emb_rows_of(c), c.max_pos, h->x);
   CUDA_TRY(h, cudaGetLastError());
   h->launches += 1;
   return TTS_GPT_OK;
@@ -527,7 +533,7 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   const tts_gpt_config_t &c = h->cfg;
   const int d = c.d_model;
 #define TRY_(expr) do { rc = (expr); if (rc) { g_last_error = h->err; delete h; return rc; } } while (0)
-  TRY_(copy_bf16(h, h->tok_emb, w->tok_emb, (size_t)c.vocab * d, "tok_emb"));
+  TRY_(copy_bf16(h, h->tok_emb, w->tok_emb, (size_t)emb_rows_of(c) * d, "tok_emb"));
   TRY_(copy_bf16(h, h->pos_emb, w->pos_emb, (size_t)c.max_pos * d, "pos_emb"));
   TRY_(copy_bf16(h, h->lnf_g, w->lnf_g, d, "lnf_g"));
   TRY_(copy_bf16(h, h->lnf_b, w->lnf_b, d, "lnf_b"));
@@ -616,24 +622,35 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   return TTS_GPT_OK;
 }
 
-int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, const int32_t *prefix_len,
+// Both prefill entries.  text == nullptr: every prefix row is a given embedding (n_cond is then the
+// prefix length); otherwise stream i has n_cond[i] given rows followed by n_text[i] text tokens.
+static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const int32_t *n_cond,
+                        const int32_t *const *text, const int32_t *n_text, int32_t text_shift, int32_t text_pos0,
                         const int32_t *pos0, int32_t top_k, float temperature, const float *uniforms,
                         int32_t *out_stream_ids, int32_t *out_tokens, float *out_logits, void *out_hidden) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   const tts_gpt_config_t &c = h->cfg;
-  if (n < 1 || n > c.max_streams || !prefix_emb || !prefix_len || !out_stream_ids || !out_tokens)
+  if (n < 1 || n > c.max_streams || !emb || !n_cond || !out_stream_ids || !out_tokens || (text && !n_text))
     return fail(h, TTS_GPT_E_ARG, "prefill: bad n or null argument");
   int rc = check_top_k(h, top_k, temperature, uniforms);
   if (rc) return rc;
   rc = check_io_alignment(h, nullptr, uniforms, out_tokens, out_logits, out_hidden);
   if (rc) return rc;
+  if (text && (text_pos0 < 0 || text_pos0 >= c.max_pos)) return fail(h, TTS_GPT_E_ARG, "prefill: text_pos0 out of range");
   int pages = 0;
+  int plen[kMaxRows];
   for (int i = 0; i < n; ++i) {
-    if (prefix_len[i] < 1 || !prefix_emb[i]) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has an empty prefix", i);
-    if ((uintptr_t)prefix_emb[i] % 16) return fail(h, TTS_GPT_E_ARG, "prefill: prefix %d is not 16-byte aligned", i);
-    if (prefix_len[i] > c.max_context) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "prefill: prefix %d exceeds max_context %d", prefix_len[i], c.max_context);
+    const int nc = n_cond[i], nt = text ? n_text[i] : 0;
+    if (nc < 0 || nt < 0 || nc + nt < 1) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has an empty prefix", i);
+    if (nc > 0 && !emb[i]) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has no embedding rows", i);
+    if (nt > 0 && !text[i]) return fail(h, TTS_GPT_E_ARG, "prefill: stream %d has no text ids", i);
+    if (nc > 0 && (uintptr_t)emb[i] % 16) return fail(h, TTS_GPT_E_ARG, "prefill: prefix %d is not 16-byte aligned", i);
+    if (nt > 0 && (uintptr_t)text[i] % 4) return fail(h, TTS_GPT_E_ARG, "prefill: text ids %d are not 4-byte aligned", i);
+    if (nt > 0 && text_pos0 + nt > c.max_pos) return fail(h, TTS_GPT_E_ARG, "prefill: text of stream %d runs past max_pos %d", i, c.max_pos);
+    plen[i] = nc + nt;
+    if (plen[i] > c.max_context) return fail(h, TTS_GPT_E_CTX_OVERFLOW, "prefill: prefix %d exceeds max_context %d", plen[i], c.max_context);
     if (pos0 && (pos0[i] < 0 || pos0[i] >= c.max_pos)) return fail(h, TTS_GPT_E_ARG, "prefill: pos0 out of range");
-    pages += (prefix_len[i] + 63) / 64;
+    pages += (plen[i] + 63) / 64;
   }
   PrefillParams pp;
   memset(&pp, 0, sizeof pp);
@@ -644,16 +661,25 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
   if (found < n) return fail(h, TTS_GPT_E_STREAM, "prefill: %d free stream slots, %d needed", found, n);
   if (pages > h->n_free) return fail(h, TTS_GPT_E_NO_PAGES, "prefill: %d pages needed, %d free", pages, h->n_free);
   for (int i = 0; i < n; ++i) {
-    pp.prefix_len[i] = prefix_len[i];
+    pp.prefix_len[i] = plen[i];
     pp.pos0[i] = pos0 ? pos0[i] : 0;
-    pp.emb[i] = (const uint16_t *)prefix_emb[i];
+    pp.emb[i] = (const uint16_t *)emb[i];
   }
   prefill_open_kernel<<<1, kMaxRows, 0, h->stream>>>(pp, h->ps);
   CUDA_TRY(h, cudaGetLastError());
   h->launches += 1;
+  if (text) {
+    TextParams tp;
+    memset(&tp, 0, sizeof tp);
+    tp.n = n;
+    for (int i = 0; i < n; ++i) { tp.stream_ids[i] = pp.stream_ids[i]; tp.n_cond[i] = n_cond[i]; tp.text[i] = text[i]; }
+    prefill_text_kernel<<<1, kMaxRows, 0, h->stream>>>(tp, h->ps);
+    CUDA_TRY(h, cudaGetLastError());
+    h->launches += 1;
+  }
   for (int i = 0; i < n; ++i) {
     const int s = pp.stream_ids[i];
-    h->open[s] = 1; h->ctx[s] = prefix_len[i]; h->pos_next[s] = pp.pos0[i];
+    h->open[s] = 1; h->ctx[s] = plen[i]; h->pos_next[s] = pp.pos0[i];
     out_stream_ids[i] = s;
   }
   h->n_free -= pages;
@@ -665,6 +691,7 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
   PassParams ps;
   memset(&ps, 0, sizeof ps);
   ps.io = io;
+  ps.text_shift = text_shift; ps.text_pos0 = text_pos0; ps.emb_rows = emb_rows_of(c);
   auto flush = [&]() -> int {
     if (ps.n_rows == 0) return TTS_GPT_OK;
     ps.io.n_out = ps.n_out;
@@ -680,11 +707,11 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     return r;
   };
   for (int i = 0; i < n; ++i) {
-    for (int t = 0; t < prefix_len[i]; ++t) {
+    for (int t = 0; t < plen[i]; ++t) {
       const int r = ps.n_rows++;
       ps.row_stream[r] = (short)pp.stream_ids[i];
       ps.row_pos[r] = (short)t;
-      if (t == prefix_len[i] - 1) {
+      if (t == plen[i] - 1) {
         ps.out_rows[ps.n_out] = (short)r;
         ps.out_slot[ps.n_out] = (short)i;
         ++ps.n_out;
@@ -693,6 +720,23 @@ int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, 
     }
   }
   return flush();
+}
+
+int32_t tts_gpt_prefill(tts_gpt_t *h, int32_t n, const void *const *prefix_emb, const int32_t *prefix_len,
+                        const int32_t *pos0, int32_t top_k, float temperature, const float *uniforms,
+                        int32_t *out_stream_ids, int32_t *out_tokens, float *out_logits, void *out_hidden) {
+  return prefill_impl(h, n, prefix_emb, prefix_len, nullptr, nullptr, 0, 0, pos0, top_k, temperature, uniforms,
+                      out_stream_ids, out_tokens, out_logits, out_hidden);
+}
+
+int32_t tts_gpt_prefill_tokens(tts_gpt_t *h, int32_t n, const void *const *cond_emb, const int32_t *n_cond,
+                               const int32_t *const *text_ids, const int32_t *n_text, int32_t text_shift,
+                               int32_t text_pos0, const int32_t *pos0, int32_t top_k, float temperature,
+                               const float *uniforms, int32_t *out_stream_ids, int32_t *out_tokens,
+                               float *out_logits, void *out_hidden) {
+  if (!text_ids || !n_text) return fail(h, TTS_GPT_E_ARG, "prefill_tokens: null text argument");
+  return prefill_impl(h, n, cond_emb, n_cond, text_ids, n_text, text_shift, text_pos0, pos0, top_k, temperature,
+                      uniforms, out_stream_ids, out_tokens, out_logits, out_hidden);
 }
 
 int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, const int32_t *in_tokens,

@@ -365,3 +365,63 @@ def test_erf_gelu_variant():
     ref, _ = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
     assert_logits_close(logits, ref, "erf gelu")
     eng.destroy()
+
+
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC])
+def test_prefill_tokens_assembles_the_prefix_on_the_device(wfmt):
+    """Section II-C: conditioning rows as given, text ids shifted into the merged table, text positions
+    in their own range, generated tokens in another.  Four streams: conditioning + text across a page
+    boundary (34 + 75 rows), conditioning + short text, text only, conditioning only."""
+    n_text_vocab = 50
+    cfg = _tiny(wfmt, emb_rows=1024 + n_text_vocab, max_pos=160)
+    w = C.make_weights(cfg, seed=3)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    rng = np.random.default_rng(17)
+    n_cond = [34, 34, 0, 5]
+    n_text = [75, 9, 40, 0]
+    conds = [C.make_prefixes(cfg, [max(nc, 1)], seed=20 + i)[0][:nc] for i, nc in enumerate(n_cond)]
+    texts = [rng.integers(0, n_text_vocab, size=nt).astype(np.int32) for nt in n_text]
+    shift, text_pos0, pos0 = cfg.vocab, 80, [0, 3, 5, 0]
+    S, n_dec = 4, 6
+    V = cfg.vocab
+    toks = torch.zeros((n_dec + 1, S), dtype=torch.int32, device=DEV)
+    logits = torch.zeros((n_dec + 1, S, V), dtype=torch.float32, device=DEV)
+    cond_dev = [bits_dev(c) if len(c) else None for c in conds]
+    text_dev = [torch.from_numpy(t).to(DEV) if len(t) else None for t in texts]
+    torch.cuda.synchronize()
+    ids, _ = eng.prefill_tokens(cond_dev, text_dev, shift, text_pos0, pos0=pos0, out_tokens=toks[0], out_logits=logits[0])
+    for k in range(1, n_dec + 1):
+        eng.decode_step(ids, toks[k], out_logits=logits[k])
+    eng.sync()
+    toks = toks.cpu().numpy(); logits = logits.cpu().numpy()
+    for i in range(S):
+        assert eng.stream_context(ids[i]) == n_cond[i] + n_text[i] + n_dec
+        rows = O.assemble_prefix(model, O.bf16_to_f64(conds[i]).reshape(-1, cfg.d_model), texts[i], shift, text_pos0)
+        ref, _ = O.replay_full(model, rows, toks[:-1, i], pos0=pos0[i])
+        assert_logits_close(logits[:, i], ref, "stream %d" % i)
+        check_tokens(toks[:, i], ref, 0, 1.0, None, "stream %d" % i)
+    # the text range matters: the same ids counted from another position give other first logits
+    other = O.assemble_prefix(model, O.bf16_to_f64(conds[1]).reshape(-1, cfg.d_model), texts[1], shift, text_pos0 + 1)
+    ref_other, _ = O.replay_full(model, other, toks[:0, 1], pos0=pos0[1])
+    assert np.max(np.abs(ref_other[0] - logits[0, 1])) > 1e-3
+    # errors leave the engine as it was: text running past the position table, and a missing id array
+    for i in ids:
+        eng.release_stream(i)
+    before = eng.stats()
+    with pytest.raises(B.TtsGptError) as e:
+        eng.prefill_tokens([cond_dev[3]], [torch.zeros(100, dtype=torch.int32, device=DEV)], shift, 100)
+    assert e.value.code == B.E_ARG
+    with pytest.raises(B.TtsGptError) as e:
+        eng.prefill_tokens([None], [None], shift, text_pos0)
+    assert e.value.code == B.E_ARG
+    assert eng.stats() == before
+    # ids outside the table are clamped into it, not followed out of bounds
+    wild = torch.tensor([-5000, 10 ** 6, 3], dtype=torch.int32, device=DEV)
+    lg = torch.zeros((1, V), dtype=torch.float32, device=DEV)
+    ids2, _ = eng.prefill_tokens([None], [wild], shift, text_pos0, out_logits=lg)
+    eng.sync()
+    rows = O.assemble_prefix(model, np.zeros((0, cfg.d_model)), [-shift, n_text_vocab - 1, 3], shift, text_pos0)
+    ref, _ = O.replay_full(model, rows, toks[:0, 0])
+    assert_logits_close(lg.cpu().numpy(), ref, "clamped ids")
+    eng.destroy()
