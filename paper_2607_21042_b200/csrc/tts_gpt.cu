@@ -16,6 +16,7 @@
 #include "linear.cuh"
 #include "attention.cuh"
 #include "attention_prefill.cuh"
+#include "qkv_attention.cuh"
 #include "gemm_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
@@ -80,6 +81,8 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (TTS_GPT_NO_TC=1 switches it off)
+  bool use_qkv_attn = false;     // one-row steps: LayerNorm + QKV + attention in one kernel; measured no faster than the
+                                 // two kernels it replaces, so it is off unless TTS_GPT_QKV_ATTN=1
   bool use_attn_mma = true;      // tensor-core attention in prefill passes (TTS_GPT_NO_ATTN_MMA=1 switches it off)
   bool use_attn_prefill = true;  // shared-page attention in prefill passes (TTS_GPT_NO_ATTN_PREFILL=1 switches it off)
   bool use_attn_stream = true;   // streaming attention for large batches (TTS_GPT_NO_ATTN_STREAM=1 switches it off)
@@ -385,33 +388,50 @@ int run_layers(tts_gpt *h, int R, bool decode) {
   const int fc2_ks = (!fuse_ln && h->use_fc2_ksplit && (c.d_ff / k_per_tile(c.wfmt)) % kSmallKSplit == 0 &&
                       (size_t)kSmallKSplit * kMaxRows * d <= h->partials_floats) ? kSmallKSplit : 1;
   h->pending_parts = 0;
+  const bool fuse_qa = decode && fuse_ln && h->use_qkv_attn &&
+                       can_fuse_qkv_attention(c.wfmt, R, d, c.n_head, h->n_sm, h->attn_cluster_fill);
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
-    LinearArgs qa = linear_args(h, L.qkv, h->a, R, EPI_QKV);
-    if (fuse_ln) {
-      qa.ln_x = h->x; qa.ln_g = L.ln1_g; qa.ln_b = L.ln1_b; qa.ln_eps = c.ln_eps;
-    } else if (fc2_ks > 1) {
-      int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : fc2_ks, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
-                            nullptr, h->a, nullptr, nullptr, nullptr, 1);
-      if (rc) return rc;
+    if (fuse_qa) {
+      // one row: LayerNorm, QKV and attention in one kernel (a cluster of 8 CTAs per head)
+      QkvAttnArgs fa;
+      memset(&fa, 0, sizeof fa);
+      fa.w = L.qkv.w; fa.scales = L.qkv.s; fa.bias = L.qkv.bias; fa.x = h->x; fa.ln_g = L.ln1_g; fa.ln_b = L.ln1_b;
+      fa.ln_eps = c.ln_eps; fa.d = d;
+      fa.at.kv_layer = kvl; fa.at.page_table = h->ps.page_table; fa.at.row_stream = h->rt.row_stream;
+      fa.at.row_pos = h->rt.row_pos; fa.at.out = h->o; fa.at.H = c.n_head; fa.at.pps = h->pps; fa.at.old_pages_final = 1;
+      fa.at.err = h->dev_err;
+      trace_attach(h, fa.at);
+      if (h->trace) h->trace_next++;   // keeps the slot numbering of the two kernels it replaces
+      CUDA_TRY(h, launch_qkv_attention(c.wfmt, fa, R, st, pdl));
+      h->launches -= 1;                // 4 kernels in this layer, not 5
     } else {
-      CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(R), dim3(kLnThreads), 0, st, pdl, (const float *)h->x, d,
-                                (const uint16_t *)L.ln1_g, (const uint16_t *)L.ln1_b, c.ln_eps, h->a,
-                                (const int *)nullptr, (const int *)nullptr, (const StepIO *)nullptr));
-      h->launches += 1;
+      LinearArgs qa = linear_args(h, L.qkv, h->a, R, EPI_QKV);
+      if (fuse_ln) {
+        qa.ln_x = h->x; qa.ln_g = L.ln1_g; qa.ln_b = L.ln1_b; qa.ln_eps = c.ln_eps;
+      } else if (fc2_ks > 1) {
+        int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : fc2_ks, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
+                              nullptr, h->a, nullptr, nullptr, nullptr, 1);
+        if (rc) return rc;
+      } else {
+        CUDA_TRY(h, launch_kernel(layernorm_kernel, dim3(R), dim3(kLnThreads), 0, st, pdl, (const float *)h->x, d,
+                                  (const uint16_t *)L.ln1_g, (const uint16_t *)L.ln1_b, c.ln_eps, h->a,
+                                  (const int *)nullptr, (const int *)nullptr, (const StepIO *)nullptr));
+        h->launches += 1;
+      }
+      qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
+      qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+      trace_attach(h, qa);
+      CUDA_TRY(h, launch_linear(c.wfmt, qa, st, pdl, 2 * h->n_sm));
+      AttnArgs aa;
+      memset(&aa, 0, sizeof aa);
+      aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
+      aa.row_pos = h->rt.row_pos; aa.out = h->o; aa.partials = h->attn_partials; aa.tickets = h->attn_tickets;
+      aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
+      trace_attach(h, aa);
+      CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     }
-    qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
-    qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
-    trace_attach(h, qa);
-    CUDA_TRY(h, launch_linear(c.wfmt, qa, st, pdl, 2 * h->n_sm));
-    AttnArgs aa;
-    memset(&aa, 0, sizeof aa);
-    aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
-    aa.row_pos = h->rt.row_pos; aa.out = h->o; aa.partials = h->attn_partials; aa.tickets = h->attn_tickets;
-    aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
-    trace_attach(h, aa);
-    CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     LinearArgs oa = linear_args(h, L.o, h->o, R, EPI_RESID);
     oa.out_f32 = h->x; oa.out_stride = d;
     trace_attach(h, oa);
@@ -603,6 +623,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   }
   const char *ntc = getenv("TTS_GPT_NO_TC");
   h->use_tc = !(ntc && ntc[0] == '1');
+  const char *qa = getenv("TTS_GPT_QKV_ATTN");
+  h->use_qkv_attn = qa && qa[0] == '1';
   const char *nam = getenv("TTS_GPT_NO_ATTN_MMA");
   h->use_attn_mma = !(nam && nam[0] == '1');
   const char *nap = getenv("TTS_GPT_NO_ATTN_PREFILL");

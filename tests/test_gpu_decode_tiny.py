@@ -425,3 +425,30 @@ def test_prefill_tokens_assembles_the_prefix_on_the_device(wfmt):
     ref, _ = O.replay_full(model, rows, toks[:0, 0])
     assert_logits_close(lg.cpu().numpy(), ref, "clamped ids")
     eng.destroy()
+
+
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
+def test_fused_qkv_attention_kernel_matches_oracle(tiny_models, wfmt, monkeypatch):
+    """The optional one-kernel LayerNorm + QKV + attention of one-row steps (switched on by an environment
+    variable read at engine creation) against the oracle, across a page boundary, and against the default
+    schedule of the same engine build."""
+    cfg, w, model = tiny_models[wfmt]
+    prefix = C.make_prefixes(cfg, [60], seed=31)[0]
+    n = 12
+    monkeypatch.setenv("TTS_GPT_QKV_ATTN", "1")
+    eng = B.TtsGpt(cfg, w, DEV)
+    l0 = eng.kernel_launches()
+    toks, logits, hidden, sid = gpu_run_stream(eng, bits_dev(prefix), n, want_hidden=True)
+    fused_launches = eng.kernel_launches() - l0
+    ref_logits, ref_hidden = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
+    assert_logits_close(logits, ref_logits, "fused")
+    check_tokens(toks, ref_logits, 0, 1.0, None, "fused")
+    eng.destroy()
+    monkeypatch.delenv("TTS_GPT_QKV_ATTN")
+    eng = B.TtsGpt(cfg, w, DEV)
+    l0 = eng.kernel_launches()
+    toks2, logits2, _, _ = gpu_run_stream(eng, bits_dev(prefix), n)
+    plain_launches = eng.kernel_launches() - l0
+    eng.destroy()
+    assert fused_launches == plain_launches - n * cfg.n_layer      # one kernel fewer per layer and step
+    assert_same_up_to_ties(toks, logits, toks2, logits2, "fused vs default")
