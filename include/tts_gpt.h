@@ -162,6 +162,18 @@ int32_t tts_gpt_decode_steps(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
                              float temperature, const float *uniforms, int32_t *out_tokens,
                              float *out_logits, void *out_hidden);
 
+/* tts_gpt_decode_step with HOST buffers: copies in_tokens (HOST int32 [n], or NULL as above) and
+ * uniforms (HOST fp32 [n], needed when top_k > 1) to staging arrays inside the workspace, enqueues
+ * the step, copies out_tokens (HOST int32 [n]), out_logits (HOST fp32 [n,vocab] or NULL) and
+ * out_hidden (HOST bf16 [n,d] or NULL) back and waits for the engine's stream before it returns, so
+ * the results are valid on return.  Page-locked host buffers make the copies asynchronous to the
+ * host; pageable ones work.  Errors: those of tts_gpt_decode_step (nothing is enqueued but the
+ * staging copies) and those of tts_gpt_sync. */
+int32_t tts_gpt_decode_step_host(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
+                                 const int32_t *in_tokens, int32_t top_k, float temperature,
+                                 const float *uniforms, int32_t *out_tokens, float *out_logits,
+                                 void *out_hidden);
+
 /* Close a stream and return its pages to the pool.  E_STREAM if the id is not open. */
 int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t stream_id);
 

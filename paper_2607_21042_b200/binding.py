@@ -21,7 +21,7 @@ OK, E_ARG, E_NO_PAGES, E_STREAM, E_CTX_OVERFLOW, E_CUDA, E_TIMEOUT, E_WORKSPACE,
     0, -1, -2, -3, -4, -5, -6, -7, -8
 
 EXPORTS = [
-    "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_prefill_tokens", "tts_gpt_decode_step", "tts_gpt_decode_steps",
+    "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_prefill_tokens", "tts_gpt_decode_step", "tts_gpt_decode_step_host", "tts_gpt_decode_steps",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
     "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace", "tts_gpt_debug_expire_wait",
@@ -219,6 +219,16 @@ class TtsGpt:
                                                    C.c_int32(top_k), C.c_float(temperature),
                                                    _ptr(uniforms), _ptr(out_tokens), _ptr(out_logits),
                                                    _ptr(out_hidden)), self.handle)
+
+    def decode_step_host(self, stream_ids, out_tokens, in_tokens=None, top_k=0, temperature=1.0,
+                         uniforms=None, out_logits=None, out_hidden=None):
+        """One step with HOST tensors (ideally pinned): inputs are copied in, results are valid on return."""
+        n = len(stream_ids)
+        ids = stream_ids if isinstance(stream_ids, C.Array) else _i32_array(stream_ids)
+        return _check(self.lib.tts_gpt_decode_step_host(self.handle, C.c_int32(n), ids, _ptr(in_tokens),
+                                                        C.c_int32(top_k), C.c_float(temperature),
+                                                        _ptr(uniforms), _ptr(out_tokens), _ptr(out_logits),
+                                                        _ptr(out_hidden)), self.handle)
 
     def decode_steps(self, stream_ids, n_steps, out_tokens, in_tokens=None, top_k=0, temperature=1.0,
                      uniforms=None, out_logits=None, out_hidden=None):

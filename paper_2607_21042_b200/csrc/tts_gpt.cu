@@ -60,6 +60,9 @@ struct tts_gpt {
   StepIO *io;
   // activations
   float *x, *q, *logits;
+  int *st_in, *st_tok;          // staging of the host-buffer entry: input tokens, sampled tokens
+  float *st_uni, *st_log;       // uniforms, logits [kMaxRows][vocab]
+  uint16_t *st_hid;             // hidden rows [kMaxRows][d]
   uint16_t *a, *o, *hbuf, *hf;
   // tensor-core path (more than 16 rows, bf16 weights): activation images and k-split partial sums
   void *a_img = nullptr, *o_img = nullptr, *h_img = nullptr, *hf_img = nullptr;
@@ -204,6 +207,11 @@ size_t carve(tts_gpt *h, void *base) {
   h->x = cv.take<float>((size_t)kMaxRows * d);
   h->q = cv.take<float>((size_t)kMaxRows * d);
   h->logits = cv.take<float>((size_t)kMaxRows * V);
+  h->st_in = cv.take<int>(kMaxRows);
+  h->st_tok = cv.take<int>(kMaxRows);
+  h->st_uni = cv.take<float>(kMaxRows);
+  h->st_log = cv.take<float>((size_t)kMaxRows * V);
+  h->st_hid = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->a = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->o = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->hbuf = cv.take<uint16_t>((size_t)kMaxRows * F);
@@ -871,6 +879,27 @@ int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
   h->n_free += (h->ctx[s] + 63) / 64;
   h->open[s] = 0; h->ctx[s] = 0;
   return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_decode_step_host(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, const int32_t *in_tokens,
+                                 int32_t top_k, float temperature, const float *uniforms, int32_t *out_tokens,
+                                 float *out_logits, void *out_hidden) {
+  if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
+  const tts_gpt_config_t &c = h->cfg;
+  if (n < 1 || n > c.max_streams || !stream_ids || !out_tokens) return fail(h, TTS_GPT_E_ARG, "decode_step_host: bad n or null argument");
+  if (top_k > 1 && !uniforms) return fail(h, TTS_GPT_E_ARG, "decode_step_host: top-k sampling needs uniforms");
+  if (in_tokens) CUDA_TRY(h, cudaMemcpyAsync(h->st_in, in_tokens, (size_t)n * sizeof(int), cudaMemcpyHostToDevice, h->stream));
+  if (top_k > 1) CUDA_TRY(h, cudaMemcpyAsync(h->st_uni, uniforms, (size_t)n * sizeof(float), cudaMemcpyHostToDevice, h->stream));
+  const int rc = tts_gpt_decode_step(h, n, stream_ids, in_tokens ? h->st_in : nullptr, top_k, temperature,
+                                     top_k > 1 ? h->st_uni : nullptr, h->st_tok, out_logits ? h->st_log : nullptr,
+                                     out_hidden ? h->st_hid : nullptr);
+  if (rc) return rc;
+  CUDA_TRY(h, cudaMemcpyAsync(out_tokens, h->st_tok, (size_t)n * sizeof(int), cudaMemcpyDeviceToHost, h->stream));
+  if (out_logits)
+    CUDA_TRY(h, cudaMemcpyAsync(out_logits, h->st_log, (size_t)n * c.vocab * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+  if (out_hidden)
+    CUDA_TRY(h, cudaMemcpyAsync(out_hidden, h->st_hid, (size_t)n * c.d_model * sizeof(uint16_t), cudaMemcpyDeviceToHost, h->stream));
+  return tts_gpt_sync(h);
 }
 
 int32_t tts_gpt_sync(tts_gpt_t *h) {

@@ -452,3 +452,59 @@ def test_fused_qkv_attention_kernel_matches_oracle(tiny_models, wfmt, monkeypatc
     eng.destroy()
     assert fused_launches == plain_launches - n * cfg.n_layer      # one kernel fewer per layer and step
     assert_same_up_to_ties(toks, logits, toks2, logits2, "fused vs default")
+
+
+@pytest.mark.parametrize("top_k", [0, 8])
+def test_decode_step_host_equals_device_entry(tiny_models, top_k):
+    """The host-buffer entry (copies in, step, copies out, wait) gives bit for bit what the device-pointer
+    entry gives, with page-locked and with pageable host buffers; results are valid on return."""
+    cfg, w, model = tiny_models[C.W_BF16]
+    S, n = 3, 9
+    prefixes = [bits_dev(p) for p in C.make_prefixes(cfg, [40, 64, 7], seed=12)]
+    uni = C.make_uniforms(n + 1, S, seed=4) if top_k > 1 else None
+    V, d = cfg.vocab, cfg.d_model
+    uni_dev = None if uni is None else torch.from_numpy(uni).to(DEV)   # resident before the engine's stream reads it
+    torch.cuda.synchronize()
+
+    def open_engine():
+        eng = B.TtsGpt(cfg, w, DEV)
+        t0 = torch.zeros(S, dtype=torch.int32, device=DEV)
+        torch.cuda.synchronize()
+        ids, _ = eng.prefill(prefixes, top_k=top_k, uniforms=None if uni is None else uni_dev[0], out_tokens=t0)
+        eng.sync()
+        return eng, ids, t0.cpu()
+
+    # device entry, tokens fed back by the caller
+    eng, ids, t0 = open_engine()
+    dev_tok = torch.zeros((n, S), dtype=torch.int32, device=DEV)
+    dev_log = torch.zeros((n, S, V), dtype=torch.float32, device=DEV)
+    dev_hid = torch.zeros((n, S, d), dtype=torch.int16, device=DEV)
+    prev = t0.to(DEV)
+    torch.cuda.synchronize()
+    for k in range(n):
+        eng.decode_step(ids, dev_tok[k], in_tokens=prev, top_k=top_k,
+                        uniforms=None if uni is None else uni_dev[k + 1],
+                        out_logits=dev_log[k], out_hidden=dev_hid[k])
+        prev = dev_tok[k]
+    eng.sync(); eng.destroy()
+    for pinned in (True, False):
+        eng, ids2, t0b = open_engine()
+        assert torch.equal(t0, t0b)
+        mk = (lambda *a, **kw: torch.zeros(*a, **kw).pin_memory()) if pinned else torch.zeros
+        h_in = mk(S, dtype=torch.int32); h_in.copy_(t0)
+        h_tok = mk(S, dtype=torch.int32); h_log = mk((S, V), dtype=torch.float32); h_hid = mk((S, d), dtype=torch.int16)
+        for k in range(n):
+            eng.decode_step_host(ids2, h_tok, in_tokens=h_in, top_k=top_k,
+                                 uniforms=None if uni is None else torch.from_numpy(uni[k + 1].copy()),
+                                 out_logits=h_log, out_hidden=h_hid)
+            # valid on return, without any further synchronisation
+            assert torch.equal(h_tok, dev_tok[k].cpu()) and torch.equal(h_log, dev_log[k].cpu()) and torch.equal(h_hid, dev_hid[k].cpu())
+            h_in.copy_(h_tok)
+        with pytest.raises(B.TtsGptError) as e:
+            eng.decode_step_host([ids2[0], ids2[0]], h_tok, in_tokens=h_in)
+        assert e.value.code == B.E_STREAM
+        if top_k > 1:
+            with pytest.raises(B.TtsGptError) as e:
+                eng.decode_step_host(ids2, h_tok, in_tokens=h_in, top_k=top_k)
+            assert e.value.code == B.E_ARG
+        eng.destroy()
