@@ -12,6 +12,7 @@ timing is the max over ranks.  `--impl reference` times the fp64 CPU oracle inst
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import sys
@@ -243,6 +244,7 @@ def run_ours(args):
     h_uni = None if uni is None else uni.cpu().pin_memory()
     h_in.copy_(toks[0].cpu())
     d2h_bytes = 0
+    all_ids = (ctypes.c_int32 * S)(*ids)      # marshalled once for the steps in which every stream is active
     barrier()
     t0 = time.perf_counter()
     e2e_tokens = 0
@@ -250,8 +252,8 @@ def run_ours(args):
         act = active_at(k, ids)
         if not act:
             break
-        sids = [s for _, s in act]
-        n = len(sids)
+        n = len(act)
+        sids = all_ids if n == S else [s for _, s in act]
         eng.decode_step_host(sids, h_tok, in_tokens=h_in, top_k=wl.top_k, temperature=wl.temperature,
                              uniforms=None if h_uni is None else h_uni[k], out_logits=h_log, out_hidden=h_hid)
         h_in[:n].copy_(h_tok[:n])
