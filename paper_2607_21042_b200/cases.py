@@ -159,6 +159,23 @@ def linear_shapes(cfg: GPTConfig):
     return {"qkv": (3 * d, d), "o": (d, d), "fc1": (f, d), "fc2": (d, f)}
 
 
+def quantize_weights(w_bf16: dict, wfmt: int) -> dict:
+    """Derive the packed W8A16 / W4A16 weight set from a bf16 draw of ``make_weights``: the four block
+    linears of every layer are quantized, everything else is shared.  With W_BF16 the draw itself
+    comes back."""
+    if wfmt == W_BF16:
+        return w_bf16
+    if wfmt not in (W_INT8_PC, W_INT4_G128):
+        raise ValueError("unknown weight format")
+    quant = quantize_int8_per_channel if wfmt == W_INT8_PC else quantize_int4_group128
+    out = dict(w_bf16)
+    for lin in LINEARS:
+        qs = [quant(wb) for wb in w_bf16[lin + "_w"]]
+        out[lin + "_w"] = [q for q, _ in qs]
+        out[lin + "_s"] = [s for _, s in qs]
+    return out
+
+
 def make_weights(cfg: GPTConfig, seed: int = 0) -> dict:
     """Draw every tensor of the decoder in a fixed order from the (seed, TAG_WEIGHTS) stream.
 
@@ -183,22 +200,9 @@ def make_weights(cfg: GPTConfig, seed: int = 0) -> dict:
 
     def put_linear(name):
         n, k = shapes[name]
-        wb = _normal_bf16(rng, (n, k), 0.02)
-        bb = _normal_bf16(rng, (n,), 0.02)
-        if cfg.wfmt == W_BF16:
-            w[name + "_w"].append(wb)
-            w[name + "_s"].append(None)
-        elif cfg.wfmt == W_INT8_PC:
-            q, s = quantize_int8_per_channel(wb)
-            w[name + "_w"].append(q)
-            w[name + "_s"].append(s)
-        elif cfg.wfmt == W_INT4_G128:
-            q, s = quantize_int4_group128(wb)
-            w[name + "_w"].append(q)
-            w[name + "_s"].append(s)
-        else:
-            raise ValueError("unknown weight format")
-        w[name + "_b"].append(bb)
+        w[name + "_w"].append(_normal_bf16(rng, (n, k), 0.02))
+        w[name + "_s"].append(None)
+        w[name + "_b"].append(_normal_bf16(rng, (n,), 0.02))
 
     for _ in range(cfg.n_layer):
         w["ln1_g"].append(_normal_bf16(rng, (d,), 0.01, 1.0))
@@ -213,7 +217,7 @@ def make_weights(cfg: GPTConfig, seed: int = 0) -> dict:
     w["lnf_b"] = _normal_bf16(rng, (d,), 0.01)
     w["head_w"] = _normal_bf16(rng, (v, d), 0.02)
     w["head_b"] = None
-    return w
+    return quantize_weights(w, cfg.wfmt)
 
 
 # ---------------------------------------------------------------------------------------------

@@ -11,10 +11,30 @@ decode path has no exchange step and uses no collective.  What is left for the h
 """
 from __future__ import annotations
 
+import os
+import socket
+import subprocess
+import sys
 from dataclasses import dataclass, field
 
 import torch
 import torch.distributed as dist
+
+
+def launch_ranks(script: str, argv, n_ranks: int, port: int = 0) -> int:
+    """Runs `script argv...` as n_ranks processes of one node (one per GPU) under
+    torch.distributed.run, rendezvous on 127.0.0.1, and returns its exit code.  Each rank finds
+    RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* in its environment."""
+    if port <= 0:
+        s = socket.socket()
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+        s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(int(n_ranks)),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), script] + list(argv)
+    env = dict(os.environ)
+    env.setdefault("OMP_NUM_THREADS", "4")
+    return subprocess.call(cmd, env=env)
 
 
 def max_over_ranks(value: float, device=None) -> float:

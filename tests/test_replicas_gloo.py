@@ -78,3 +78,22 @@ def test_reductions_with_two_gloo_ranks():
 def test_reductions_without_process_group_are_identity():
     assert R.max_over_ranks(3.5) == 3.5
     assert R.whole_job_throughput(100, 50.0) == 2000.0
+
+
+def test_bench_gpus_2_starts_two_ranks():
+    """`python bench.py --gpus 2` from a plain process re-executes itself as two ranks; in the dry
+    mode (gloo, no GPU work) rank 0 prints one line for the whole job."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--dry-run"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["dry_run"] is True
+    # two ranks of 100 tokens each over the slower rank's 11 ms
+    assert abs(out["value"] - 200 / 11e-3) < 1e-6
