@@ -64,16 +64,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   return t;
 }
 __device__ __forceinline__ void trace_mark(unsigned long long *trace, int slot, int which, int tid = 0) {
-#ifdef TTS_TRACE_GRID_MAX   // experiments: word 7 of the slot = latest end mark over all CTAs of the grid
-  if (trace && threadIdx.x == tid && which == 2) atomicMax(trace + 8 * slot + 7, global_timer_ns());
-#endif
-#ifdef TTS_TRACE_CTA_EIGHTH   // experiments: the CTA at TTS_TRACE_CTA_EIGHTH/8 of the grid marks instead of the first
-  const unsigned lin = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-  const unsigned tot = gridDim.x * gridDim.y * gridDim.z;
-  if (trace && threadIdx.x == tid && lin == min(tot - 1, tot * TTS_TRACE_CTA_EIGHTH / 8))
-#else
   if (trace && threadIdx.x == tid && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
-#endif
     trace[8 * slot + which] = global_timer_ns();
 }
 

@@ -428,30 +428,72 @@ def test_prefill_tokens_assembles_the_prefix_on_the_device(wfmt):
 
 
 @pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
-def test_fused_qkv_attention_kernel_matches_oracle(tiny_models, wfmt, monkeypatch):
-    """The optional one-kernel LayerNorm + QKV + attention of one-row steps (switched on by an environment
-    variable read at engine creation) against the oracle, across a page boundary, and against the default
-    schedule of the same engine build."""
+def test_persistent_step_kernel_matches_oracle_and_stage_kernels(tiny_models, wfmt):
+    """Decode steps of one row run as one persistent kernel (embedding to logits) plus sampling; the
+    same engine with that schedule switched off runs one kernel per stage.  Both against the oracle,
+    across a page boundary, and against each other."""
     cfg, w, model = tiny_models[wfmt]
     prefix = C.make_prefixes(cfg, [60], seed=31)[0]
     n = 12
-    monkeypatch.setenv("TTS_GPT_QKV_ATTN", "1")
     eng = B.TtsGpt(cfg, w, DEV)
     l0 = eng.kernel_launches()
     toks, logits, hidden, sid = gpu_run_stream(eng, bits_dev(prefix), n, want_hidden=True)
-    fused_launches = eng.kernel_launches() - l0
+    ps_launches = eng.kernel_launches() - l0
     ref_logits, ref_hidden = O.replay_full(model, O.bf16_to_f64(prefix), toks[:-1])
-    assert_logits_close(logits, ref_logits, "fused")
-    check_tokens(toks, ref_logits, 0, 1.0, None, "fused")
-    eng.destroy()
-    monkeypatch.delenv("TTS_GPT_QKV_ATTN")
-    eng = B.TtsGpt(cfg, w, DEV)
+    assert_logits_close(logits, ref_logits, "persistent")
+    check_tokens(toks, ref_logits, 0, 1.0, None, "persistent")
+    assert np.max(np.abs(O.bf16_to_f64(hidden) - ref_hidden)) <= 3e-2 * max(1.0, np.abs(ref_hidden).max())
+    eng.release_stream(sid)
+    eng.set_option("persistent", 0)
     l0 = eng.kernel_launches()
     toks2, logits2, _, _ = gpu_run_stream(eng, bits_dev(prefix), n)
     plain_launches = eng.kernel_launches() - l0
     eng.destroy()
-    assert fused_launches == plain_launches - n * cfg.n_layer      # one kernel fewer per layer and step
-    assert_same_up_to_ties(toks, logits, toks2, logits2, "fused vs default")
+    # per step: set-up + persistent kernel + sampling, against set-up + embed + 5 per layer + head + sampling
+    assert plain_launches - ps_launches == n * (5 * cfg.n_layer + 1)
+    assert_same_up_to_ties(toks, logits, toks2, logits2, "persistent vs stage kernels")
+
+
+@pytest.mark.parametrize("n_streams", [2, 3, 4])
+def test_persistent_step_kernel_batches(tiny_models, n_streams):
+    """Steps of 2 to 4 rows through the persistent kernel: ragged contexts, top-k sampling, streams
+    leaving the batch; every stream replayed by the oracle."""
+    cfg, w, model = tiny_models[C.W_INT4_G128]
+    eng = B.TtsGpt(cfg, w, DEV)
+    lens = [70, 5, 129, 64][:n_streams]
+    prefixes = C.make_prefixes(cfg, lens, seed=77)
+    n = 10
+    V = cfg.vocab
+    uni = torch.from_numpy(C.make_uniforms(n + 1, n_streams, seed=5)).to(DEV)
+    t0 = torch.zeros(n_streams, dtype=torch.int32, device=DEV)
+    l0 = torch.zeros((n_streams, V), dtype=torch.float32, device=DEV)
+    toks = torch.zeros((n, n_streams), dtype=torch.int32, device=DEV)
+    logits = torch.zeros((n, n_streams, V), dtype=torch.float32, device=DEV)
+    torch.cuda.synchronize()
+    # uniforms of the streams still alive at each step, resident before the engine's stream reads them
+    alive_at = [[i for i in range(n_streams) if not (k >= 6 and i == 1)] for k in range(n + 1)]
+    u_step = [torch.stack([uni[k, i] for i in alive_at[k]]) for k in range(n + 1)]
+    torch.cuda.synchronize()
+    ids, _ = eng.prefill([bits_dev(p) for p in prefixes], top_k=8, uniforms=uni[0], out_tokens=t0, out_logits=l0)
+    alive = list(range(n_streams))
+    rows = [[] for _ in range(n_streams)]
+    for k in range(1, n + 1):
+        if k == 6:                      # the second stream leaves
+            eng.release_stream(ids[alive.pop(1)])
+        m = len(alive)
+        eng.decode_step([ids[i] for i in alive], toks[k - 1, :m], top_k=8, uniforms=u_step[k], out_logits=logits[k - 1, :m])
+        for j, i in enumerate(alive):
+            rows[i].append((k - 1, j))
+    eng.sync()
+    tk, lg, t0, l0 = toks.cpu().numpy(), logits.cpu().numpy(), t0.cpu().numpy(), l0.cpu().numpy()
+    un = uni.cpu().numpy()
+    for i in range(n_streams):
+        seq = np.array([int(t0[i])] + [int(tk[k, j]) for k, j in rows[i]])
+        lgs = np.stack([l0[i]] + [lg[k, j] for k, j in rows[i]])
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
+        assert_logits_close(lgs, ref, "stream %d" % i)
+        check_tokens(seq, ref, 8, 1.0, un[:len(seq), i], "stream %d" % i)
+    eng.destroy()
 
 
 @pytest.mark.parametrize("top_k", [0, 8])
