@@ -197,27 +197,29 @@ int32_t tts_gpt_stream_context(const tts_gpt_t *h, int32_t stream_id);
 int32_t tts_gpt_debug_kernel_launches(const tts_gpt_t *h, uint64_t *n);
 
 /* Timeline tracing (off by default).  `trace` is a DEVICE array of 8 * n_slots uint64, or NULL to
- * switch tracing off; *n_slots (HOST, may be NULL): on entry the number of slots `trace` holds (0 or
- * less: unknown, then only the per-kernel slots below are written), on return the number of slots a
- * step can fill (an upper bound: 5 per layer — QKV, attention, O-proj, FC1, FC2 — then the LM head on the
+ * switch tracing off; *n_slots (HOST, may be NULL) receives the number of traced kernels per step
+ * (an upper bound: 5 per layer — QKV, attention, O-proj, FC1, FC2 — then the LM head on the
  * small-batch path; 7 per layer — LN1, QKV, attention, O-proj, LN2, FC1, FC2 — on the tensor-core path).  While set, CTA 0 of each
  * traced kernel stores the GPU's global nanosecond timer at entry, after its dependency wait and
- * at its end into trace[8*slot + 0..2] (3..5: inner points of the linear kernels).  The persistent
- * kernel of small decode steps fills slot l with CTA 0's stage ends of layer l (LN1, QKV, attention,
- * O-proj, FC1, FC2), slot n_layer with the end of the LM head and, if the buffer is large enough, 16
- * marks per CTA for the middle layer in slots n_layer + 1 + 2 * cta.  Synchronises and drops captured graphs. */
+ * at its end into trace[8*slot + 0..2] (3..5: inner points of the linear kernels).  Synchronises and drops captured graphs. */
 int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots);
 
 /* Test aid: permute the free-page list with a seeded shuffle (between calls, any time no stream
  * is open).  Results must not depend on which physical pages a stream receives. */
 int32_t tts_gpt_debug_shuffle_free_pages(tts_gpt_t *h, uint32_t seed);
 
+/* Test aid: the KV pool sits between two guard regions of the workspace that are filled with a pattern at
+ * creation; *bad_bytes (HOST) receives the number of guard bytes that no longer hold it (0 = no kernel
+ * wrote outside the pool on either side).  Waits for the stream. */
+int32_t tts_gpt_debug_check_canaries(tts_gpt_t *h, int32_t *bad_bytes);
+
 /* Experiments and tests: switches a kernel schedule of this engine on or off (value 0 / 1) or sets
  * a threshold.  Defaults are what the measurements use.  Waits for the stream and drops captured
- * step graphs.  Names: "persistent" (one persistent kernel for decode steps of few rows; Section II-C,
- * the decode iteration), "persistent_max_rows" (0..4), "graph", "pdl", "tc" and "tc_min_rows" (tensor-core
+ * step graphs.  Names: "graph", "pdl", "tc" and "tc_min_rows" (tensor-core
  * linears), "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
- * "fc2_ksplit".  Unknown name or value out of range: TTS_GPT_E_ARG. */
+ * "fc2_ksplit"; "poison_free_pages" (test aid standing in for a memory checker: every free page, and
+ * from then on every released page, is filled with NaN in all layers, so that a kernel reading a slot no
+ * token was written to poisons its result).  Unknown name or value out of range: TTS_GPT_E_ARG. */
 int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value);
 
 /* Test aid for the device-side error path: enqueues a one-thread kernel that waits, with the same

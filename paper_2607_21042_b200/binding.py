@@ -24,7 +24,7 @@ EXPORTS = [
     "tts_gpt_query_workspace", "tts_gpt_create", "tts_gpt_prefill", "tts_gpt_prefill_tokens", "tts_gpt_decode_step", "tts_gpt_decode_step_host", "tts_gpt_decode_steps",
     "tts_gpt_release_stream", "tts_gpt_sync", "tts_gpt_destroy", "tts_gpt_last_error",
     "tts_gpt_stats", "tts_gpt_stream_context", "tts_gpt_debug_shuffle_free_pages",
-    "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace", "tts_gpt_debug_expire_wait", "tts_gpt_debug_set_option",
+    "tts_gpt_debug_kernel_launches", "tts_gpt_debug_set_trace", "tts_gpt_debug_expire_wait", "tts_gpt_debug_set_option", "tts_gpt_debug_check_canaries",
     "tts_gpt_op_linear_packed_bytes", "tts_gpt_op_linear_pack", "tts_gpt_op_linear",
     "tts_gpt_op_linear_tc_scratch_bytes", "tts_gpt_op_linear_tc", "tts_gpt_op_attention_scratch_bytes", "tts_gpt_op_attention", "tts_gpt_op_attention_static", "tts_gpt_op_attention_cluster",
     "tts_gpt_op_layernorm",
@@ -271,7 +271,7 @@ class TtsGpt:
     def set_trace(self, trace_tensor):
         """trace_tensor: int64 device tensor with 8 * slots entries (or None to switch off).
         Returns the number of traced kernels per step."""
-        n = C.c_int32(0 if trace_tensor is None else trace_tensor.numel() // 8)
+        n = C.c_int32(0)
         _check(self.lib.tts_gpt_debug_set_trace(self.handle, _ptr(trace_tensor), C.byref(n)), self.handle)
         return n.value
 
@@ -282,6 +282,12 @@ class TtsGpt:
         """Switch a kernel schedule on or off, or set a threshold (see tts_gpt_debug_set_option)."""
         return _check(self.lib.tts_gpt_debug_set_option(self.handle, C.c_char_p(name.encode()), C.c_int32(int(value))),
                       self.handle)
+
+    def check_canaries(self):
+        """Number of guard bytes around the KV pool that were overwritten (0 = intact)."""
+        n = C.c_int32(0)
+        _check(self.lib.tts_gpt_debug_check_canaries(self.handle, C.byref(n)), self.handle)
+        return n.value
 
     def debug_expire_wait(self, limit_us):
         return _check(self.lib.tts_gpt_debug_expire_wait(self.handle, C.c_uint32(limit_us)), self.handle)

@@ -687,7 +687,9 @@ inline cudaError_t launch_attention_prefill(const AttnArgs &a, int R, cudaStream
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kAttnWarps * 32) attention_ticket_kernel(const AttnArgs a) {
   const int c = blockIdx.x, h = blockIdx.y, r = blockIdx.z;
-  const int n_tok = a.row_pos[r] + 1;
+  // a position beyond the stream's page table (the caller's mistake) is cut to what the table and the grid
+  // cover: every chunk then exists, so the ticket completes, the row is written and the ticket returns to zero
+  const int n_tok = min(min(a.row_pos[r] + 1, a.pps * kPageTokens), (int)gridDim.x * kAttnWarps * kPageTokens);
   const int n_pages = (n_tok + kPageTokens - 1) / kPageTokens;
   const int n_chunks = (n_pages + kAttnWarps - 1) / kAttnWarps;
   if (c >= n_chunks) return;

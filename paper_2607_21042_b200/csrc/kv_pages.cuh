@@ -166,6 +166,23 @@ __global__ void __launch_bounds__(kMaxRows) prefill_pass_kernel(const PassParams
   if (i == 0) *io = p.io;
 }
 
+// Debug aid: fills the K and V blocks of the given pages, in every layer, with bf16 NaN.  A kernel that reads
+// a slot no token was written to (a stale page, a slot beyond the context) then poisons its result.
+// pages == nullptr: the n pages on top of the free stack (all free pages when n = *free_top).
+__global__ void poison_pages_kernel(uint16_t *kv, size_t kv_layer_elems, int n_layer, size_t page_elems,
+                                    const int *pages, const int *free_list, int n) {
+  const size_t per_page = page_elems / 8;   // 16-byte units of one page in one layer
+  const size_t total = (size_t)n * n_layer * per_page;
+  const uint4 nan4 = make_uint4(0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u, 0x7FC07FC0u);
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t u = i % per_page;
+    const size_t t = i / per_page;
+    const int l = (int)(t % n_layer), j = (int)(t / n_layer);
+    const int page = pages ? pages[j] : free_list[j];
+    reinterpret_cast<uint4 *>(kv + kv_layer_elems * l + (size_t)page * page_elems)[u] = nan4;
+  }
+}
+
 // Returns a stream's pages to the stack (last page first, so that the next stream to open pops
 // them in the order this one received them).
 __global__ void release_kernel(PageState ps, int s) {

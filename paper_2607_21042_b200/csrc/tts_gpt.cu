@@ -3,6 +3,7 @@
 #include "../../include/tts_gpt.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstdarg>
@@ -19,7 +20,6 @@
 #include "gemm_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
-#include "step_persistent.cuh"
 
 using namespace ttsgpt;
 
@@ -30,7 +30,6 @@ thread_local std::string g_last_error;
 struct PackedLinear {
   void *w_img = nullptr;   // bf16 only: operand image for the tensor-core path (rows padded to 128)
   void *w = nullptr;
-  void *ps_w = nullptr;    // records of the persistent step kernel (steps of up to kPsMaxRows rows)
   uint16_t *s = nullptr;
   uint16_t *bias = nullptr;
   int N = 0, K = 0;
@@ -91,23 +90,14 @@ struct tts_gpt {
   int attn_cluster_fill = 1;     // clusters grow until the grid covers the GPU this many times
   int attn_stream_min_pairs = 0; // (row, head) pairs from which it is used; 0: attention_use_stream decides
   int tc_min_rows = 17; // rows from which the tensor-core path is taken (option "tc_min_rows")
-  // persistent step kernel (decode steps of up to ps_max_rows rows)
-  bool have_ps = false;          // the configuration has records and exchange buffers for it
-  bool use_ps = true;            // option "persistent"
-  int ps_max_rows = kPsMaxRows;  // option "persistent_max_rows"
-  PsLayerDesc *ps_layers = nullptr;
-  std::vector<PsLayerDesc> ps_layers_host;
-  unsigned long long *ps_xchg = nullptr;
-  int *ps_abort = nullptr;
-  uint32_t ps_seq = 0;
-  int ps_grid = 0, ps_smem = 0;   // CTAs of the launch; shared memory a CTA may opt in to
+  bool poison_free = false;     // option "poison_free_pages": released pages are filled with NaN
+  unsigned char *canary_lo = nullptr, *canary_hi = nullptr;   // guard regions either side of the KV pool
   int n_sm = 148;
   unsigned long long launches = 0;
   int *dev_err = nullptr;               // error word set by a kernel whose bounded wait expired:
   volatile int *host_err = nullptr;     //   4 bytes of pinned, device-mapped host memory (read after a sync without a copy)
   unsigned long long *trace = nullptr;  // optional device buffer for kernel timelines
   int trace_next = 0;  // kernels enqueued so far (graph nodes counted per replay)
-  int trace_slots = 0; // slots the caller's trace buffer holds (0: only the per-kernel slots are assumed)
 };
 
 namespace {
@@ -149,6 +139,9 @@ int check_config(const tts_gpt_config_t *c) {
 // rows of the embedding table: the semantic codes and specials the head predicts, then the text region if any
 inline int emb_rows_of(const tts_gpt_config_t &c) { return c.emb_rows > 0 ? c.emb_rows : c.vocab; }
 
+constexpr size_t kCanaryBytes = 4096;      // guard region in front of and behind the KV pool
+constexpr unsigned char kCanaryByte = 0xA5;
+
 // Walks the workspace; with base == nullptr only measures.
 struct Carver {
   char *base;
@@ -162,9 +155,8 @@ struct Carver {
   }
 };
 
-void carve_linear(Carver &cv, PackedLinear &pl, int wf, int N, int K, int ps_d) {
+void carve_linear(Carver &cv, PackedLinear &pl, int wf, int N, int K) {
   pl.N = N; pl.K = K;
-  pl.ps_w = ps_d > 0 ? cv.take<char>(ps_weight_bytes(wf, N, K, ps_d)) : nullptr;
   pl.w_img = (K % 128 == 0) ? cv.take<char>(weight_image_bytes(N, K)) : nullptr;
   pl.w = cv.take<char>(packed_weight_bytes(wf, N, K));
   size_t sb = packed_scale_bytes(wf, N, K);
@@ -181,20 +173,20 @@ size_t carve(tts_gpt *h, void *base) {
   h->pos_emb = cv.take<uint16_t>((size_t)c.max_pos * d);
   h->lnf_g = cv.take<uint16_t>(d);
   h->lnf_b = cv.take<uint16_t>(d);
-  h->have_ps = ps_supported(d, F, c.n_head, c.n_layer, V, 148);
-  const int ps_d = h->have_ps ? d : 0;
-  carve_linear(cv, h->head, WF_BF16, V, d, ps_d);
+  carve_linear(cv, h->head, WF_BF16, V, d);
   h->layers.resize(c.n_layer);
   for (auto &L : h->layers) {
     L.ln1_g = cv.take<uint16_t>(d); L.ln1_b = cv.take<uint16_t>(d);
     L.ln2_g = cv.take<uint16_t>(d); L.ln2_b = cv.take<uint16_t>(d);
-    carve_linear(cv, L.qkv, c.wfmt, 3 * d, d, ps_d);
-    carve_linear(cv, L.o, c.wfmt, d, d, ps_d);
-    carve_linear(cv, L.fc1, c.wfmt, F, d, ps_d);
-    carve_linear(cv, L.fc2, c.wfmt, d, F, ps_d);
+    carve_linear(cv, L.qkv, c.wfmt, 3 * d, d);
+    carve_linear(cv, L.o, c.wfmt, d, d);
+    carve_linear(cv, L.fc1, c.wfmt, F, d);
+    carve_linear(cv, L.fc2, c.wfmt, d, F);
   }
   h->kv_layer_elems = (size_t)c.n_pages * 2 * c.n_head * kPageElems;
+  h->canary_lo = cv.take<unsigned char>(kCanaryBytes);
   h->kv = cv.take<uint16_t>(h->kv_layer_elems * c.n_layer);
+  h->canary_hi = cv.take<unsigned char>(kCanaryBytes);
   PageState &ps = h->ps;
   ps.pps = h->pps; ps.n_pages = c.n_pages; ps.max_streams = S;
   ps.ctx_len = cv.take<int>(S);
@@ -231,11 +223,6 @@ size_t carve(tts_gpt *h, void *base) {
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
   h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
-  if (h->have_ps) {
-    h->ps_layers = cv.take<PsLayerDesc>(c.n_layer);
-    h->ps_xchg = cv.take<unsigned long long>(ps_exchange_words(d, F, c.n_head));
-    h->ps_abort = cv.take<int>(1);
-  }
   h->have_tc = true;
   if (h->have_tc) {
     h->a_img = cv.take<char>(act_image_bytes(d));
@@ -258,7 +245,6 @@ int load_linear(tts_gpt *h, PackedLinear &pl, int wf, const void *w, const void 
   if (!w || !b || (wf != WF_BF16 && !s)) return fail(h, TTS_GPT_E_ARG, "weights: %s has a null tensor", what);
   CUDA_TRY(h, launch_pack(wf, pl.N, pl.K, w, s, pl.w, pl.s, h->stream));
   if (pl.w_img) CUDA_TRY(h, launch_pack_image(wf, pl.N, pl.K, w, pl.w_img, h->stream));
-  if (pl.ps_w) CUDA_TRY(h, launch_ps_pack(wf, pl.N, pl.K, h->cfg.d_model, w, s, b, pl.ps_w, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(pl.bias, b, (size_t)pl.N * 2, cudaMemcpyDeviceToDevice, h->stream));
   return TTS_GPT_OK;
 }
@@ -526,53 +512,6 @@ int check_io_alignment(tts_gpt *h, const void *in_tokens, const void *uniforms, 
   return TTS_GPT_OK;
 }
 
-// Ring size of the persistent kernel for a step of R rows: what the fixed buffers leave of shared memory.
-long long ps_ring_bytes(const tts_gpt *h, int R) {
-  return ((long long)h->ps_smem - (long long)ps_fixed_smem(h->cfg.d_model, h->cfg.d_ff, R) - 1024) / 128 * 128;
-}
-
-// A decode step of a few rows: the whole step after the set-up kernel is one persistent kernel
-// (embedding to logits), followed by sampling.
-int run_step_persistent(tts_gpt *h, int R) {
-  const tts_gpt_config_t &c = h->cfg;
-  const int d = c.d_model, F = c.d_ff;
-  PsArgs a;
-  memset(&a, 0, sizeof a);
-  a.layers = h->ps_layers; a.n_layer = c.n_layer;
-  a.head_w = (const unsigned char *)h->head.ps_w; a.lnf_g = h->lnf_g; a.lnf_b = h->lnf_b;
-  a.kv = h->kv; a.kv_layer_elems = h->kv_layer_elems;
-  a.tok_emb = h->tok_emb; a.pos_emb = h->pos_emb; a.emb_rows = emb_rows_of(c); a.max_pos = c.max_pos;
-  a.d = d; a.d_ff = F; a.H = c.n_head; a.V = c.vocab; a.ln_eps = c.ln_eps; a.gelu_tanh = c.gelu_tanh;
-  a.row_stream = h->rt.row_stream; a.row_pos = h->rt.row_pos; a.row_token = h->rt.row_token; a.row_posidx = h->rt.row_posidx;
-  a.page_table = h->ps.page_table; a.pps = h->pps; a.R = R;
-  a.io = h->io;
-  h->ps_seq = h->ps_seq % 0xFFFFFFu + 1u;      // 1 .. 2^24 - 1: (seq << 8) never is 0 and fits 32 bits
-  a.seq = h->ps_seq;
-  unsigned long long *x = h->ps_xchg;
-  const size_t rd = (size_t)kPsMaxRows * d;
-  a.xa = x; x += rd;
-  a.xb = x; x += rd;
-  a.hb = x; x += (size_t)kPsMaxRows * F;
-  a.qb = x; x += rd;
-  a.kn = x; x += 2 * rd;
-  a.pb = x; x += (size_t)kPsMaxRows * c.n_head * kPsMaxSplit * kPsPartialWords;
-  a.ob = x;
-  a.logits = h->logits;
-  a.abort_g = h->ps_abort; a.err = h->dev_err;
-  a.trace = h->trace;
-  a.trace_detail = h->trace && h->trace_slots >= c.n_layer + 1 + 8 * h->ps_grid ? 1 : 0;
-  a.ring_bytes = (uint32_t)ps_ring_bytes(h, R);
-  CUDA_TRY(h, launch_step_persistent(c.wfmt, a, h->ps_grid, ps_smem_bytes(d, F, R, a.ring_bytes), h->stream));
-  SampleArgs sa;
-  memset(&sa, 0, sizeof sa);
-  sa.logits = h->logits; sa.V = c.vocab; sa.io = h->io; sa.out_slot = h->rt.out_slot; sa.out_rows = h->rt.out_rows;
-  sa.row_stream = h->rt.row_stream; sa.last_token = h->ps.last_token; sa.stop_flag = h->ps.stop_flag;
-  sa.stop_token = c.stop_token;
-  CUDA_TRY(h, launch_kernel(sample_kernel, dim3(R), dim3(kSampleThreads), (size_t)c.vocab * sizeof(float), h->stream, false, sa));
-  h->launches += 2;
-  return TTS_GPT_OK;
-}
-
 int check_top_k(tts_gpt *h, int top_k, float temperature, const float *uniforms) {
   if (top_k < 0 || top_k > kMaxTopK) return fail(h, TTS_GPT_E_ARG, "top_k must be in 0..%d", kMaxTopK);
   if (top_k > 1 && !(temperature > 0.f)) return fail(h, TTS_GPT_E_ARG, "temperature must be positive");
@@ -620,7 +559,6 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   {
     cudaError_t e = launch_pack(WF_BF16, h->head.N, h->head.K, w->head_w, nullptr, h->head.w, nullptr, h->stream);
     if (e == cudaSuccess && h->head.w_img) e = launch_pack_image(WF_BF16, h->head.N, h->head.K, w->head_w, h->head.w_img, h->stream);
-    if (e == cudaSuccess && h->head.ps_w) e = launch_ps_pack(WF_BF16, h->head.N, h->head.K, d, w->head_w, nullptr, w->head_b, h->head.ps_w, h->stream);
     if (e != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "pack head: %s", cudaGetErrorString(e)); }
     if (w->head_b) {
       TRY_(copy_bf16(h, h->head.bias, w->head_b, c.vocab, "head_b"));
@@ -649,25 +587,11 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
     TRY_(load_linear(h, L.fc2, c.wfmt, w->fc2_w[l], qz ? w->fc2_s[l] : nullptr, w->fc2_b[l], "fc2"));
   }
 #undef TRY_
-  if (h->have_ps) {
-    h->ps_layers_host.resize(c.n_layer);
-    for (int l = 0; l < c.n_layer; ++l) {
-      LayerW &L = h->layers[l];
-      PsLayerDesc &pd = h->ps_layers_host[l];
-      pd.qkv_w = (const unsigned char *)L.qkv.ps_w; pd.o_w = (const unsigned char *)L.o.ps_w;
-      pd.fc1_w = (const unsigned char *)L.fc1.ps_w; pd.fc2_w = (const unsigned char *)L.fc2.ps_w;
-      pd.ln1_g = L.ln1_g; pd.ln1_b = L.ln1_b; pd.ln2_g = L.ln2_g; pd.ln2_b = L.ln2_b;
-    }
-    cudaError_t pe = cudaMemcpyAsync(h->ps_layers, h->ps_layers_host.data(), sizeof(PsLayerDesc) * c.n_layer,
-                                     cudaMemcpyHostToDevice, h->stream);
-    // tag 0 never names a launch: the exchange words start out as "not written"
-    if (pe == cudaSuccess) pe = cudaMemsetAsync(h->ps_xchg, 0, ps_exchange_words(d, c.d_ff, c.n_head) * 8, h->stream);
-    if (pe == cudaSuccess) pe = cudaMemsetAsync(h->ps_abort, 0, sizeof(int), h->stream);
-    if (pe != cudaSuccess) { delete h; return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(pe)); }
-  }
   const int init_n = std::max(std::max(c.n_pages, c.max_streams * h->pps), c.max_streams);
   init_pages_kernel<<<(init_n + 255) / 256, 256, 0, h->stream>>>(h->ps);
   cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)kMaxRows * c.n_head * sizeof(unsigned int), h->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_lo, kCanaryByte, kCanaryBytes, h->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_hi, kCanaryByte, kCanaryBytes, h->stream);
   if (e == cudaSuccess) {
     void *hp = nullptr, *dp = nullptr;
     e = cudaHostAlloc(&hp, sizeof(int), cudaHostAllocMapped);
@@ -692,18 +616,9 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   // the legacy default stream cannot be captured
   h->use_graph = h->stream != nullptr && h->stream != cudaStreamLegacy;
   h->use_pdl = true;
-  int dev = 0, sms = 0, smem_optin = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) {
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) h->n_sm = sms;
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-  }
-  if (h->have_ps) {
-    // persistent step kernel: one CTA per SM, the ring takes what the fixed buffers leave of shared memory
-    h->ps_grid = h->n_sm;
-    h->ps_smem = smem_optin;
-    const long long need = 2 * (long long)std::max<uint32_t>(kPsItemBytes, kPsChunkTokens * 256u);
-    if (ps_ring_bytes(h, kPsMaxRows) < need || !ps_supported(d, c.d_ff, c.n_head, c.n_layer, c.vocab, h->ps_grid)) h->use_ps = false;
-  }
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+    h->n_sm = sms;
   *out = h;
   return TTS_GPT_OK;
 }
@@ -849,6 +764,33 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   }
   if (pages > h->n_free) return fail(h, TTS_GPT_E_NO_PAGES, "decode_step: %d pages needed, %d free", pages, h->n_free);
 
+  // The step's graph is captured (nothing runs during capture) before anything of the call is committed: a
+  // failure to capture or instantiate leaves the engine exactly as it was.
+  cudaGraphExec_t exec = nullptr;
+  if (h->use_graph) {
+    auto it = h->graphs.find(n);
+    if (it == h->graphs.end()) {
+      cudaGraph_t g = nullptr;
+      const unsigned long long before = h->launches;
+      CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
+      rc = run_embed(h, n);
+      if (!rc) rc = run_layers(h, n, true);
+      if (!rc) rc = run_head(h, n, n);
+      cudaError_t e = cudaStreamEndCapture(h->stream, &g);
+      const int nodes = (int)(h->launches - before);
+      h->launches = before;  // captured, not run
+      if (rc) { if (g) cudaGraphDestroy(g); return rc; }
+      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph capture: %s", cudaGetErrorString(e));
+      cudaGraphExec_t ge = nullptr;
+      e = cudaGraphInstantiate(&ge, g, 0);
+      cudaGraphDestroy(g);
+      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
+      it = h->graphs.emplace(n, ge).first;
+      h->graph_nodes[n] = nodes;
+    }
+    exec = it->second;
+  }
+
   StepParams sp;
   sp.n = n;
   memcpy(sp.stream_ids, stream_ids, (size_t)n * sizeof(int));
@@ -860,28 +802,8 @@ int32_t tts_gpt_decode_step(tts_gpt_t *h, int32_t n, const int32_t *stream_ids, 
   for (int i = 0; i < n; ++i) { h->ctx[stream_ids[i]] += 1; h->pos_next[stream_ids[i]] += 1; }
   h->n_free -= pages;
 
-  if (h->have_ps && h->use_ps && n <= h->ps_max_rows && n * c.n_head <= h->ps_grid) return run_step_persistent(h, n);
-  if (h->use_graph) {
-    auto it = h->graphs.find(n);
-    if (it == h->graphs.end()) {
-      cudaGraph_t g = nullptr;
-      const unsigned long long before = h->launches;
-      CUDA_TRY(h, cudaStreamBeginCapture(h->stream, cudaStreamCaptureModeThreadLocal));
-      rc = run_embed(h, n);
-      if (!rc) rc = run_layers(h, n, true);
-      if (!rc) rc = run_head(h, n, n);
-      cudaError_t e = cudaStreamEndCapture(h->stream, &g);
-      if (rc) { if (g) cudaGraphDestroy(g); return rc; }
-      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph capture: %s", cudaGetErrorString(e));
-      cudaGraphExec_t ge = nullptr;
-      e = cudaGraphInstantiate(&ge, g, 0);
-      cudaGraphDestroy(g);
-      if (e != cudaSuccess) return fail(h, TTS_GPT_E_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
-      it = h->graphs.emplace(n, ge).first;
-      h->graph_nodes[n] = (int)(h->launches - before);
-      h->launches = before;  // captured, not run
-    }
-    CUDA_TRY(h, cudaGraphLaunch(it->second, h->stream));
+  if (exec) {
+    CUDA_TRY(h, cudaGraphLaunch(exec, h->stream));
     h->launches += h->graph_nodes[n];
     return TTS_GPT_OK;
   }
@@ -930,6 +852,12 @@ int32_t tts_gpt_decode_steps(tts_gpt_t *h, int32_t n, const int32_t *stream_ids,
 int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   if (s < 0 || s >= h->cfg.max_streams || !h->open[s]) return fail(h, TTS_GPT_E_STREAM, "release_stream: stream %d is not open", s);
+  if (h->poison_free) {   // before the pages go back: the page table row still names them
+    const int np = (h->ctx[s] + 63) / 64;
+    if (np > 0)
+      poison_pages_kernel<<<256, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, (size_t)2 * h->cfg.n_head * kPageElems,
+                                                      h->ps.page_table + (size_t)s * h->pps, nullptr, np);
+  }
   release_kernel<<<1, 32, 0, h->stream>>>(h->ps, s);
   CUDA_TRY(h, cudaGetLastError());
   h->launches += 1;
@@ -964,10 +892,6 @@ int32_t tts_gpt_sync(tts_gpt_t *h) {
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
   if (h->host_err && *h->host_err) {
     *h->host_err = 0;
-    if (h->ps_abort) {   // the persistent kernel's launch-wide abort flag: cleared for the next launch
-      cudaMemsetAsync(h->ps_abort, 0, sizeof(int), h->stream);
-      cudaStreamSynchronize(h->stream);
-    }
     return fail(h, TTS_GPT_E_TIMEOUT, "a kernel's bounded wait for its weight copy expired; results of the last steps are invalid");
   }
   return TTS_GPT_OK;
@@ -1004,9 +928,7 @@ int32_t tts_gpt_debug_set_trace(tts_gpt_t *h, void *trace, int32_t *n_slots) {
   h->graphs.clear();
   h->graph_nodes.clear();
   h->trace = (unsigned long long *)trace;
-  h->trace_slots = (trace && n_slots && *n_slots > 0) ? *n_slots : 0;
-  if (n_slots) *n_slots = std::max(7 * h->cfg.n_layer + 2, h->cfg.n_layer + 1 + 8 * h->ps_grid);   // upper bound: the tensor-core path traces 7 kernels per layer;
-                                                      // the persistent step kernel fills one slot per layer, one for the head and two per CTA
+  if (n_slots) *n_slots = 7 * h->cfg.n_layer + 2;   // upper bound: the tensor-core path traces 7 kernels per layer
   return TTS_GPT_OK;
 }
 
@@ -1038,9 +960,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   h->graph_nodes.clear();
   const std::string k(name);
   const bool on = value != 0;
-  if (k == "persistent") h->use_ps = on && h->have_ps && h->ps_smem > 0 && ps_supported(h->cfg.d_model, h->cfg.d_ff, h->cfg.n_head, h->cfg.n_layer, h->cfg.vocab, h->ps_grid);
-  else if (k == "persistent_max_rows") { if (value < 0 || value > kPsMaxRows) return fail(h, TTS_GPT_E_ARG, "persistent_max_rows must be in 0..%d", kPsMaxRows); h->ps_max_rows = value; }
-  else if (k == "graph") h->use_graph = on && h->stream != nullptr && h->stream != cudaStreamLegacy;
+  if (k == "graph") h->use_graph = on && h->stream != nullptr && h->stream != cudaStreamLegacy;
   else if (k == "pdl") h->use_pdl = on;
   else if (k == "tc") h->use_tc = on;
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
@@ -1050,7 +970,27 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "attn_stream_min_pairs") h->attn_stream_min_pairs = value > 0 ? value : 0;
   else if (k == "attn_cluster_fill") h->attn_cluster_fill = value > 0 ? value : 1;
   else if (k == "fc2_ksplit") h->use_fc2_ksplit = on;
+  else if (k == "poison_free_pages") {
+    h->poison_free = on;
+    if (on && h->n_free > 0) {   // every page that is free right now
+      poison_pages_kernel<<<1024, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, (size_t)2 * h->cfg.n_head * kPageElems,
+                                                       nullptr, h->ps.free_list, h->n_free);
+      CUDA_TRY(h, cudaGetLastError());
+    }
+  }
   else return fail(h, TTS_GPT_E_ARG, "unknown option %s", name);
+  return TTS_GPT_OK;
+}
+
+int32_t tts_gpt_debug_check_canaries(tts_gpt_t *h, int32_t *bad_bytes) {
+  if (!h || !bad_bytes) return fail(nullptr, TTS_GPT_E_ARG, "null argument");
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  std::vector<unsigned char> buf(2 * kCanaryBytes);
+  CUDA_TRY(h, cudaMemcpy(buf.data(), h->canary_lo, kCanaryBytes, cudaMemcpyDeviceToHost));
+  CUDA_TRY(h, cudaMemcpy(buf.data() + kCanaryBytes, h->canary_hi, kCanaryBytes, cudaMemcpyDeviceToHost));
+  int bad = 0;
+  for (unsigned char b : buf) bad += b != kCanaryByte;
+  *bad_bytes = bad;
   return TTS_GPT_OK;
 }
 
@@ -1195,7 +1135,8 @@ static __device__ __align__(256) unsigned char g_static_attn_scratch[kStaticAttn
 // The symbol above is only a host-side stand-in when named in host code: its device address has to
 // be asked for, once per device, with that device current.
 constexpr int kMaxDevices = 64;
-void *g_static_attn_ptr[kMaxDevices] = {nullptr};
+std::atomic<void *> g_static_attn_ptr[kMaxDevices];   // zero-initialised; first calls from several host threads may race
+                                                       // harmlessly (they store the same address)
 }  // namespace
 
 extern "C" {
@@ -1218,13 +1159,13 @@ int32_t tts_gpt_op_attention_static(int32_t R, int32_t n_head, const float *q, c
   int dev = -1;
   CUDA_TRY(nullptr, cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return fail(nullptr, TTS_GPT_E_UNSUPPORTED, "op_attention_static: device index %d", dev);
-  if (!g_static_attn_ptr[dev]) {  // first call on this device: resolve the array's device address
-    void *p = nullptr;
-    CUDA_TRY(nullptr, cudaGetSymbolAddress(&p, g_static_attn_scratch));
-    if (!p) return fail(nullptr, TTS_GPT_E_CUDA, "op_attention_static: no device address for the scratch array");
-    g_static_attn_ptr[dev] = p;
+  void *resolved = g_static_attn_ptr[dev].load(std::memory_order_relaxed);
+  if (!resolved) {  // first call on this device: resolve the array's device address
+    CUDA_TRY(nullptr, cudaGetSymbolAddress(&resolved, g_static_attn_scratch));
+    if (!resolved) return fail(nullptr, TTS_GPT_E_CUDA, "op_attention_static: no device address for the scratch array");
+    g_static_attn_ptr[dev].store(resolved, std::memory_order_relaxed);
   }
-  unsigned char *base = (unsigned char *)g_static_attn_ptr[dev];
+  unsigned char *base = (unsigned char *)resolved;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   AttnArgs a;
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;

@@ -47,10 +47,9 @@ def test_query_workspace_and_config_errors_need_no_gpu(lib):
     from paper_2607_21042_b200 import binding, cases
     cfg = cases.workload(2).cfg
     n = binding.query_workspace(cfg)
-    # bf16 weights three times (965 MB as records for the persistent step kernel, 965 MB in the tile layout
-    # for 5-16 rows and prefill tails, 985 MB as tensor-core operand images for more than 16 rows) + 32 pages
-    # * 7.86 MB of KV + activations
-    assert 3.0e9 < n < 3.4e9
+    # bf16 weights twice (965 MB in the streaming layout for small batches + 985 MB as tensor-core
+    # operand images for more than 16 rows) + 32 pages * 7.86 MB of KV + activations
+    assert 2.1e9 < n < 2.4e9
     bad = cases.GPTConfig(**{**cfg.as_dict(), "head_dim": 32})
     with pytest.raises(binding.TtsGptError) as e:
         binding.query_workspace(bad)
@@ -59,9 +58,9 @@ def test_query_workspace_and_config_errors_need_no_gpu(lib):
     with pytest.raises(binding.TtsGptError) as e:
         binding.query_workspace(bad)
     assert e.value.code == binding.E_ARG
-    # quantized formats need less: 264 MB of tiles + 254 MB of records + 985 MB of bf16 integer images for the tensor cores
+    # quantized formats need less: 264 MB packed + 985 MB of bf16 integer images for the tensor cores
     n4 = binding.query_workspace(cases.workload(4).cfg)
-    assert n4 < 16 * 32 * 7.9e6 + 1.65e9
+    assert n4 < 16 * 32 * 7.9e6 + 1.4e9
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):

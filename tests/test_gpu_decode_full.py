@@ -106,6 +106,54 @@ def test_workload2_bf16_batch1_replay():
     print("workload2: max-abs %.4g rel-L2 %.4g excused %d/%d" % (ma, rl, exc, n + 1))
     eng.destroy()
 
+def _teacher_forced(wl, wfmt, top_k, n):
+    """The oracle runs free (cached decode, its own samples); the GPU is fed the oracle's tokens and must
+    reproduce its logits and choices at every step."""
+    w, model = _model(wfmt)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    P = 96                                  # prefix rows: the oracle prefills row by row
+    prefix = C.make_prefixes(wl.cfg, [P], seed=3)[0]
+    u = C.make_uniforms(n + 1, 1, seed=3)[:, 0] if top_k > 1 else None
+    run = O.run_stream(model, O.bf16_to_f64(prefix), n, top_k=top_k, temperature=1.0, uniforms=u)
+    forced = torch.from_numpy(run["tokens"][:-1].astype(np.int32)).to(DEV)
+    toks, logits, _, _ = gpu_run_stream(eng, bits_dev(prefix), n, top_k=top_k, temperature=1.0,
+                                        uniforms_dev=None if u is None else torch.from_numpy(u).to(DEV),
+                                        forced_tokens=forced)
+    ma, rl = assert_logits_close(logits, run["logits"], "teacher-forced %s" % wl.name)
+    exc = check_tokens(toks, run["logits"], top_k, 1.0, u, "teacher-forced %s" % wl.name)
+    print("teacher-forced %s: max-abs %.4g rel-L2 %.4g excused %d/%d" % (wl.name, ma, rl, exc, n + 1))
+    eng.destroy()
+
+
+def test_workload2_bf16_teacher_forced():
+    _teacher_forced(C.workload(2), C.W_BF16, 0, 64)
+
+
+def test_workload3_w8a16_topk_teacher_forced():
+    _teacher_forced(C.workload(3), C.W_INT8_PC, 30, 64)
+
+
+def test_context_2048_inside_a_batch_of_128():
+    """One stream reaches the maximum context while it decodes inside a batch of 128 (tensor-core linears,
+    streaming attention); it is replayed by the oracle, a second long stream too."""
+    w, model = _model(C.W_BF16)
+    cfg = C.full_config(wfmt=C.W_BF16, max_streams=128, n_pages=128 * 6 + 2 * 32, max_pos=1024)
+    eng = B.TtsGpt(cfg, w, DEV)
+    n = 58
+    lens = [200 + (7 * i) % 100 for i in range(128)]
+    lens[5], lens[77] = 2048 - n, 1500
+    prefixes = C.make_prefixes(cfg, lens, seed=8)
+    wl = C.Workload("ctx2048_in_batch", cfg, tuple(lens), (n,) * 128, 0)
+    res = _batch_run(eng, wl, prefixes, n)
+    for i in (5, 77):
+        seq, lg = res[i]
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
+        ma, rl = assert_logits_close(lg, ref, "stream %d" % i)
+        check_tokens(seq, ref, 0, 1.0, None, "stream %d" % i)
+        print("context %d in a batch of 128: max-abs %.4g rel-L2 %.4g" % (lens[i] + n, ma, rl))
+    eng.destroy()
+
+
 def test_long_context_2048_full_model():
     """One stream driven to the maximum context (2048 tokens = 32 pages = 8 chunks)."""
     wl = C.workload(2)
@@ -163,3 +211,7 @@ def test_workload4_w4a16_batch16_replay_and_batch_invariance():
 
 def test_workload5_w4a16_batch128_ragged_drain():
     _workload5(C.W_INT4_G128)
+
+
+def test_workload5_w8a16_batch128_ragged_drain():
+    _workload5(C.W_INT8_PC)

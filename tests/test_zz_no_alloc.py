@@ -9,12 +9,11 @@ and that it refuses sizes beyond its stated limit.  It is named to be collected 
 stops at the first failure has already run everything else; it must also pass alone in a fresh
 process (its first call is then the one that looks up the array's device address).
 """
-import ctypes as C
-
 import numpy as np
 import pytest
 import torch
 
+from oracle import gpt_oracle as O
 from paper_2607_21042_b200 import binding as B
 from paper_2607_21042_b200 import cases
 
@@ -39,6 +38,23 @@ def _case(seed, H, ctxs):
             dev(np.array([c - 1 for c in ctxs], dtype=np.int32)))
 
 
+def _reference(args, H, rows):
+    """softmax(q K^T / 8) V per head in fp64, written out, for the given rows of a case."""
+    q, kv, pt, rs, rp = [t.cpu().numpy() for t in args]
+    kvf = O.bf16_to_f64(kv.view(np.uint16))
+    out = {}
+    for r in rows:
+        n = int(rp[r]) + 1
+        K = np.concatenate([kvf[pt[rs[r], p], 0] for p in range((n + 63) // 64)], axis=1)[:, :n]   # [H, n, 64]
+        V = np.concatenate([kvf[pt[rs[r], p], 1] for p in range((n + 63) // 64)], axis=1)[:, :n]
+        o = np.empty(H * 64)
+        for h in range(H):
+            s = K[h] @ q[r, h * 64:(h + 1) * 64].astype(np.float64) / 8.0
+            o[h * 64:(h + 1) * 64] = O.softmax(s) @ V[h]
+        out[r] = o
+    return out
+
+
 def test_static_scratch_attention_matches_caller_scratch_attention_twice():
     # first case: several chunks per row, so partials and tickets are really used
     a = _case(1, 20, [900, 2048, 257, 64, 1])
@@ -54,6 +70,11 @@ def test_static_scratch_attention_matches_caller_scratch_attention_twice():
         # same kernel, same inputs: the tolerance the attention parity tests use (half a bf16 ulp
         # of the largest output plus fp32 noise) is met with room to spare — equality is expected
         assert np.max(np.abs(g - w)) <= 2.0 ** -8 * np.abs(w).max() + 1e-5
+    # against the definition itself, not only against the sibling entry point
+    got = B.bf16_bits_tensor_to_f32(B.op_attention_static(*a)).cpu().numpy().astype(np.float64)
+    torch.cuda.synchronize()
+    for r, ref in _reference(a, 20, [0, 1, 4]).items():
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, r
     # and once more on the first case, after the second has dirtied the array
     got = B.op_attention_static(*a)
     want = B.op_attention(*a)
@@ -68,8 +89,15 @@ def test_static_scratch_attention_rejects_sizes_beyond_its_limit():
         B.op_attention_static(q, kv, pt, rs, rp)
     assert e.value.code == B.E_WORKSPACE
     assert "1280" in str(e.value)
-    q, kv, pt, rs, rp = _case(4, 20, [10] * 64)            # exactly at the limit
-    got = B.op_attention_static(q, kv, pt, rs, rp)
-    want = B.op_attention(q, kv, pt, rs, rp)
+    # exactly at the limit, with several chunks in the first and the last row: the last partial slots and
+    # the last ticket of the built-in array are used
+    ctxs = [10] * 64
+    ctxs[0], ctxs[63], ctxs[31] = 700, 1030, 300
+    args = _case(4, 20, ctxs)
+    got = B.op_attention_static(*args)
+    want = B.op_attention(*args)
     torch.cuda.synchronize()
     assert torch.equal(got, want)
+    g = B.bf16_bits_tensor_to_f32(got).cpu().numpy().astype(np.float64)
+    for r, ref in _reference(args, 20, [0, 63]).items():
+        assert np.max(np.abs(g[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5, r
