@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Decode-throughput bench of the GPT decode step: batch 1, 16 and 128 in one invocation.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workloads 2,3,4,5,5w4] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workloads 2,3,4,5,5w4,5k8] [--impl ours|reference]
 
 A step is one tts_gpt_decode_step over the workload's batch of streams (the whole hot path: page
 allocation, embed, 24 blocks, final LayerNorm, LM head, sampling).  The first workload of the list is
@@ -36,8 +36,10 @@ METRIC = "GPT decode tokens/s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0          # the "about 8 TB/s" the target statement quotes
 TARGET_FRAC = 0.70                # of the HBM roofline at batch 1-16
-WORKLOAD_KEYS = {"1": (1, None), "2": (2, None), "3": (3, None), "4": (4, None), "5": (5, None),
-                 "5w8": (5, C.W_INT8_PC), "5w4": (5, C.W_INT4_G128)}
+# key -> (workload, weight format override, KV cache format)
+WORKLOAD_KEYS = {"1": (1, None, C.KV_BF16), "2": (2, None, C.KV_BF16), "3": (3, None, C.KV_BF16), "4": (4, None, C.KV_BF16),
+                 "5": (5, None, C.KV_BF16), "5w8": (5, C.W_INT8_PC, C.KV_BF16), "5w4": (5, C.W_INT4_G128, C.KV_BF16),
+                 "4k8": (4, None, C.KV_FP8_E4M3), "5k8": (5, None, C.KV_FP8_E4M3), "5w4k8": (5, C.W_INT4_G128, C.KV_FP8_E4M3)}
 DTYPE = {C.W_BF16: "bf16", C.W_INT8_PC: "bf16 activations x int8 weights (fp32 accumulate)",
          C.W_INT4_G128: "bf16 activations x int4 weights (fp32 accumulate)"}
 
@@ -60,7 +62,8 @@ def algorithmic_bytes_per_step(cfg: C.GPTConfig, ctx_before):
         w = n_lin // 2 + n_lin // 128 * 2
     small = (3 * d + d + F + d) * 2 + 4 * d * 2           # biases + LN per layer
     weights = L * (w + small) + V * d * 2 + 2 * d * 2
-    kv_per_tok = 2 * d * 2 * L
+    # per cached token: K and V rows of every layer, bf16, or e4m3 codes with one fp32 scale per head
+    kv_per_tok = (2 * d * 2 * L) if cfg.kv_fmt == C.KV_BF16 else (2 * cfg.n_head * (cfg.head_dim + 4) * L)
     kv = sum((c + 1) * kv_per_tok for c in ctx_before)
     return weights + kv + len(ctx_before) * V * 4
 
@@ -158,8 +161,8 @@ def run_workload(key, args, wcache, device, local, world, peaks):
     from paper_2607_21042_b200 import binding as B
     from paper_2607_21042_b200 import replicas as R
 
-    idx, wfmt = WORKLOAD_KEYS[key]
-    wl = C.workload(idx, wfmt=wfmt)
+    idx, wfmt, kv_fmt = WORKLOAD_KEYS[key]
+    wl = C.workload(idx, wfmt=wfmt, kv_fmt=kv_fmt)
     cfg = wl.cfg
     S = wl.n_streams
     W = max(args.warmup, 3)
@@ -289,7 +292,8 @@ def run_workload(key, args, wcache, device, local, world, peaks):
         roofline["target_met"] = bool(gbs / hbm_peak >= TARGET_FRAC)
 
     entry = {
-        "workload": wl.name, "batch": S, "weights": C.WFMT_NAMES[cfg.wfmt], "dtype": DTYPE[cfg.wfmt],
+        "workload": wl.name, "batch": S, "weights": C.WFMT_NAMES[cfg.wfmt], "kv_cache": C.KV_NAMES[cfg.kv_fmt],
+        "dtype": DTYPE[cfg.wfmt],
         "value": value, "unit": UNIT, "ms_per_step": ms / max(steps_done, 1),
         "steps": K, "repetitions": reps, "timed_steps": steps_done, "timed_ms": ms, "tokens": tokens,
         "gpu_launches": int(launches), "roofline": roofline,
@@ -519,8 +523,8 @@ def run_reference(args):
     if rank != 0:
         return
     key = [k.strip() for k in args.workloads.split(",") if k.strip()][0]
-    idx, wfmt = WORKLOAD_KEYS[key]
-    wl = C.workload(idx, wfmt=wfmt)
+    idx, wfmt, kv_fmt = WORKLOAD_KEYS[key]
+    wl = C.workload(idx, wfmt=wfmt, kv_fmt=kv_fmt)
     steps = max(1, min(args.steps, 400))
     w = C.make_weights(wl.cfg, seed=wl.seed)
     ctx = mid_context(wl)
@@ -568,8 +572,9 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workloads", default="2,3,4,5,5w4",
-                    help="comma list of 1,2,3,4,5,5w8,5w4; the first is the headline of the JSON line")
+    ap.add_argument("--workloads", default="2,3,4,5,5w4,5k8",
+                    help="comma list of 1,2,3,4,5,5w8,5w4 and, on the 8-bit KV cache, 4k8,5k8,5w4k8; the first is the "
+                         "headline of the JSON line")
     ap.add_argument("--workload", default=None, help="shorthand for --workloads with one entry")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="lower bound of each workload's timed region")
     ap.add_argument("--max-reps", type=int, default=200)

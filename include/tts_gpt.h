@@ -36,6 +36,9 @@ extern "C" {
 
 typedef struct tts_gpt tts_gpt_t; /* opaque */
 
+/* Storage format of the KV cache (config field kv_fmt). */
+enum { TTS_GPT_KV_BF16 = 0, TTS_GPT_KV_FP8_E4M3 = 1 };
+
 /* Storage format of the four block linears (QKV, attention out, FC1, FC2).  Embeddings,
  * LayerNorm parameters, biases and the LM head are bf16 in every format. */
 enum {
@@ -70,6 +73,9 @@ typedef struct {
   float ln_eps;          /* LayerNorm epsilon (inside the square root) */
   int32_t emb_rows;      /* rows of tok_emb: the merged embedding table of Section II-C holds the semantic
                             codes first and the text ids after them; 0 = vocab (no text region) */
+  int32_t kv_fmt;        /* KV cache: TTS_GPT_KV_BF16, or TTS_GPT_KV_FP8_E4M3 (beyond the precisions of Table I: every
+                            cached token and head keeps its 64 K (and V) values as e4m3 codes with one fp32 scale
+                            s = max|x| / 448; a page then takes 4352 instead of 8192 bytes per head and K|V) */
 } tts_gpt_config_t;
 
 /* All DEVICE pointers, read only during tts_gpt_create (the library keeps its own re-laid-out

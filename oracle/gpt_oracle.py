@@ -10,7 +10,7 @@ range of the position table) and what it must return at every step (token id, lo
 hidden state of the last layer); the caption of Table I and Section III-B state that W8A16 /
 W4A16 weight-only quantization is applied to it.  The paper prints no dimensions, equations or
 worked numbers for the network, so the block below is the textbook pre-LayerNorm GPT-2 block in
-fp64 with the readings listed in the design notes (LN eps 1e-5 inside the square root with
+fp64 with these readings (LN eps 1e-5 inside the square root with
 biased variance, tanh-GELU, bias on every linear, rows [Q;K;V] head-major, scale 1/sqrt(head_dim),
 causal mask, untied LM head, hidden = output of the final LayerNorm).
 
@@ -29,6 +29,7 @@ import math
 import numpy as np
 
 W_BF16, W_INT8_PC, W_INT4_G128 = 0, 1, 2
+KV_BF16, KV_FP8_E4M3 = 0, 1
 
 
 # ---------------------------------------------------------------------------------------------
@@ -84,6 +85,59 @@ def dequant(wfmt: int, w, s) -> np.ndarray:
 
 
 # ---------------------------------------------------------------------------------------------
+# 8-bit KV cache (a precision variant beyond Table I: the cached K and V rows as e4m3 codes)
+# ---------------------------------------------------------------------------------------------
+E4M3_MAX = 448.0
+
+
+def e4m3_decode(code: int) -> float:
+    """Value of an OCP e4m3 code (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities,
+    S.1111.111 is NaN): the format's definition, bit by bit."""
+    code = int(code) & 0xFF
+    sign = -1.0 if code & 0x80 else 1.0
+    e, m = (code >> 3) & 0xF, code & 0x7
+    if e == 0xF and m == 0x7:
+        return float("nan")
+    if e == 0:
+        return sign * (m / 8.0) * 2.0 ** -6          # subnormal
+    return sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+
+
+def e4m3_round(x: np.ndarray) -> np.ndarray:
+    """Nearest e4m3 value (ties to the even mantissa), saturating at +-448: the grid spacing is 2^(e-3)
+    for 2^e <= |x| < 2^(e+1), e clamped below at -6 (subnormal spacing 2^-9)."""
+    x = np.asarray(x, dtype=np.float64)
+    a = np.minimum(np.abs(x), E4M3_MAX)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.clip(e, -6, 8)
+    step = 2.0 ** (e - 3)
+    q = np.rint(a / step) * step                     # numpy rounds half to even; a / step is exact
+    return np.sign(x) * np.minimum(q, E4M3_MAX)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Nearest bf16 value (ties to even) of each entry, returned as float64."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(np.float64)
+
+
+def kv_quant_dequant(row: np.ndarray, head_dim: int) -> np.ndarray:
+    """What an e4m3 KV cache returns for a K or V row [d].  The row is first rounded to bf16 (what the
+    16-bit cache would hold); every head's head_dim values then share one scale s = max|x| / 448 (1 if the
+    slice is zero), each value is stored as the e4m3 code nearest to x / s and read back as code * s.
+    Which code represents a value is a decision taken in one precision on both sides of a comparison:
+    scale and quotient are formed in fp32, as a kernel forms them."""
+    row = np.asarray(row, dtype=np.float64)
+    x = bf16_round(row).astype(np.float32).reshape(-1, head_dim)
+    amax = np.abs(x).max(axis=1, keepdims=True)
+    s = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    q = (x / s).astype(np.float32)
+    return (e4m3_round(q.astype(np.float64)) * s.astype(np.float64)).reshape(row.shape)
+
+
+# ---------------------------------------------------------------------------------------------
 # elementwise pieces
 # ---------------------------------------------------------------------------------------------
 def layer_norm(x: np.ndarray, g: np.ndarray, b: np.ndarray, eps: float) -> np.ndarray:
@@ -125,6 +179,7 @@ class OracleModel:
         self.n_layer = int(c["n_layer"]); self.d = int(c["d_model"]); self.n_head = int(c["n_head"])
         self.head_dim = int(c["head_dim"]); self.d_ff = int(c["d_ff"]); self.vocab = int(c["vocab"])
         self.eps = float(c["ln_eps"]); self.gelu_is_tanh = bool(c["gelu_tanh"])
+        self.kv_fmt = int(c.get("kv_fmt", KV_BF16))
         wfmt = int(c["wfmt"])
         assert self.n_head * self.head_dim == self.d
         f = bf16_to_f64
@@ -144,6 +199,10 @@ class OracleModel:
 
     def gelu(self, x):
         return gelu_tanh(x) if self.gelu_is_tanh else gelu_erf(x)
+
+    def cached(self, row):
+        """A K or V row as the cache hands it back: unchanged, or through the e4m3 encoding."""
+        return kv_quant_dequant(row, self.head_dim) if self.kv_fmt == KV_FP8_E4M3 else row
 
     def token_row(self, token: int, pos: int) -> np.ndarray:
         """Input row of a generated token: its embedding plus the positional embedding of its
@@ -185,7 +244,7 @@ class OracleStream:
             a = layer_norm(x, lay["ln1_g"], lay["ln1_b"], m.eps)
             z = lay["qkv_w"] @ a + lay["qkv_b"]
             q, kt, vt = z[0:m.d], z[m.d:2 * m.d], z[2 * m.d:3 * m.d]
-            self.k[l].append(kt); self.v[l].append(vt)
+            self.k[l].append(m.cached(kt)); self.v[l].append(m.cached(vt))
             K = np.stack(self.k[l]); V = np.stack(self.v[l])          # [t+1, d]
             o = np.empty(m.d)
             for h in range(H):
@@ -218,6 +277,9 @@ def forward_full(model: OracleModel, X: np.ndarray):
         a = layer_norm(x, lay["ln1_g"], lay["ln1_b"], m.eps)
         z = a @ lay["qkv_w"].T + lay["qkv_b"]
         q, k, v = z[:, 0:m.d], z[:, m.d:2 * m.d], z[:, 2 * m.d:3 * m.d]
+        if m.kv_fmt == KV_FP8_E4M3:
+            k = np.stack([m.cached(k[t]) for t in range(T)])
+            v = np.stack([m.cached(v[t]) for t in range(T)])
         o = np.empty((T, m.d))
         for h in range(H):
             sl = slice(h * hd, (h + 1) * hd)

@@ -42,7 +42,7 @@ class ConfigStruct(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_layer", "d_model", "n_head", "head_dim", "d_ff", "vocab", "wfmt", "max_streams",
                  "max_context", "page_tokens", "n_pages", "max_pos", "gelu_tanh", "stop_token")] + \
-               [("ln_eps", C.c_float), ("emb_rows", C.c_int32)]
+               [("ln_eps", C.c_float), ("emb_rows", C.c_int32), ("kv_fmt", C.c_int32)]
 
 
 _PP = C.POINTER(C.c_void_p)

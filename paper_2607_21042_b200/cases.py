@@ -21,6 +21,9 @@ import numpy as np
 W_BF16, W_INT8_PC, W_INT4_G128 = 0, 1, 2
 WFMT_NAMES = {W_BF16: "bf16", W_INT8_PC: "w8a16", W_INT4_G128: "w4a16"}
 
+KV_BF16, KV_FP8_E4M3 = 0, 1
+KV_NAMES = {KV_BF16: "bf16", KV_FP8_E4M3: "e4m3"}
+
 TAG_WEIGHTS, TAG_PREFIX, TAG_UNIFORMS, TAG_LENGTHS = 1, 2, 3, 4
 
 
@@ -42,6 +45,7 @@ class GPTConfig:
     stop_token: int = -1
     ln_eps: float = 1e-5
     emb_rows: int = 0       # rows of the merged embedding table (semantic codes, then text ids); 0 = vocab
+    kv_fmt: int = 0         # KV cache: 0 = bf16, 1 = e4m3 codes with one scale per cached row and head
 
     @property
     def n_emb_rows(self) -> int:
@@ -265,8 +269,12 @@ def draw_lengths(n_streams, p_lo, p_hi, n_lo=None, n_hi=None, max_context=2048, 
     return tuple(int(x) for x in p), tuple(n)
 
 
-def workload(idx: int, wfmt=None, seed: int = 0) -> Workload:
-    """The five workloads (1-based, in the order the baseline lists them)."""
+def workload(idx: int, wfmt=None, seed: int = 0, kv_fmt: int = KV_BF16) -> Workload:
+    """The five workloads (1-based, in the order the baseline lists them).  kv_fmt = KV_FP8_E4M3 gives the
+    same workload on an 8-bit KV cache."""
+    if kv_fmt != KV_BF16:
+        wl = workload(idx, wfmt=wfmt, seed=seed)
+        return replace(wl, name=wl.name + "_kv" + KV_NAMES[kv_fmt], cfg=replace(wl.cfg, kv_fmt=kv_fmt))
     if idx == 1:
         cfg = tiny_config(max_streams=1, n_pages=32)
         return Workload("cfg1_tiny_bf16_b1", cfg, (64,), (32,), 0, seed=seed)

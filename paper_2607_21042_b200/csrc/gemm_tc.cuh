@@ -211,6 +211,7 @@ struct GemmTcArgs {
   void *out_img;            // EPI_GELU: activation image of the next linear (row length N)
   int gelu_tanh;
   uint16_t *kv_layer;
+  uint16_t *kv_stage;       // if set, K/V rows go here as bf16 [B][2][d] instead of into their page slots (8-bit KV cache)
   const int *page_table, *row_stream, *row_pos;
   int pps, d, H;
   int *err;
@@ -272,9 +273,13 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     const int b = bc * kTcChunkN + bl;
     uint16_t *p = nullptr;
     if (b < a.B) {
-      const int pos = a.row_pos[b];
-      const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
-      p = a.kv_layer + ((size_t)page * 2 * a.H) * kPageElems + (size_t)(pos & 63) * kHeadDim;
+      if (a.kv_stage) {
+        p = a.kv_stage + (size_t)b * 2 * a.d;
+      } else {
+        const int pos = a.row_pos[b];
+        const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
+        p = a.kv_layer + ((size_t)page * 2 * a.H) * kPageElems + (size_t)(pos & 63) * kHeadDim;
+      }
     }
     kv_base[bl] = p;
   }
@@ -425,7 +430,7 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
     } else if (a.mode == EPI_QKV && n >= a.d) {
       const int which = n >= 2 * a.d;
       const int col = n - (which ? 2 * a.d : a.d);
-      const size_t off = ((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63);
+      const size_t off = a.kv_stage ? (size_t)which * a.d + col : ((size_t)which * a.H + (col >> 6)) * kPageElems + (col & 63);
 #pragma unroll
       for (int c = 0; c < kTcEpiCols; ++c)
         if (c < nb) kv_base[c0 + c][off] = float_to_bf16_bits(v[c]);

@@ -140,6 +140,7 @@ struct LinearArgs {
   int gelu_tanh;
   // EPI_QKV: rows [0,d) -> q (fp32), [d,2d) -> K pages, [2d,3d) -> V pages
   uint16_t *kv_layer;
+  uint16_t *kv_stage;         // if set, K/V rows go here as bf16 [B][2][d] instead of into their page slots (8-bit KV cache)
   const int *page_table, *row_stream, *row_pos;
   int pps, d, H;
   unsigned long long *trace;  // optional timeline trace (see trace_mark)
@@ -245,10 +246,14 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
     if (a.mode == EPI_QKV && en >= a.d && en < a.N && b < a.B && b < 16) {
       const int which = en >= 2 * a.d;  // 0 = K, 1 = V
       const int col = en - (which ? 2 * a.d : a.d);
-      const int pos = a.row_pos[b];
-      const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
-      kv_dst[e] = a.kv_layer + (((size_t)page * 2 + which) * a.H + (col >> 6)) * kPageElems +
-                  (size_t)(pos & 63) * kHeadDim + (col & 63);
+      if (a.kv_stage) {
+        kv_dst[e] = a.kv_stage + ((size_t)b * 2 + which) * a.d + col;
+      } else {
+        const int pos = a.row_pos[b];
+        const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
+        kv_dst[e] = a.kv_layer + (((size_t)page * 2 + which) * a.H + (col >> 6)) * kPageElems +
+                    (size_t)(pos & 63) * kHeadDim + (col & 63);
+      }
     }
   }
   uint2 ln_gg = make_uint2(0, 0), ln_bb = make_uint2(0, 0);
@@ -568,10 +573,14 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
             const int which = n >= 2 * a.d;  // 0 = K, 1 = V
             const int col = n - (which ? 2 * a.d : a.d);
             const int head = col >> 6, ee = col & 63;
-            const int pos = a.row_pos[b];
-            const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
-            a.kv_layer[(((size_t)page * 2 + which) * a.H + head) * kPageElems + (size_t)(pos & 63) * kHeadDim + ee] =
-                float_to_bf16_bits(v);
+            if (a.kv_stage) {
+              a.kv_stage[((size_t)b * 2 + which) * a.d + col] = float_to_bf16_bits(v);
+            } else {
+              const int pos = a.row_pos[b];
+              const int page = a.page_table[(size_t)a.row_stream[b] * a.pps + (pos >> 6)];
+              a.kv_layer[(((size_t)page * 2 + which) * a.H + head) * kPageElems + (size_t)(pos & 63) * kHeadDim + ee] =
+                  float_to_bf16_bits(v);
+            }
           }
         }
       }

@@ -20,6 +20,7 @@
 #include "gemm_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
+#include "kv_fp8.cuh"
 
 using namespace ttsgpt;
 
@@ -53,7 +54,10 @@ struct tts_gpt {
   std::vector<LayerW> layers;
   // KV pool
   uint16_t *kv;
-  size_t kv_layer_elems;
+  size_t kv_layer_elems;      // 16-bit units of one layer's slice of the pool
+  size_t kv_page_elems;       // ... of one page in one layer
+  bool kv_fp8 = false;        // e4m3 pages with a scale per cached row and head
+  uint16_t *kv_stage = nullptr;   // 8-bit cache: the pass's new K/V rows as bf16 [kMaxRows][2][d], encoded by kv_quantize_kernel
   // state
   PageState ps;
   RowTable rt;
@@ -133,6 +137,7 @@ int check_config(const tts_gpt_config_t *c) {
   if (c->n_pages < 1 || c->max_pos < 1) return fail(nullptr, TTS_GPT_E_ARG, "n_pages and max_pos must be positive");
   if (!(c->ln_eps > 0.f)) return fail(nullptr, TTS_GPT_E_ARG, "ln_eps must be positive");
   if (c->emb_rows != 0 && c->emb_rows < c->vocab) return fail(nullptr, TTS_GPT_E_ARG, "emb_rows must be 0 or at least vocab");
+  if (c->kv_fmt != TTS_GPT_KV_BF16 && c->kv_fmt != TTS_GPT_KV_FP8_E4M3) return fail(nullptr, TTS_GPT_E_ARG, "unknown KV cache format");
   return TTS_GPT_OK;
 }
 
@@ -183,7 +188,9 @@ size_t carve(tts_gpt *h, void *base) {
     carve_linear(cv, L.fc1, c.wfmt, F, d);
     carve_linear(cv, L.fc2, c.wfmt, d, F);
   }
-  h->kv_layer_elems = (size_t)c.n_pages * 2 * c.n_head * kPageElems;
+  h->kv_fp8 = c.kv_fmt == TTS_GPT_KV_FP8_E4M3;
+  h->kv_page_elems = (size_t)2 * c.n_head * (h->kv_fp8 ? (size_t)kFp8BlockBytes / 2 : (size_t)kPageElems);   // 16-bit units of a page in one layer
+  h->kv_layer_elems = (size_t)c.n_pages * h->kv_page_elems;
   h->canary_lo = cv.take<unsigned char>(kCanaryBytes);
   h->kv = cv.take<uint16_t>(h->kv_layer_elems * c.n_layer);
   h->canary_hi = cv.take<unsigned char>(kCanaryBytes);
@@ -221,6 +228,7 @@ size_t carve(tts_gpt *h, void *base) {
   h->o = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->hbuf = cv.take<uint16_t>((size_t)kMaxRows * F);
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
+  h->kv_stage = h->kv_fp8 ? cv.take<uint16_t>((size_t)kMaxRows * 2 * d) : nullptr;
   h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
   h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
   h->have_tc = true;
@@ -274,6 +282,20 @@ void trace_attach(tts_gpt *h, Args &a) {
 // Attention for R rows: clusters while (row, head) pairs are scarce, one streaming CTA per pair
 // once they cover the GPU several times.
 cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool pdl) {
+  if (h->kv_fp8) {
+    // 8-bit cache: the QKV linear left the new K/V rows in the staging area; encode them into their page
+    // slots, then attend over e4m3 pages (the same kernel for prefill passes and decode steps)
+    unsigned char *kvl = reinterpret_cast<unsigned char *>(const_cast<uint16_t *>(aa.kv_layer));
+    cudaError_t e = launch_kv_quantize(h->kv_stage, kvl, aa.page_table, aa.row_stream, aa.row_pos, aa.pps, aa.H, R, st, pdl);
+    if (e != cudaSuccess) return e;
+    h->launches += 1;
+    Fp8AttnArgs fa;
+    memset(&fa, 0, sizeof fa);
+    fa.q = aa.q; fa.kv_layer = kvl; fa.page_table = aa.page_table; fa.row_stream = aa.row_stream; fa.row_pos = aa.row_pos;
+    fa.out = aa.out; fa.partials = h->attn_partials; fa.tickets = h->attn_tickets; fa.H = aa.H; fa.pps = aa.pps;
+    fa.out_image = aa.out_image; fa.trace = aa.trace; fa.trace_slot = aa.trace_slot;
+    return launch_attention_fp8(fa, R, attention_fp8_splits(R, aa.H, h->n_sm), st, pdl);
+  }
   aa.err = h->dev_err;
   aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
   // prefill passes: rows of one stream share their pages (one CTA per 16 rows and head on the tensor cores;
@@ -328,6 +350,7 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+    qa.kv_stage = h->kv_stage;
     trace_attach(h, qa);
     CUDA_TRY(h, launch_gemm_tc(qa, st, pdl));
     AttnArgs aa;
@@ -420,6 +443,7 @@ int run_layers(tts_gpt *h, int R, bool decode) {
       }
       qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
       qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
+      qa.kv_stage = h->kv_stage;
       trace_attach(h, qa);
       CUDA_TRY(h, launch_linear(c.wfmt, qa, st, pdl, 2 * h->n_sm));
       AttnArgs aa;
@@ -855,7 +879,7 @@ int32_t tts_gpt_release_stream(tts_gpt_t *h, int32_t s) {
   if (h->poison_free) {   // before the pages go back: the page table row still names them
     const int np = (h->ctx[s] + 63) / 64;
     if (np > 0)
-      poison_pages_kernel<<<256, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, (size_t)2 * h->cfg.n_head * kPageElems,
+      poison_pages_kernel<<<256, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, h->kv_page_elems,
                                                       h->ps.page_table + (size_t)s * h->pps, nullptr, np);
   }
   release_kernel<<<1, 32, 0, h->stream>>>(h->ps, s);
@@ -973,7 +997,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "poison_free_pages") {
     h->poison_free = on;
     if (on && h->n_free > 0) {   // every page that is free right now
-      poison_pages_kernel<<<1024, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, (size_t)2 * h->cfg.n_head * kPageElems,
+      poison_pages_kernel<<<1024, 256, 0, h->stream>>>(h->kv, h->kv_layer_elems, h->cfg.n_layer, h->kv_page_elems,
                                                        nullptr, h->ps.free_list, h->n_free);
       CUDA_TRY(h, cudaGetLastError());
     }

@@ -13,6 +13,16 @@ GAP = 3e-2
 # top-k: a mismatch is excused when u is within this distance of an oracle CDF boundary
 # ((e^{2*0.03} - 1)/2: both neighbouring weights can move by a factor e^{+-0.03})
 CDF_MARGIN = 0.031
+# 8-bit (e4m3) KV cache.  The encoding is a step function of the K/V values, and the two sides reach those
+# values through different rounding histories (relative difference about 1e-3, the same that gives the
+# 16-bit cache its 0.5 % logit error): one to two percent of the cached codes land one step apart (6-12 % of
+# the value).  Over the 24 layers this adds, in quadrature, about as much logit error again as the bf16
+# operands cause (0.09 x sqrt(0.015 / 50 attended tokens) = 0.16 % of an attention output per layer), so the
+# bar is the usual one times 1.5; below 32 attended tokens the flips do not average out (1.1 % of the
+# attention output with a single token) and the relative bar is 2.5e-2.
+E4M3_MAX_ABS = 4.5e-2
+E4M3_REL_L2 = 1.5e-2
+E4M3_REL_L2_SHORT = 2.5e-2
 
 
 def bits_dev(arr, device="cuda:0"):
@@ -34,10 +44,10 @@ def logits_errors(gpu: np.ndarray, ref: np.ndarray):
     return max_abs, float(np.max(rel))
 
 
-def assert_logits_close(gpu, ref, what=""):
+def assert_logits_close(gpu, ref, what="", max_abs_bar=LOGIT_MAX_ABS, rel_bar=LOGIT_REL_L2):
     max_abs, rel = logits_errors(gpu, ref)
-    assert max_abs <= LOGIT_MAX_ABS, "%s: logits max-abs error %.4g > %.3g" % (what, max_abs, LOGIT_MAX_ABS)
-    assert rel <= LOGIT_REL_L2, "%s: logits relative L2 error %.4g > %.3g" % (what, rel, LOGIT_REL_L2)
+    assert max_abs <= max_abs_bar, "%s: logits max-abs error %.4g > %.3g" % (what, max_abs, max_abs_bar)
+    assert rel <= rel_bar, "%s: logits relative L2 error %.4g > %.3g" % (what, rel, rel_bar)
     return max_abs, rel
 
 

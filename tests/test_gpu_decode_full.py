@@ -8,7 +8,8 @@ import torch
 from oracle import gpt_oracle as O
 from paper_2607_21042_b200 import binding as B
 from paper_2607_21042_b200 import cases as C
-from helpers import assert_logits_close, assert_same_up_to_ties, bits_dev, check_tokens, gpu_run_stream
+from helpers import (E4M3_MAX_ABS, E4M3_REL_L2, assert_logits_close, assert_same_up_to_ties, bits_dev, check_tokens,
+                     gpu_run_stream)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -16,14 +17,14 @@ DEV = "cuda:0"
 _cache = {}
 
 
-def _model(wfmt):
+def _model(wfmt, kv_fmt=C.KV_BF16):
     """Weights of the full model in one format (drawn once per session) and its oracle."""
-    if wfmt not in _cache:
+    if (wfmt, kv_fmt) not in _cache:
         _cache.clear()              # one fp64 model (3.9 GB) at a time
-        cfg = C.full_config(wfmt=wfmt)
+        cfg = C.full_config(wfmt=wfmt, kv_fmt=kv_fmt)
         w = C.make_weights(cfg, seed=0)
-        _cache[wfmt] = (w, O.OracleModel(cfg, w))
-    return _cache[wfmt]
+        _cache[(wfmt, kv_fmt)] = (w, O.OracleModel(cfg, w))
+    return _cache[(wfmt, kv_fmt)]
 
 
 def _batch_run(eng, wl, prefixes, n_steps, decode_lens=None):
@@ -63,9 +64,9 @@ def _batch_run(eng, wl, prefixes, n_steps, decode_lens=None):
         out.append((np.array(seq), lgs))
     return out
 
-def _workload5(wfmt):
-    wl = C.workload(5, wfmt=wfmt)
-    w, model = _model(wfmt)
+def _workload5(wfmt, kv_fmt=C.KV_BF16):
+    wl = C.workload(5, wfmt=wfmt, kv_fmt=kv_fmt)
+    w, model = _model(wfmt, kv_fmt)
     eng = B.TtsGpt(wl.cfg, w, DEV)
     prefixes = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)
     # shorten the drain so the test stays in minutes: every stream leaves after min(n_i, cap) steps
@@ -79,17 +80,19 @@ def _workload5(wfmt):
         seq, lg = res[i]
         assert len(seq) == dl[i] + 1
         ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
-        ma, rl = assert_logits_close(lg, ref, "workload 5 stream %d" % i)
+        bars = {} if kv_fmt == C.KV_BF16 else dict(max_abs_bar=E4M3_MAX_ABS, rel_bar=E4M3_REL_L2)
+        ma, rl = assert_logits_close(lg, ref, "workload 5 stream %d" % i, **bars)
         exc = check_tokens(seq, ref, 0, 1.0, None, "workload 5 stream %d" % i)
-        print("workload5[%s] stream %d (P=%d, n=%d): max-abs %.4g rel-L2 %.4g excused %d" % (
-            C.WFMT_NAMES[wfmt], i, wl.prefix_lens[i], dl[i], ma, rl, exc))
+        print("workload5[%s, KV %s] stream %d (P=%d, n=%d): max-abs %.4g rel-L2 %.4g excused %d" % (
+            C.WFMT_NAMES[wfmt], C.KV_NAMES[kv_fmt], i, wl.prefix_lens[i], dl[i], ma, rl, exc))
     # batch invariance for two streams the oracle did not replay
     for i in (5, 64):
         if i in picks:
             continue
         alone = _batch_run(eng, wl, [prefixes[i]], 24)[0]
         m = min(25, len(res[i][0]))
-        assert_same_up_to_ties(alone[0][:m], alone[1][:m], res[i][0][:m], res[i][1][:m], "batch invariance stream %d" % i)
+        assert_same_up_to_ties(alone[0][:m], alone[1][:m], res[i][0][:m], res[i][1][:m], "batch invariance stream %d" % i,
+                               **({} if kv_fmt == C.KV_BF16 else dict(tol=E4M3_MAX_ABS)))
     eng.destroy()
 
 def test_workload2_bf16_batch1_replay():
@@ -215,3 +218,25 @@ def test_workload5_w4a16_batch128_ragged_drain():
 
 def test_workload5_w8a16_batch128_ragged_drain():
     _workload5(C.W_INT8_PC)
+
+
+def test_workload5_bf16_weights_e4m3_kv_cache():
+    """Batch 128 on the 8-bit KV cache: contexts of 200 and more, where the parity bar is the usual one."""
+    _workload5(C.W_BF16, C.KV_FP8_E4M3)
+
+
+def test_workload4_w4a16_e4m3_kv_cache():
+    wl = C.workload(4, kv_fmt=C.KV_FP8_E4M3)
+    w, model = _model(C.W_INT4_G128, C.KV_FP8_E4M3)
+    eng = B.TtsGpt(wl.cfg, w, DEV)
+    prefixes = C.make_prefixes(wl.cfg, wl.prefix_lens, seed=0)
+    n = 60
+    res = _batch_run(eng, wl, prefixes, n)
+    lens = list(wl.prefix_lens)
+    for i in sorted({int(np.argmin(lens)), int(np.argmax(lens))}):
+        seq, lg = res[i]
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[i]), seq[:-1])
+        ma, rl = assert_logits_close(lg, ref, "workload 4 (e4m3 KV) stream %d" % i, max_abs_bar=E4M3_MAX_ABS, rel_bar=E4M3_REL_L2)
+        exc = check_tokens(seq, ref, 0, 1.0, None, "workload 4 (e4m3 KV) stream %d" % i)
+        print("workload4 e4m3 KV stream %d (P=%d): max-abs %.4g rel-L2 %.4g excused %d/%d" % (i, lens[i], ma, rl, exc, n + 1))
+    eng.destroy()

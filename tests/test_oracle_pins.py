@@ -492,3 +492,104 @@ def test_assembled_prefix_feeds_the_decoder_like_given_rows():
     # position matters: the same ids counted from another text position give other logits
     other = O.run_stream(m, O.assemble_prefix(m, cond, [1, 5, 0, 2], shift, 10), 3, pos0=2)
     assert np.abs(run["logits"] - other["logits"]).max() > 1e-6
+
+
+# ---------------------------------------------------------------------------------------------
+# e4m3 KV cache
+# ---------------------------------------------------------------------------------------------
+def test_e4m3_decode_matches_hand_worked_codes():
+    # sign | exponent (bias 7) | mantissa, worked by hand from the format's definition
+    assert O.e4m3_decode(0x00) == 0.0
+    assert O.e4m3_decode(0x01) == 2.0 ** -9            # smallest subnormal
+    assert O.e4m3_decode(0x07) == 7 * 2.0 ** -9
+    assert O.e4m3_decode(0x08) == 2.0 ** -6            # smallest normal
+    assert O.e4m3_decode(0x38) == 1.0
+    assert O.e4m3_decode(0x3C) == 1.5
+    assert O.e4m3_decode(0x40) == 2.0
+    assert O.e4m3_decode(0x7E) == 448.0                # largest finite: 1.75 * 2^8
+    assert O.e4m3_decode(0xBC) == -1.5
+    assert np.isnan(O.e4m3_decode(0x7F)) and np.isnan(O.e4m3_decode(0xFF))
+
+
+def test_e4m3_round_is_the_identity_on_every_code_and_nearest_elsewhere():
+    vals = np.array(sorted({O.e4m3_decode(c) for c in range(256) if not np.isnan(O.e4m3_decode(c))}))
+    assert len(vals) == 253                                     # 254 finite codes, +0 and -0 coincide
+    assert np.array_equal(O.e4m3_round(vals), vals)
+    # nearest value by brute force over the whole grid, on a dense set of points (ties excluded here)
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.uniform(-448, 448, 4000), rng.uniform(-1, 1, 4000), rng.uniform(-0.02, 0.02, 4000)])
+    near = vals[np.argmin(np.abs(x[:, None] - vals[None, :]), axis=1)]
+    assert np.array_equal(O.e4m3_round(x), near)
+    # ties go to the even mantissa: the midpoint of 1.0 (mantissa 0) and 1.125 (mantissa 1) is 1.0625 -> 1.0;
+    # the midpoint of 1.125 and 1.25 (mantissa 2) -> 1.25; same in the subnormal range
+    assert O.e4m3_round(np.array([1.0625]))[0] == 1.0
+    assert O.e4m3_round(np.array([1.1875]))[0] == 1.25
+    assert O.e4m3_round(np.array([1.5 * 2.0 ** -9]))[0] == 2.0 ** -8
+    # saturation, sign symmetry, monotonicity
+    assert O.e4m3_round(np.array([1e6, -1e6, 460.0]))[0] == 448.0 and O.e4m3_round(np.array([-1e6]))[0] == -448.0
+    xs = np.sort(x)
+    assert np.all(np.diff(O.e4m3_round(xs)) >= 0)
+    assert np.array_equal(O.e4m3_round(-x), -O.e4m3_round(x))
+
+
+def test_e4m3_round_matches_the_library_cast():
+    # torch's float8_e4m3fn cast is an independent implementation of the same rounding (in range)
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.uniform(-448, 448, 20000), rng.standard_normal(20000) * 0.05]).astype(np.float32)
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(O.e4m3_round(x.astype(np.float64)), lib)
+
+
+def test_kv_quant_dequant_scale_per_head_slice_and_error_bound():
+    rng = np.random.default_rng(2)
+    row = O.bf16_round(rng.standard_normal(4 * 64) * np.repeat([0.01, 1.0, 30.0, 1e-6], 64))   # four heads of very different size
+    y = O.kv_quant_dequant(row, 64)
+    for h in range(4):
+        x, z = row[64 * h:64 * h + 64], y[64 * h:64 * h + 64]
+        s = float(np.float32(np.abs(x).max()) / np.float32(448.0))
+        i = np.argmax(np.abs(x))
+        assert np.isclose(z[i], x[i], rtol=2.0 ** -23)                             # the largest value is kept (up to the fp32 scale)
+        # error at most half a grid step of the value's binade (relative 2^-4), or half the subnormal step
+        assert np.all(np.abs(z - x) <= np.maximum(np.abs(x) * 2.0 ** -4, s * 2.0 ** -10) * (1 + 1e-6))
+        codes = z / s
+        assert np.array_equal(O.e4m3_round(codes), codes)                          # values sit on the grid of their head
+    # scaling a head's slice by a power of two scales its decoded values exactly; other heads unchanged
+    row2 = row.copy(); row2[64:128] *= 8.0
+    y2 = O.kv_quant_dequant(row2, 64)
+    assert np.array_equal(y2[64:128], 8.0 * y[64:128]) and np.array_equal(y2[:64], y[:64])
+    assert np.array_equal(O.kv_quant_dequant(np.zeros(64), 64), np.zeros(64))
+    # the row is taken as bf16: a perturbation below half a bf16 ulp changes nothing
+    assert np.array_equal(O.kv_quant_dequant(row * (1 + 2.0 ** -12), 64), y)
+
+
+def test_bf16_round_on_hand_written_cases():
+    x = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, -3.0, 0.0, 2.0 ** -130])
+    # 1 + 2^-8 is the midpoint of 1 and 1 + 2^-7: ties to the even mantissa (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    want = np.array([1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, -3.0, 0.0, 2.0 ** -130])
+    assert np.array_equal(O.bf16_round(x), want)
+    rng = np.random.default_rng(3)
+    y = rng.standard_normal(1000)
+    r = O.bf16_round(y)
+    assert np.all(np.abs(r - y) <= np.abs(y) * 2.0 ** -8) and np.array_equal(O.bf16_round(r), r)
+
+
+def test_e4m3_cache_decoder_equals_recompute_and_plain_attention_on_decoded_rows():
+    """With the 8-bit cache, cached decode still equals the no-cache recompute, and both equal ordinary
+    attention run on explicitly encoded-and-decoded K and V rows."""
+    cfg = C.tiny_config(kv_fmt=C.KV_FP8_E4M3)
+    w = C.make_weights(cfg, seed=4)
+    model = O.OracleModel(cfg, w)
+    X = O.bf16_to_f64(C.make_prefixes(cfg, [20], seed=4)[0])
+    st = O.OracleStream(model)
+    rows = np.stack([st.step(X[t])[0] for t in range(X.shape[0])])
+    full, _ = O.forward_full(model, X)
+    assert np.max(np.abs(rows - full)) <= 1e-10
+    # the cache holds decoded rows: every cached K row is a fixed point of the encoding
+    for l in range(model.n_layer):
+        for kt in st.k[l]:
+            assert np.array_equal(O.kv_quant_dequant(kt, model.head_dim), kt)
+    # and it differs from the exact cache by what the 2^-4 relative grid allows, not more
+    plain = O.OracleModel(C.tiny_config(), w)
+    exact, _ = O.forward_full(plain, X)
+    diff = np.max(np.abs(full - exact))
+    assert 0 < diff < 0.25
