@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
   //      (mean = (ma+mb)/2, M2 = M2a + M2b + (mb-ma)^2 * n/2), first by shuffles, then across the
   //      warps through shared memory: one block barrier, no cancellation.
   const int stride = ln_stage_stride(WF, KB * KT);   // staged columns: this CTA's k-range
-  constexpr int RPR = 4;  // rows per LayerNorm round
+  constexpr int RPR = NB == 1 ? 1 : 4;  // rows per LayerNorm round (a one-row launch carries the code of one row only)
   if (LN) {
     float2 *lnred = reinterpret_cast<float2 *>(red);  // [warps][RPR] (mean, M2), reused later for the partial sums
     const int nw_used = (a.K / 4 + 31) / 32;           // warps that hold columns (K is a multiple of 128)
@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(kLinearThreads, 2) linear_kernel(const LinearA
       for (int j = 0; j < RT; ++j)
 #pragma unroll
         for (int b = 0; b < NBA; ++b) facc[j][b] = 0.f;
-#pragma unroll 4
+#pragma unroll 1   // small code matters more than overlap here: a one-row step executes most instructions once, and fetching them costs about what executing them does
       for (int kb = warp; kb < KB; kb += kLinearWarps) {
         const int col = kb * KT + t * (KT / 4);
         uint4 wq[RT];
