@@ -222,7 +222,8 @@ int32_t tts_gpt_debug_check_canaries(tts_gpt_t *h, int32_t *bad_bytes);
 /* Experiments and tests: switches a kernel schedule of this engine on or off (value 0 / 1) or sets
  * a threshold.  Defaults are what the measurements use.  Waits for the stream and drops captured
  * step graphs.  Names: "graph", "pdl", "tc" and "tc_min_rows" (tensor-core
- * linears), "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
+ * linears), "prefill_pass_rows" (128, 256, 384 or 512 rows per prefill pass; passes of more than 128 rows need
+ * the tensor-core path and bf16 pages), "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
  * "fc2_ksplit"; "poison_free_pages" (test aid standing in for a memory checker: every free page, and
  * from then on every released page, is filled with NaN in all layers, so that a kernel reading a slot no
  * token was written to poisons its result).  Unknown name or value out of range: TTS_GPT_E_ARG. */
@@ -256,8 +257,11 @@ int32_t tts_gpt_op_linear(int32_t wfmt, int32_t N, int32_t K, const void *packed
                           int32_t B, const void *act, float *out, void *cuda_stream);
 
 /* The same linear on the 5th-generation tensor cores (the engine's path for more than 16 rows):
- * w, s in the canonical formats above, K a multiple of 128, 1 <= B <= 128, ksplit 1 or 4 (4: the
- * k-range partial sums are folded in range order, as the engine's next LayerNorm does).  Quantized
+ * w, s in the canonical formats above, K a multiple of 128, 1 <= B <= 128.  ksplit 1 or 4: the
+ * kernel of decode steps and one-tile passes (chunks of 32 batch rows per CTA), over all of K or
+ * over 4 k-ranges; ksplit -1 .. -4: the kernel of prefill passes of several row tiles (128 rows x
+ * 128 features per CTA), here on one row tile, over 1 .. 4 k-ranges.  With more than one range the
+ * partial sums are folded in range order, as the engine's next LayerNorm does.  Quantized
  * codes enter the tensor cores as exact bf16 integers; scales multiply fp32 sums (per row for int8,
  * per row and 128-column group for int4).  `scratch` (1024-byte aligned, >= scratch_bytes) receives
  * the operand images. */

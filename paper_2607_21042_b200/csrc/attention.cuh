@@ -665,7 +665,7 @@ __global__ void __launch_bounds__(kAttnPrefillRows * 32, 3) attention_prefill_ke
     const uint4 y = make_uint4(pack_bf16x2(o[0] * inv, o[1] * inv), pack_bf16x2(o[2] * inv, o[3] * inv),
                                pack_bf16x2(o[4] * inv, o[5] * inv), pack_bf16x2(o[6] * inv, o[7] * inv));
     const int col = h * kHeadDim + 8 * sub;
-    if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, col)) = y;
+    if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, col, a.H * kHeadDim)) = y;
     else *reinterpret_cast<uint4 *>(a.out + (size_t)r * a.H * kHeadDim + col) = y;
   }
   trace_mark(a.trace, a.trace_slot, 2);

@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(kPrefillMmaWarps * 32) attention_prefill_mma_k
     const uint4 yy = make_uint4(pack_bf16x2(y[0] * inv, y[1] * inv), pack_bf16x2(y[2] * inv, y[3] * inv),
                                 pack_bf16x2(y[4] * inv, y[5] * inv), pack_bf16x2(y[6] * inv, y[7] * inv));
     const int col = h * kHeadDim + d0;
-    if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, col)) = yy;
+    if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, col, a.H * kHeadDim)) = yy;
     else *reinterpret_cast<uint4 *>(a.out + (size_t)r * a.H * kHeadDim + col) = yy;
   }
   trace_mark(a.trace, a.trace_slot, 2);

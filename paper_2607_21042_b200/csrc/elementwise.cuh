@@ -117,13 +117,18 @@ __host__ __device__ inline size_t act_image_offset(int row, int k) {
   return (size_t)kc * (kMaxRows * 128) + (size_t)row * 128 + (size_t)((u ^ (row & 7)) << 4) + (size_t)(k & 7) * 2;
 }
 
+// the same for passes of more than 128 rows: row tiles of 128 rows, each a complete image of a K-column matrix
+__host__ __device__ inline size_t act_image_offset_tiled(int row, int k, int K) {
+  return (size_t)(row >> 7) * (size_t)(K >> 6) * (kMaxRows * 128) + act_image_offset(row & (kMaxRows - 1), k);
+}
+
 // LayerNorm in front of a tensor-core linear.  First folds what the previous k-split linear left
 // behind into the residual stream, in a fixed order: x[r] += bias + partial[0][r] + partial[1][r] + ...
 // (written back unless `write_back` is 0), then normalises and writes the row into the activation
 // image (`out_img`) and/or a plain bf16 row (`out_plain`, row j).  With `gather`, row j is x row gather[j].
 struct LnTcArgs {
   float *x; int d;
-  const float *partials; int n_part, part_cols;   // [n_part][kMaxRows][part_cols]
+  const float *partials; int n_part, part_cols;   // [row tile][n_part][kMaxRows][part_cols]
   const uint16_t *add_bias;
   const uint16_t *g, *b; float eps;
   void *out_img; uint16_t *out_plain;
@@ -165,7 +170,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
       if (a.n_part > 0) {
 #pragma unroll
         for (int p = 0; p < kMaxPart; ++p)
-          if (p < a.n_part) pp[i][p] = __ldcg(a.partials + ((size_t)p * kMaxRows + r) * a.part_cols + c);
+          if (p < a.n_part) pp[i][p] = __ldcg(a.partials + (((size_t)(r >> 7) * a.n_part + p) * kMaxRows + (r & (kMaxRows - 1))) * a.part_cols + c);
       }
     }
   }
@@ -197,7 +202,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
     const int c = threadIdx.x + i * kLnThreads;
     if (c < a.d) {
       const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * gg[i] + bb[i]);
-      if (a.out_img) *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset(j, c)) = y;
+      if (a.out_img) *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset_tiled(j, c, a.d)) = y;
       if (a.out_plain) a.out_plain[(size_t)j * a.d + c] = y;
       if (hid) hid[c] = y;
     }

@@ -459,6 +459,315 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
   if (warp == 0) tmem_dealloc(tmem_d, 2 * kTcChunkN);
 }
 
+// ------------------------------------------------------------------------------------------
+// Wide variant for passes of more than 128 rows (prefill): all 128 rows of a row tile in one
+// instruction.
+//
+// A tcgen05.mma with M = 128 takes about 72 ns on this part whether its N extent is 32 or 128, so
+// the kernel above, whose instructions are 32 batch rows wide, wastes three quarters of each.  It
+// still wins while a pass has at most 128 rows, because it spreads a linear over four times as many
+// CTAs without any merge.  A prefill pass of several row tiles has enough independent output tiles
+// for the wide shape: here the operand roles are swapped, the activation block of a k-chunk (128
+// rows x 64 columns, 16 KB) is the M operand, a 128-row weight block the N operand, and one CTA
+// computes a whole [128 rows] x [128 output features] tile for its k-range: K/16 instructions where
+// four CTAs of the kernel above issue K/16 each, and the weights cross from L2 once per 128 rows
+// instead of once per 32.  Grid = feature tiles x k-ranges x row tiles.  Accumulator lane = row,
+// column = output feature; the epilogue parks the accumulator rows in the idle ring and writes
+// them out with the lanes along the row.  The residual linears split K over up to 4 CTAs whose
+// partial sums the next LayerNorm folds (partials [row tile][range][128][N]); the others take all
+// of K in one CTA.
+constexpr int kTwStages = 3;
+constexpr uint32_t kTwStageBytes = 2 * 16384;   // activations (M operand) | weights (N operand)
+constexpr int kTwThreads = 320;                 // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue
+constexpr int kTwMaxPartials = 4;               // k-ranges the following LayerNorm folds
+
+
+template <bool GROUPED>
+__global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a) {
+  extern __shared__ __align__(16) unsigned char tc_smem_raw[];
+  unsigned char *ring = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
+  uint64_t *full = reinterpret_cast<uint64_t *>(ring + kTwStages * kTwStageBytes);
+  uint64_t *empty = full + kTwStages;
+  uint64_t *acc_done = empty + kTwStages;
+  uint64_t *grp_done = acc_done + 1;   // [2]
+  uint64_t *grp_free = grp_done + 2;   // [2]
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(grp_free + 2);
+  volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
+  float *s_bias = reinterpret_cast<float *>(tmem_slot + 6);         // [128] bias of this tile's features (16-byte aligned)
+  float *s_rsc = s_bias + 128;                                      // [128] int8: per-feature scale, else 1
+  uint16_t **kv_base = reinterpret_cast<uint16_t **>(s_rsc + 128);  // [128] EPI_QKV: where batch row b's K/V go
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nt = blockIdx.x, ks = blockIdx.y;
+  const int row0 = blockIdx.z * kMaxRows;              // first row of this CTA's row tile
+  const int Bt = min(kMaxRows, a.B - row0);            // rows of the tile
+  trace_mark(a.trace, a.trace_slot, 0);
+  const int KC = a.K / kTcKChunk;
+  int per = (KC + a.ksplit - 1) / a.ksplit;
+  if (GROUPED) per = (per + 1) & ~1;   // k-ranges hold whole 128-column groups (2 k-chunks each)
+  const int kc0 = min(KC, ks * per), kc1 = min(KC, kc0 + per);
+  const int n_it = kc1 - kc0;
+  constexpr uint32_t kCols = GROUPED ? 256u : 128u;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kTwStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    mbar_init(acc_done, 1);
+    mbar_init(grp_done, 1); mbar_init(grp_done + 1, 1);
+    mbar_init(grp_free, kTcEpiThreads); mbar_init(grp_free + 1, kTcEpiThreads);
+    *failed = 0;
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, kCols);
+  if (threadIdx.x >= 64 && threadIdx.x < 192) {
+    const int b = threadIdx.x - 64;
+    uint16_t *p = nullptr;
+    if (a.mode == EPI_QKV && b < Bt) {
+      if (a.kv_stage) {
+        p = a.kv_stage + (size_t)(row0 + b) * 2 * a.d;
+      } else {
+        const int pos = a.row_pos[row0 + b];
+        const int page = a.page_table[(size_t)a.row_stream[row0 + b] * a.pps + (pos >> 6)];
+        p = a.kv_layer + ((size_t)page * 2 * a.H) * kPageElems + (size_t)(pos & 63) * kHeadDim;
+      }
+    }
+    kv_base[b] = p;
+  } else if (threadIdx.x >= 192) {
+    const int c = threadIdx.x - 192;
+    const int n = nt * 128 + c;
+    float rs = 1.f, bi = 0.f;
+    if (n < a.N) {
+      if (a.wfmt == WF_INT8) rs = bf16_bits_to_float(a.scales[n]);
+      if (a.bias && !(a.mode == EPI_RESID && a.ksplit > 1)) bi = bf16_bits_to_float(a.bias[n]);
+    }
+    s_rsc[c] = rs; s_bias[c] = bi;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+
+  const unsigned char *gW = reinterpret_cast<const unsigned char *>(a.w_img) + ((size_t)nt * KC + kc0) * kTcABytes;
+  const unsigned char *gX = reinterpret_cast<const unsigned char *>(a.act_img) + ((size_t)blockIdx.z * KC + kc0) * (kMaxRows * 128);
+
+  const int pre = min(n_it, kTwStages);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < pre; ++i) {   // weights do not depend on the previous kernel
+      mbar_expect_tx(full + i, kTwStageBytes);
+      bulk_copy_g2s(ring + (size_t)i * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + i);
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int i = 0; i < pre; ++i)
+        bulk_copy_g2s(ring + (size_t)i * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + i);
+      for (int i = pre; i < n_it; ++i) {
+        const int s = i % kTwStages;
+        tc_wait(empty + s, ((i / kTwStages) - 1) & 1, failed, a.err);
+        mbar_expect_tx(full + s, kTwStageBytes);
+        bulk_copy_g2s(ring + (size_t)s * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + s);
+        bulk_copy_g2s(ring + (size_t)s * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + s);
+      }
+      trace_mark(a.trace, a.trace_slot, 3);   // last copy issued
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = tc_instr_desc(128, 128);
+      for (int i = 0; i < n_it; ++i) {
+        const int s = i % kTwStages;
+        tc_wait(full + s, (i / kTwStages) & 1, failed, a.err);
+        const int g = i >> 1;
+        if (GROUPED && (i & 1) == 0 && g >= 2) tc_wait(grp_free + (g & 1), ((g >> 1) - 1) & 1, failed, a.err);
+        tc_fence_after_sync();
+        const unsigned char *sx = ring + (size_t)s * kTwStageBytes;
+        const uint64_t da = tc_smem_desc(sx), db = tc_smem_desc(sx + 16384);
+        const uint32_t dst = GROUPED ? tmem_d + (uint32_t)(g & 1) * 128u : tmem_d;
+#pragma unroll
+        for (int j = 0; j < kTcKChunk / 16; ++j) {
+          const bool fresh = GROUPED ? ((i & 1) == 0 && j == 0) : (i == 0 && j == 0);
+          tc_mma(dst, da + 2 * j, db + 2 * j, idesc, fresh ? 0u : 1u);
+        }
+        tc_commit(empty + s);
+        if (GROUPED && ((i & 1) == 1 || i == n_it - 1)) tc_commit(grp_done + (g & 1));
+      }
+      if (!GROUPED) tc_commit(acc_done);
+    }
+    __syncwarp();
+  } else {
+    // ---- epilogue: warp w may read accumulator lanes 32*(w%4)..+31 = batch rows; warps w and w+4 share a lane
+    //      quarter and take 64 of the 128 columns (output features) each ----
+    const int lw = warp & 3;
+    const int b = lw * 32 + lane;
+    const int cb = ((warp - 2) >> 2) * 64;
+    const uint32_t t_row = tmem_d + ((uint32_t)(lw * 32) << 16) + (uint32_t)cb;
+    float v[64];
+    if (GROUPED) {
+#pragma unroll
+      for (int c = 0; c < 64; ++c) v[c] = 0.f;
+      const int n_groups = (n_it + 1) >> 1;
+      const int KG = a.K / 128;
+      for (int g = 0; g < n_groups; ++g) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          // scales of this group for 32 features (tiled scales [n/8][K/128][8]: 8 features are 16 bytes); same
+          // addresses in every lane, fetched ahead of the wait
+          uint4 sc[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int n = nt * 128 + cb + hh * 32 + q * 8;
+            sc[q] = n < a.N ? __ldg(reinterpret_cast<const uint4 *>(a.scales + ((size_t)(n >> 3) * KG + (kc0 >> 1) + g) * 8))
+                            : make_uint4(0, 0, 0, 0);
+          }
+          if (hh == 0) {
+            tc_wait(grp_done + (g & 1), (g >> 1) & 1, failed, a.err);
+            tc_fence_after_sync();
+            __syncwarp();
+          }
+          float t[32];
+          tmem_ld32(t_row + (uint32_t)(g & 1) * 128u + (uint32_t)(hh * 32), t);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint32_t wds[4] = {sc[q].x, sc[q].y, sc[q].z, sc[q].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float s0 = __uint_as_float(wds[e] << 16), s1 = __uint_as_float(wds[e] & 0xffff0000u);
+              v[hh * 32 + q * 8 + 2 * e] = fmaf(s0, t[q * 8 + 2 * e], v[hh * 32 + q * 8 + 2 * e]);
+              v[hh * 32 + q * 8 + 2 * e + 1] = fmaf(s1, t[q * 8 + 2 * e + 1], v[hh * 32 + q * 8 + 2 * e + 1]);
+            }
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(grp_free + (g & 1));
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 64; ++c) v[c] = 0.f;
+      tc_wait(acc_done, 0, failed, a.err);
+      trace_mark(a.trace, a.trace_slot, 4, 64);   // accumulator complete
+      tc_fence_after_sync();
+      __syncwarp();
+      if (n_it > 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          float t[32];
+          tmem_ld32(t_row + (uint32_t)(hh * 32), t);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) v[hh * 32 + c] += t[c];
+        }
+      }
+      trace_mark(a.trace, a.trace_slot, 5, 64);   // accumulator in registers
+    }
+    {
+      // ---- out of the registers: a thread owns a batch row, but rows are kilobytes apart in every destination, so
+      //      each warp parks its 32 rows x 64 raw sums in its own patch of the (now idle) ring and a short rolled
+      //      loop writes them out with the lanes along the row, applying scale, bias and GELU on the way.  The loop
+      //      is kept small on purpose: this code runs once per CTA, from a cold instruction cache. ----
+      const int n0 = nt * 128 + cb;                 // this warp's 64 features
+      const int nv = min(64, a.N - n0);
+      const int rows = min(32, Bt - lw * 32);       // real rows of this warp
+      unsigned char *patch = ring + (size_t)(warp - 2) * (32 * 272);
+      {
+        float4 *mine = reinterpret_cast<float4 *>(patch + lane * 272);   // 256 bytes per row, pitch 272: conflict-free
+#pragma unroll
+        for (int q = 0; q < 16; ++q) mine[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      }
+      __syncwarp();
+      const bool as_bf16 = a.mode == EPI_GELU || (a.mode == EPI_QKV && n0 >= a.d);
+      const bool partial = a.mode == EPI_RESID && a.ksplit > 1;
+      const bool use_bias = a.bias && !partial;
+      if (*failed || nv <= 0) {
+        // nothing is stored after an expired wait, or for features beyond N
+      } else if (as_bf16) {
+        // four rows per instruction: lane = (row in the group of four, 16-byte unit = 8 features of the row)
+        const int r4 = lane >> 3, u = lane & 7;
+        float sc8[8], bi8[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { sc8[e] = s_rsc[cb + 8 * u + e]; bi8[e] = use_bias ? s_bias[cb + 8 * u + e] : 0.f; }
+        const int which = n0 >= 2 * a.d;
+        const int col = n0 - (which ? 2 * a.d : a.d);
+        const size_t kv_off = a.kv_stage ? (size_t)which * a.d + col : ((size_t)which * a.H + (col >> 6)) * kPageElems;
+        unsigned char *blk = reinterpret_cast<unsigned char *>(a.out_img) + ((size_t)blockIdx.z * (a.N >> 6) + (n0 >> 6)) * (kMaxRows * 128);
+#pragma unroll 2
+        for (int r = r4; r < rows; r += 4) {
+          const int bb = lw * 32 + r;
+          float x[8];
+          *reinterpret_cast<float4 *>(x) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32);
+          *reinterpret_cast<float4 *>(x + 4) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32 + 16);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            x[e] = fmaf(x[e], sc8[e], bi8[e]);
+            if (a.mode == EPI_GELU) x[e] = a.gelu_tanh ? gelu_tanh_f(x[e]) : gelu_erf_f(x[e]);
+          }
+          const uint4 pk = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+          if (a.mode == EPI_GELU) *reinterpret_cast<uint4 *>(blk + (size_t)bb * 128 + ((u ^ (bb & 7)) << 4)) = pk;   // the unit moves with bb % 8
+          else reinterpret_cast<uint4 *>(kv_base[bb] + kv_off)[u] = pk;
+        }
+      } else {
+        // fp32 rows: logits, q, the residual stream, or this k-range's partial sums
+        const bool add = a.mode == EPI_RESID && !partial;
+        float *dst0 = partial ? a.out_f32 + (((size_t)blockIdx.z * a.ksplit + ks) * kMaxRows + lw * 32) * a.N + n0
+                              : a.out_f32 + (size_t)(row0 + lw * 32) * a.out_stride + n0;
+        const size_t pitch = partial ? (size_t)a.N : (size_t)a.out_stride;
+        if (!add && nv == 64 && (reinterpret_cast<uintptr_t>(dst0) & 15) == 0 && (pitch & 3) == 0) {
+          // two rows per instruction, 16 bytes per lane
+          const int r2 = lane >> 4, u16 = lane & 15;
+          float sc4[4], bi4[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { sc4[e] = s_rsc[cb + 4 * u16 + e]; bi4[e] = use_bias ? s_bias[cb + 4 * u16 + e] : 0.f; }
+#pragma unroll 4
+          for (int r = r2; r < rows; r += 2) {
+            float4 x = *reinterpret_cast<const float4 *>(patch + r * 272 + u16 * 16);
+            x.x = fmaf(x.x, sc4[0], bi4[0]); x.y = fmaf(x.y, sc4[1], bi4[1]); x.z = fmaf(x.z, sc4[2], bi4[2]); x.w = fmaf(x.w, sc4[3], bi4[3]);
+            *reinterpret_cast<float4 *>(dst0 + (size_t)r * pitch + 4 * u16) = x;
+          }
+        } else {
+          // any alignment, ragged last tile, or adding into the residual stream: one row per step, two features per lane
+          float sc2[2], bi2[2];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) { sc2[e] = s_rsc[cb + lane + 32 * e]; bi2[e] = use_bias ? s_bias[cb + lane + 32 * e] : 0.f; }
+#pragma unroll 2
+          for (int r = 0; r < rows; ++r) {
+            const float *src = reinterpret_cast<const float *>(patch + r * 272);
+            float *dst = dst0 + r * pitch;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int c = lane + 32 * e;
+              if (c < nv) {
+                const float x = fmaf(src[c], sc2[e], bi2[e]);
+                dst[c] = add ? dst[c] + x : x;
+              }
+            }
+          }
+        }
+      }
+    }
+    trace_mark(a.trace, a.trace_slot, 6, 64);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  trace_mark(a.trace, a.trace_slot, 2, 64);
+  if (warp == 0) tmem_dealloc(tmem_d, kCols);
+}
+
+inline size_t gemm_tcw_smem_bytes() { return (size_t)kTwStages * kTwStageBytes + 1024 + 2304; }
+
+// k-ranges of a residual linear in the wide kernel: at least 4 k-chunks per CTA, at most what LayerNorm folds
+inline int tcw_ksplit_resid(int K) { return std::max(1, std::min(kTwMaxPartials, (K / 64) / 4)); }
+
+inline cudaError_t launch_gemm_tcw(const GemmTcArgs &a, cudaStream_t st, bool pdl) {
+  static PerDeviceOnce attr_once;
+  if (attr_once.first()) {
+    cudaFuncSetAttribute(gemm_tcw_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes());
+    cudaFuncSetAttribute(gemm_tcw_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes());
+  }
+  dim3 grid((a.N + 127) / 128, a.ksplit, (a.B + kMaxRows - 1) / kMaxRows);
+  if (a.wfmt == WF_INT4)
+    return launch_kernel(gemm_tcw_kernel<true>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(), st, pdl, a);
+  return launch_kernel(gemm_tcw_kernel<false>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(), st, pdl, a);
+}
+
 // out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)
 __global__ void fold_partials_kernel(const float *__restrict__ part, int n_part, int B, int N,
                                      const uint16_t *__restrict__ bias, float *__restrict__ out) {

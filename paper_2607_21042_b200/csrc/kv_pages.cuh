@@ -136,18 +136,22 @@ __global__ void __launch_bounds__(kMaxRows) prefill_text_kernel(const TextParams
   }
 }
 
+// A prefill pass: rows in stream-major order, given as runs of consecutive positions of one stream.
 struct PassParams {
-  int n_rows, n_out;
-  short row_stream[kMaxRows], row_pos[kMaxRows], out_rows[kMaxRows], out_slot[kMaxRows];
+  int n_rows, n_out, n_runs;
+  short run_stream[kMaxRows], run_pos0[kMaxRows], run_row0[kMaxRows + 1];   // run j covers rows run_row0[j] .. run_row0[j+1]-1
+  short out_rows[kMaxRows], out_slot[kMaxRows];
   StepIO io;
   int text_shift, text_pos0, emb_rows;   // text rows: table row = id + text_shift (clamped), position row = text_pos0 + j
 };
 
-// Row table of one prefill pass: up to 128 (stream, position) rows taken from the prefixes.
-__global__ void __launch_bounds__(kMaxRows) prefill_pass_kernel(const PassParams p, PageState ps, RowTable rt, StepIO *io, int d) {
+// Row table of one prefill pass: up to kMaxPassRows (stream, position) rows taken from the prefixes.
+__global__ void __launch_bounds__(kMaxPassRows) prefill_pass_kernel(const PassParams p, PageState ps, RowTable rt, StepIO *io, int d) {
   const int i = threadIdx.x;
   if (i < p.n_rows) {
-    const int s = p.row_stream[i], t = p.row_pos[i];
+    int j = 0;
+    while (j + 1 < p.n_runs && p.run_row0[j + 1] <= i) ++j;
+    const int s = p.run_stream[j], t = p.run_pos0[j] + (i - p.run_row0[j]);
     rt.row_stream[i] = s;
     rt.row_pos[i] = t;
     const int nc = ps.stream_ncond[s];
@@ -156,9 +160,9 @@ __global__ void __launch_bounds__(kMaxRows) prefill_pass_kernel(const PassParams
       rt.row_posidx[i] = 0;
       rt.row_emb[i] = ps.stream_emb[s] + (size_t)t * d;
     } else {          // text token j of the stream
-      const int j = t - nc;
-      rt.row_token[i] = min(max(ps.stream_text[s][j] + p.text_shift, 0), p.emb_rows - 1);
-      rt.row_posidx[i] = p.text_pos0 + j;
+      const int jt = t - nc;
+      rt.row_token[i] = min(max(ps.stream_text[s][jt] + p.text_shift, 0), p.emb_rows - 1);
+      rt.row_posidx[i] = p.text_pos0 + jt;
       rt.row_emb[i] = nullptr;
     }
   }

@@ -88,6 +88,8 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
+  int prefill_pass_rows = kMaxPassRows;   // rows per prefill pass (option "prefill_pass_rows": 128, 256, 384 or 512)
+  int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
   bool use_attn_mma = true;      // tensor-core attention in prefill passes (option "attn_mma")
   bool use_attn_prefill = true;  // shared-page attention in prefill passes (option "attn_prefill")
   bool use_attn_stream = true;   // streaming attention for large batches (option "attn_stream")
@@ -207,17 +209,17 @@ size_t carve(tts_gpt *h, void *base) {
   ps.stream_text = cv.take<const int *>(S);
   ps.stream_ncond = cv.take<int>(S);
   RowTable &rt = h->rt;
-  rt.row_stream = cv.take<int>(kMaxRows);
-  rt.row_pos = cv.take<int>(kMaxRows);
-  rt.row_token = cv.take<int>(kMaxRows);
-  rt.row_posidx = cv.take<int>(kMaxRows);
-  rt.row_emb = cv.take<const uint16_t *>(kMaxRows);
+  rt.row_stream = cv.take<int>(kMaxPassRows);
+  rt.row_pos = cv.take<int>(kMaxPassRows);
+  rt.row_token = cv.take<int>(kMaxPassRows);
+  rt.row_posidx = cv.take<int>(kMaxPassRows);
+  rt.row_emb = cv.take<const uint16_t *>(kMaxPassRows);
   rt.out_rows = cv.take<int>(kMaxRows);
   rt.out_slot = cv.take<int>(kMaxRows);
   rt.row_order = cv.take<int>(kMaxRows);
   h->io = cv.take<StepIO>(1);
-  h->x = cv.take<float>((size_t)kMaxRows * d);
-  h->q = cv.take<float>((size_t)kMaxRows * d);
+  h->x = cv.take<float>((size_t)kMaxPassRows * d);
+  h->q = cv.take<float>((size_t)kMaxPassRows * d);
   h->logits = cv.take<float>((size_t)kMaxRows * V);
   h->st_in = cv.take<int>(kMaxRows);
   h->st_tok = cv.take<int>(kMaxRows);
@@ -233,12 +235,13 @@ size_t carve(tts_gpt *h, void *base) {
   h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
   h->have_tc = true;
   if (h->have_tc) {
-    h->a_img = cv.take<char>(act_image_bytes(d));
-    h->o_img = cv.take<char>(act_image_bytes(d));
-    h->h_img = cv.take<char>(act_image_bytes(F));
+    constexpr int kTiles = kMaxPassRows / kMaxRows;   // row tiles of a prefill pass
+    h->a_img = cv.take<char>(kTiles * act_image_bytes(d));
+    h->o_img = cv.take<char>(kTiles * act_image_bytes(d));
+    h->h_img = cv.take<char>(kTiles * act_image_bytes(F));
     h->hf_img = cv.take<char>(act_image_bytes(d));
-    h->partials = cv.take<float>((size_t)kTcKSplit * kMaxRows * d);
-    h->partials_floats = (size_t)kTcKSplit * kMaxRows * d;
+    h->partials_floats = (size_t)kTiles * std::max(kTcKSplit, kTwMaxPartials) * kMaxRows * d;   // [row tile][k-range][128][d]
+    h->partials = cv.take<float>(h->partials_floats);
   }
   return cv.off;
 }
@@ -335,16 +338,28 @@ int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int
   return TTS_GPT_OK;
 }
 
+int launch_gemm(tts_gpt *h, const GemmTcArgs &a, bool wide, cudaStream_t st, bool pdl) {
+  CUDA_TRY(h, wide ? launch_gemm_tcw(a, st, pdl) : launch_gemm_tc(a, st, pdl));
+  return TTS_GPT_OK;
+}
+
+// Up to 128 rows (decode steps, small prefill passes): the kernel with chunks of 32 batch rows, O-proj and FC2
+// split over 4 k-ranges.  More rows (prefill passes of several row tiles): the wide kernel, one CTA per 128 rows
+// x 128 features; O-proj and FC2 split over up to 4 k-ranges.  Either way the next LayerNorm folds the ranges.
 int run_layers_tc(tts_gpt *h, int R, bool decode) {
   const tts_gpt_config_t &c = h->cfg;
   const int d = c.d_model;
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
+  const bool wide = R > kMaxRows;
+  const int o_ks = wide ? tcw_ksplit_resid(d) : kTcKSplit;
+  const int f2_ks = wide ? tcw_ksplit_resid(c.d_ff) : kTcKSplit;
+  const int o_parts = o_ks > 1 ? o_ks : 0, f2_parts = f2_ks > 1 ? f2_ks : 0;   // 0: the linear added into x itself
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
     // fold the previous layer's FC2 partial sums into x, then LN1 -> image
-    int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : kTcKSplit, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
+    int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : f2_parts, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
                           h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
@@ -352,7 +367,7 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
     qa.kv_stage = h->kv_stage;
     trace_attach(h, qa);
-    CUDA_TRY(h, launch_gemm_tc(qa, st, pdl));
+    if ((rc = launch_gemm(h, qa, wide, st, pdl))) return rc;
     AttnArgs aa;
     memset(&aa, 0, sizeof aa);
     aa.q = h->q; aa.kv_layer = kvl; aa.page_table = h->ps.page_table; aa.row_stream = h->rt.row_stream;
@@ -360,22 +375,23 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     aa.H = c.n_head; aa.pps = h->pps; aa.old_pages_final = decode ? 1 : 0;
     trace_attach(h, aa);
     CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
-    GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, kTcKSplit);
-    oa.out_f32 = h->partials; oa.out_stride = d;
+    GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, o_ks);
+    oa.out_f32 = o_parts ? h->partials : h->x; oa.out_stride = d;
     trace_attach(h, oa);
-    CUDA_TRY(h, launch_gemm_tc(oa, st, pdl));
-    rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, kTcKSplit, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
+    if ((rc = launch_gemm(h, oa, wide, st, pdl))) return rc;
+    rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, o_parts, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs f1 = gemm_args(h, L.fc1, h->a_img, R, EPI_GELU, 1);
     f1.out_img = h->h_img; f1.gelu_tanh = c.gelu_tanh;
     trace_attach(h, f1);
-    CUDA_TRY(h, launch_gemm_tc(f1, st, pdl));
-    GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, kTcKSplit);
-    f2.out_f32 = h->partials; f2.out_stride = d;
+    if ((rc = launch_gemm(h, f1, wide, st, pdl))) return rc;
+    GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, f2_ks);
+    f2.out_f32 = f2_parts ? h->partials : h->x; f2.out_stride = d;
     trace_attach(h, f2);
-    CUDA_TRY(h, launch_gemm_tc(f2, st, pdl));
+    if ((rc = launch_gemm(h, f2, wide, st, pdl))) return rc;
     h->launches += 5;
   }
+  h->tc_tail_parts = f2_parts;
   return TTS_GPT_OK;
 }
 
@@ -385,7 +401,7 @@ int run_head_tc(tts_gpt *h, int n_out) {
   cudaStream_t st = h->stream;
   const bool pdl = h->use_pdl;
   const bool big = n_out > 16;
-  int rc = launch_ln_tc(h, n_out, h->lnf_g, h->lnf_b, kTcKSplit, h->layers[c.n_layer - 1].fc2.bias,
+  int rc = launch_ln_tc(h, n_out, h->lnf_g, h->lnf_b, h->tc_tail_parts, h->layers[c.n_layer - 1].fc2.bias,
                         big ? h->hf_img : nullptr, big ? nullptr : h->hf, h->rt.out_rows, h->rt.out_slot, h->io, 0);
   if (rc) return rc;
   if (big) {
@@ -712,7 +728,9 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
   StepIO io;
   io.in_tokens = nullptr; io.uniforms = uniforms; io.out_tokens = out_tokens; io.out_logits = out_logits;
   io.out_hidden = (uint16_t *)out_hidden; io.top_k = top_k; io.temperature = temperature; io.n_out = 0;
-  // rows in stream-major order, 128 per pass
+  // rows in stream-major order; a pass takes up to `pass_rows` of them (several row tiles of 128 when the
+  // tensor-core path with its bf16 pages is available, else one)
+  const int pass_rows = (h->have_tc && h->use_tc && !h->kv_fp8) ? h->prefill_pass_rows : kMaxRows;
   PassParams ps;
   memset(&ps, 0, sizeof ps);
   ps.io = io;
@@ -720,7 +738,8 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
   auto flush = [&]() -> int {
     if (ps.n_rows == 0) return TTS_GPT_OK;
     ps.io.n_out = ps.n_out;
-    prefill_pass_kernel<<<1, kMaxRows, 0, h->stream>>>(ps, h->ps, h->rt, h->io, c.d_model);
+    ps.run_row0[ps.n_runs] = (short)ps.n_rows;
+    prefill_pass_kernel<<<1, kMaxPassRows, 0, h->stream>>>(ps, h->ps, h->rt, h->io, c.d_model);
     CUDA_TRY(h, cudaGetLastError());
     h->launches += 1;
     int r = run_embed(h, ps.n_rows);
@@ -728,20 +747,25 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
     r = run_layers(h, ps.n_rows, false);
     if (r) return r;
     if (ps.n_out > 0) r = run_head(h, ps.n_out, ps.n_rows);
-    ps.n_rows = 0; ps.n_out = 0;
+    ps.n_rows = 0; ps.n_out = 0; ps.n_runs = 0;
     return r;
   };
   for (int i = 0; i < n; ++i) {
-    for (int t = 0; t < plen[i]; ++t) {
-      const int r = ps.n_rows++;
-      ps.row_stream[r] = (short)pp.stream_ids[i];
-      ps.row_pos[r] = (short)t;
-      if (t == plen[i] - 1) {
-        ps.out_rows[ps.n_out] = (short)r;
+    int t = 0;
+    while (t < plen[i]) {
+      const int take = std::min(plen[i] - t, pass_rows - ps.n_rows);
+      ps.run_stream[ps.n_runs] = (short)pp.stream_ids[i];
+      ps.run_pos0[ps.n_runs] = (short)t;
+      ps.run_row0[ps.n_runs] = (short)ps.n_rows;
+      ++ps.n_runs;
+      ps.n_rows += take;
+      t += take;
+      if (t == plen[i]) {
+        ps.out_rows[ps.n_out] = (short)(ps.n_rows - 1);
         ps.out_slot[ps.n_out] = (short)i;
         ++ps.n_out;
       }
-      if (ps.n_rows == kMaxRows) { rc = flush(); if (rc) return rc; }
+      if (ps.n_rows == pass_rows) { rc = flush(); if (rc) return rc; }
     }
   }
   return flush();
@@ -987,6 +1011,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   if (k == "graph") h->use_graph = on && h->stream != nullptr && h->stream != cudaStreamLegacy;
   else if (k == "pdl") h->use_pdl = on;
   else if (k == "tc") h->use_tc = on;
+  else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be 128, 256, 384 or 512"); h->prefill_pass_rows = value; }
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;
@@ -1084,8 +1109,11 @@ int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, 
   size_t bytes;
   int rc = tts_gpt_op_linear_tc_scratch_bytes(N, K, &bytes);
   if (rc) return rc;
+  const bool wide = ksplit < 0;   // the kernel of the multi-tile prefill passes, here on one row tile
+  if (wide) ksplit = -ksplit;
   if (wfmt < 0 || wfmt > 2 || !w || !act || !out || !scratch || B < 1 || B > kMaxRows || (uintptr_t)scratch % 1024 ||
-      (ksplit != 1 && ksplit != kTcKSplit) || K / 64 < ksplit || K % 128 || (wfmt != WF_BF16 && !s) ||
+      (!wide && ksplit != 1 && ksplit != kTcKSplit) || ksplit < 1 || ksplit > kTwMaxPartials || K / 64 < ksplit || K % 128 ||
+      (wfmt != WF_BF16 && !s) ||
       (uintptr_t)w % 16 || (uintptr_t)s % 16 || (uintptr_t)act % 16 || (uintptr_t)out % 16 || (uintptr_t)bias % 16)
     return fail(nullptr, TTS_GPT_E_ARG, "op_linear_tc: bad or misaligned argument");
   cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -1107,10 +1135,10 @@ int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, 
   a.w_img = wimg; a.act_img = aimg; a.N = N; a.K = K; a.B = B; a.ksplit = ksplit; a.wfmt = wfmt; a.scales = tiled_s;
   if (ksplit == 1) {
     a.mode = EPI_F32; a.bias = (const uint16_t *)bias; a.out_f32 = out; a.out_stride = N;
-    CUDA_TRY(nullptr, launch_gemm_tc(a, st, false));
+    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, st, false) : launch_gemm_tc(a, st, false));
   } else {   // partial sums per k-range, then folded in range order (what the following LayerNorm does in the engine)
     a.mode = EPI_RESID; a.out_f32 = part; a.out_stride = N;
-    CUDA_TRY(nullptr, launch_gemm_tc(a, st, false));
+    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, st, false) : launch_gemm_tc(a, st, false));
     fold_partials_kernel<<<(unsigned)(((size_t)B * N + 255) / 256), 256, 0, st>>>(part, ksplit, B, N, (const uint16_t *)bias, out);
     CUDA_TRY(nullptr, cudaGetLastError());
   }

@@ -627,3 +627,49 @@ def test_e4m3_kv_cache_differs_from_the_bf16_cache_as_the_format_allows(tiny_mod
     ref16, _ = O.replay_full(exact, O.bf16_to_f64(prefix), toks[:-1])
     d8 = np.max(np.abs(logits - ref8)); d16 = np.max(np.abs(logits - ref16))
     assert d8 <= E4M3_MAX_ABS and d8 < d16 < 0.5
+
+
+@pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
+def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
+    """Prefill passes of up to 512 rows (four row tiles of 128) run the wide tensor-core linears: a stream
+    that spans several tiles and passes, streams that end inside a tile, a pass that is exactly full, a
+    ragged last pass; then a few decode steps over the pages those passes wrote."""
+    lens = [300, 5, 207, 128, 1, 250, 133]          # 1024 rows: two full passes of 512, tile edges inside streams
+    S = len(lens)
+    cfg = _tiny(wfmt, max_streams=S, n_pages=S * 6, max_context=384, max_pos=512)
+    w = C.make_weights(cfg, seed=5)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    prefixes = C.make_prefixes(cfg, lens, seed=13)
+    lg, tk = _run_batch(eng, prefixes, 4)
+    for s in range(S):
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk[s][:-1])
+        assert_logits_close(lg[s], ref, "multi-tile prefill, stream %d" % s)
+        check_tokens(tk[s], ref, 0, 1.0, None, "multi-tile prefill, stream %d" % s)
+    # the same prefixes in passes of 128 and of 384 rows: same results up to summation order
+    for rows in (128, 384):
+        eng.set_option("prefill_pass_rows", rows)
+        lg2, tk2 = _run_batch(eng, prefixes, 4)
+        for s in range(S):
+            assert_same_up_to_ties(tk[s], lg[s], tk2[s], lg2[s], "passes of %d rows, stream %d" % (rows, s))
+    with pytest.raises(B.TtsGptError):
+        eng.set_option("prefill_pass_rows", 200)
+    eng.destroy()
+
+
+def test_prefill_large_pass_with_ragged_tail_and_poisoned_pages():
+    """A single pass of 3 tiles + 17 rows, free pages poisoned: nothing outside the written slots is read."""
+    lens = [190, 211]
+    cfg = _tiny(C.W_BF16, max_streams=2, n_pages=10, max_context=256, max_pos=256)
+    w = C.make_weights(cfg, seed=6)
+    model = O.OracleModel(cfg, w)
+    eng = B.TtsGpt(cfg, w, DEV)
+    eng.set_option("poison_free_pages", 1)
+    prefixes = C.make_prefixes(cfg, lens, seed=14)
+    lg, tk = _run_batch(eng, prefixes, 3)
+    assert np.all(np.isfinite(lg))
+    for s in range(2):
+        ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk[s][:-1])
+        assert_logits_close(lg[s], ref, "401-row pass, stream %d" % s)
+    assert eng.check_canaries() == 0
+    eng.destroy()

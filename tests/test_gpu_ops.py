@@ -77,7 +77,10 @@ def test_linear_int8_extreme_codes_exact():
 
 @pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
 @pytest.mark.parametrize("N,K,Bn,ksplit", [(128, 256, 32, 1), (256, 256, 17, 1), (200, 1280, 128, 1),
-                                             (1280, 1280, 66, 4), (130, 5120, 100, 4), (8194, 1280, 40, 1)])
+                                             (1280, 1280, 66, 4), (130, 5120, 100, 4), (8194, 1280, 40, 1),
+                                             # the kernel of multi-tile prefill passes (128 rows x 128 features per CTA)
+                                             (3840, 1280, 128, -1), (8194, 1280, 37, -1), (5120, 1280, 97, -1), (256, 256, 128, -1),
+                                             (1280, 1280, 128, -4), (1280, 5120, 111, -4), (200, 1024, 19, -3), (130, 256, 128, -2)])
 def test_tensor_core_linear_matches_oracle(wfmt, N, K, Bn, ksplit):
     rng = np.random.default_rng(N + K + Bn + wfmt)
     wb = _rand_bf16(rng, (N, K), 0.02)
