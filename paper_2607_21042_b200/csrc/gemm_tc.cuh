@@ -206,6 +206,7 @@ struct GemmTcArgs {
   int wfmt;                 // WF_* : bf16 = no scale, int8 = per row, int4 = per row and 128-column group
   int N, K, B, mode;        // mode: EPI_* of linear.cuh
   int ksplit;               // k-ranges (gridDim.z)
+  int stages;               // wide kernel: ring depth, set by its launcher
   float *out_f32;           // EPI_F32: out[b*out_stride+n]; EPI_QKV: q; EPI_RESID: x (ksplit == 1) or partials [ksplit][128][N]
   int out_stride;
   void *out_img;            // EPI_GELU: activation image of the next linear (row length N)
@@ -476,19 +477,44 @@ __global__ void __launch_bounds__(kTcThreads) gemm_tc_kernel(const GemmTcArgs a)
 // them out with the lanes along the row.  The residual linears split K over up to 4 CTAs whose
 // partial sums the next LayerNorm folds (partials [row tile][range][128][N]); the others take all
 // of K in one CTA.
-constexpr int kTwStages = 3;
+constexpr int kTwMaxStages = 6;                 // ring depth: 6 stages with one CTA per SM, 3 when two CTAs share an SM
 constexpr uint32_t kTwStageBytes = 2 * 16384;   // activations (M operand) | weights (N operand)
 constexpr int kTwThreads = 320;                 // warp 0 producer, warp 1 MMA issuer, warps 2-9 epilogue
 constexpr int kTwMaxPartials = 4;               // k-ranges the following LayerNorm folds
 
 
+// bf16 destinations of the wide kernel's epilogue: four parked rows per instruction, lane = (row in the group
+// of four, 16-byte unit = 8 features).  KIND 0: tanh-GELU into the next linear's activation image, 1: erf-GELU
+// into it, 2: K/V rows into their page slots (or the staging rows of the 8-bit cache).
+template <int KIND>
+__device__ __forceinline__ void tw_rows_bf16(const unsigned char *patch, int rows, int r4, int u, int lw, const float (&sc8)[8],
+                                             const float (&bi8)[8], unsigned char *blk, uint16_t *const *kv_base, size_t kv_off) {
+#pragma unroll 2
+  for (int r = r4; r < rows; r += 4) {
+    const int bb = lw * 32 + r;
+    float x[8];
+    *reinterpret_cast<float4 *>(x) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32);
+    *reinterpret_cast<float4 *>(x + 4) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32 + 16);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      x[e] = fmaf(x[e], sc8[e], bi8[e]);
+      if (KIND == 0) x[e] = gelu_tanh_f(x[e]);
+      if (KIND == 1) x[e] = gelu_erf_f(x[e]);
+    }
+    const uint4 pk = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+    if (KIND == 2) reinterpret_cast<uint4 *>(kv_base[bb] + kv_off)[u] = pk;
+    else *reinterpret_cast<uint4 *>(blk + (size_t)bb * 128 + ((u ^ (bb & 7)) << 4)) = pk;   // the unit moves with bb % 8
+  }
+}
+
 template <bool GROUPED>
 __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a) {
   extern __shared__ __align__(16) unsigned char tc_smem_raw[];
   unsigned char *ring = tc_smem_raw + ((1024u - (smem_u32(tc_smem_raw) & 1023u)) & 1023u);
-  uint64_t *full = reinterpret_cast<uint64_t *>(ring + kTwStages * kTwStageBytes);
-  uint64_t *empty = full + kTwStages;
-  uint64_t *acc_done = empty + kTwStages;
+  const int n_stage = a.stages;
+  uint64_t *full = reinterpret_cast<uint64_t *>(ring + n_stage * kTwStageBytes);
+  uint64_t *empty = full + kTwMaxStages;
+  uint64_t *acc_done = empty + kTwMaxStages;
   uint64_t *grp_done = acc_done + 1;   // [2]
   uint64_t *grp_free = grp_done + 2;   // [2]
   uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(grp_free + 2);
@@ -510,7 +536,7 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   constexpr uint32_t kCols = GROUPED ? 256u : 128u;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kTwStages; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+    for (int s = 0; s < n_stage; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
     mbar_init(acc_done, 1);
     mbar_init(grp_done, 1); mbar_init(grp_done + 1, 1);
     mbar_init(grp_free, kTcEpiThreads); mbar_init(grp_free + 1, kTcEpiThreads);
@@ -548,7 +574,7 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   const unsigned char *gW = reinterpret_cast<const unsigned char *>(a.w_img) + ((size_t)nt * KC + kc0) * kTcABytes;
   const unsigned char *gX = reinterpret_cast<const unsigned char *>(a.act_img) + ((size_t)blockIdx.z * KC + kc0) * (kMaxRows * 128);
 
-  const int pre = min(n_it, kTwStages);
+  const int pre = min(n_it, n_stage);
   if (threadIdx.x == 0) {
     for (int i = 0; i < pre; ++i) {   // weights do not depend on the previous kernel
       mbar_expect_tx(full + i, kTwStageBytes);
@@ -563,8 +589,8 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
       for (int i = 0; i < pre; ++i)
         bulk_copy_g2s(ring + (size_t)i * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + i);
       for (int i = pre; i < n_it; ++i) {
-        const int s = i % kTwStages;
-        tc_wait(empty + s, ((i / kTwStages) - 1) & 1, failed, a.err);
+        const int s = i % n_stage;
+        tc_wait(empty + s, ((i / n_stage) - 1) & 1, failed, a.err);
         mbar_expect_tx(full + s, kTwStageBytes);
         bulk_copy_g2s(ring + (size_t)s * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + s);
         bulk_copy_g2s(ring + (size_t)s * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + s);
@@ -576,8 +602,8 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
     if (lane == 0) {
       const uint32_t idesc = tc_instr_desc(128, 128);
       for (int i = 0; i < n_it; ++i) {
-        const int s = i % kTwStages;
-        tc_wait(full + s, (i / kTwStages) & 1, failed, a.err);
+        const int s = i % n_stage;
+        tc_wait(full + s, (i / n_stage) & 1, failed, a.err);
         const int g = i >> 1;
         if (GROUPED && (i & 1) == 0 && g >= 2) tc_wait(grp_free + (g & 1), ((g >> 1) - 1) & 1, failed, a.err);
         tc_fence_after_sync();
@@ -689,21 +715,14 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
         const int col = n0 - (which ? 2 * a.d : a.d);
         const size_t kv_off = a.kv_stage ? (size_t)which * a.d + col : ((size_t)which * a.H + (col >> 6)) * kPageElems;
         unsigned char *blk = reinterpret_cast<unsigned char *>(a.out_img) + ((size_t)blockIdx.z * (a.N >> 6) + (n0 >> 6)) * (kMaxRows * 128);
-#pragma unroll 2
-        for (int r = r4; r < rows; r += 4) {
-          const int bb = lw * 32 + r;
-          float x[8];
-          *reinterpret_cast<float4 *>(x) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32);
-          *reinterpret_cast<float4 *>(x + 4) = *reinterpret_cast<const float4 *>(patch + r * 272 + u * 32 + 16);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            x[e] = fmaf(x[e], sc8[e], bi8[e]);
-            if (a.mode == EPI_GELU) x[e] = a.gelu_tanh ? gelu_tanh_f(x[e]) : gelu_erf_f(x[e]);
-          }
-          const uint4 pk = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
-          if (a.mode == EPI_GELU) *reinterpret_cast<uint4 *>(blk + (size_t)bb * 128 + ((u ^ (bb & 7)) << 4)) = pk;   // the unit moves with bb % 8
-          else reinterpret_cast<uint4 *>(kv_base[bb] + kv_off)[u] = pk;
-        }
+        // one loop per destination kind, so that each is straight-line code (this runs once per CTA, from a cold
+        // instruction cache: a loop that chose per element between the two GELU forms took four times as long)
+        if (a.mode == EPI_GELU && a.gelu_tanh)
+          tw_rows_bf16<0>(patch, rows, r4, u, lw, sc8, bi8, blk, kv_base, kv_off);
+        else if (a.mode == EPI_GELU)
+          tw_rows_bf16<1>(patch, rows, r4, u, lw, sc8, bi8, blk, kv_base, kv_off);
+        else
+          tw_rows_bf16<2>(patch, rows, r4, u, lw, sc8, bi8, blk, kv_base, kv_off);
       } else {
         // fp32 rows: logits, q, the residual stream, or this k-range's partial sums
         const bool add = a.mode == EPI_RESID && !partial;
@@ -751,21 +770,24 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   if (warp == 0) tmem_dealloc(tmem_d, kCols);
 }
 
-inline size_t gemm_tcw_smem_bytes() { return (size_t)kTwStages * kTwStageBytes + 1024 + 2304; }
+inline size_t gemm_tcw_smem_bytes(int stages) { return (size_t)stages * kTwStageBytes + 1024 + 2304; }
 
 // k-ranges of a residual linear in the wide kernel: at least 4 k-chunks per CTA, at most what LayerNorm folds
 inline int tcw_ksplit_resid(int K) { return std::max(1, std::min(kTwMaxPartials, (K / 64) / 4)); }
 
-inline cudaError_t launch_gemm_tcw(const GemmTcArgs &a, cudaStream_t st, bool pdl) {
+// n_sm: SMs of the device; a grid that fits at one CTA per SM gets the deep ring
+inline cudaError_t launch_gemm_tcw(const GemmTcArgs &a0, int n_sm, cudaStream_t st, bool pdl) {
   static PerDeviceOnce attr_once;
   if (attr_once.first()) {
-    cudaFuncSetAttribute(gemm_tcw_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes());
-    cudaFuncSetAttribute(gemm_tcw_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes());
+    cudaFuncSetAttribute(gemm_tcw_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes(kTwMaxStages));
+    cudaFuncSetAttribute(gemm_tcw_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemm_tcw_smem_bytes(kTwMaxStages));
   }
+  GemmTcArgs a = a0;
   dim3 grid((a.N + 127) / 128, a.ksplit, (a.B + kMaxRows - 1) / kMaxRows);
+  a.stages = (int)(grid.x * grid.y * grid.z) <= n_sm ? kTwMaxStages : 3;
   if (a.wfmt == WF_INT4)
-    return launch_kernel(gemm_tcw_kernel<true>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(), st, pdl, a);
-  return launch_kernel(gemm_tcw_kernel<false>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(), st, pdl, a);
+    return launch_kernel(gemm_tcw_kernel<true>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(a.stages), st, pdl, a);
+  return launch_kernel(gemm_tcw_kernel<false>, grid, dim3(kTwThreads), gemm_tcw_smem_bytes(a.stages), st, pdl, a);
 }
 
 // out[b,n] = bias[n] + partial[0][b,n] + partial[1][b,n] + ...  (stand-alone entry point)

@@ -339,7 +339,7 @@ int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int
 }
 
 int launch_gemm(tts_gpt *h, const GemmTcArgs &a, bool wide, cudaStream_t st, bool pdl) {
-  CUDA_TRY(h, wide ? launch_gemm_tcw(a, st, pdl) : launch_gemm_tc(a, st, pdl));
+  CUDA_TRY(h, wide ? launch_gemm_tcw(a, h->n_sm, st, pdl) : launch_gemm_tc(a, st, pdl));
   return TTS_GPT_OK;
 }
 
@@ -1135,10 +1135,10 @@ int32_t tts_gpt_op_linear_tc(int32_t wfmt, int32_t N, int32_t K, const void *w, 
   a.w_img = wimg; a.act_img = aimg; a.N = N; a.K = K; a.B = B; a.ksplit = ksplit; a.wfmt = wfmt; a.scales = tiled_s;
   if (ksplit == 1) {
     a.mode = EPI_F32; a.bias = (const uint16_t *)bias; a.out_f32 = out; a.out_stride = N;
-    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, st, false) : launch_gemm_tc(a, st, false));
+    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, 148, st, false) : launch_gemm_tc(a, st, false));
   } else {   // partial sums per k-range, then folded in range order (what the following LayerNorm does in the engine)
     a.mode = EPI_RESID; a.out_f32 = part; a.out_stride = N;
-    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, st, false) : launch_gemm_tc(a, st, false));
+    CUDA_TRY(nullptr, wide ? launch_gemm_tcw(a, 148, st, false) : launch_gemm_tc(a, st, false));
     fold_partials_kernel<<<(unsigned)(((size_t)B * N + 255) / 256), 256, 0, st>>>(part, ksplit, B, N, (const uint16_t *)bias, out);
     CUDA_TRY(nullptr, cudaGetLastError());
   }
