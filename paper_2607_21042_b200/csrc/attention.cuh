@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_kernel(const AttnAr
   // plain row-major bf16, or the image layout of the tensor-core linear that consumes it
   uint16_t *out = nullptr;
   if (e < kHeadDim)
-    out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
+    out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, h * kHeadDim + e, a.H * kHeadDim))
                       : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
   if (!CLUSTER) {
     float M, L, O;
@@ -523,7 +523,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32, 3) attention_stream_kernel(co
   float M, L, O;
   cta_merge(m, l, o, warp, tg, sub, sm_m, sm_l, sm_o, M, L, O);
   if (e < kHeadDim) {
-    uint16_t *out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
+    uint16_t *out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, h * kHeadDim + e, a.H * kHeadDim))
                                 : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
     *out = float_to_bf16_bits(O / L);
   }

@@ -199,7 +199,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_fp8_kernel(const Fp
   }
   uint16_t *out = nullptr;
   if (e < kHeadDim)
-    out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset(r, h * kHeadDim + e))
+    out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, h * kHeadDim + e, a.H * kHeadDim))
                       : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
   if (n_chunks == 1) {
     if (e < kHeadDim) *out = float_to_bf16_bits(O / L);

@@ -230,9 +230,10 @@ size_t carve(tts_gpt *h, void *base) {
   h->o = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->hbuf = cv.take<uint16_t>((size_t)kMaxRows * F);
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
-  h->kv_stage = h->kv_fp8 ? cv.take<uint16_t>((size_t)kMaxRows * 2 * d) : nullptr;
-  h->attn_partials = cv.take<float>((size_t)kMaxRows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
-  h->attn_tickets = cv.take<unsigned int>((size_t)kMaxRows * c.n_head);
+  h->kv_stage = h->kv_fp8 ? cv.take<uint16_t>((size_t)kMaxPassRows * 2 * d) : nullptr;
+  const size_t attn_rows = h->kv_fp8 ? kMaxPassRows : kMaxRows;   // the 8-bit cache's attention kernel also serves prefill passes
+  h->attn_partials = cv.take<float>(attn_rows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
+  h->attn_tickets = cv.take<unsigned int>(attn_rows * c.n_head);
   h->have_tc = true;
   if (h->have_tc) {
     constexpr int kTiles = kMaxPassRows / kMaxRows;   // row tiles of a prefill pass
@@ -629,7 +630,7 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
 #undef TRY_
   const int init_n = std::max(std::max(c.n_pages, c.max_streams * h->pps), c.max_streams);
   init_pages_kernel<<<(init_n + 255) / 256, 256, 0, h->stream>>>(h->ps);
-  cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)kMaxRows * c.n_head * sizeof(unsigned int), h->stream);
+  cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)(h->kv_fp8 ? kMaxPassRows : kMaxRows) * c.n_head * sizeof(unsigned int), h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_lo, kCanaryByte, kCanaryBytes, h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_hi, kCanaryByte, kCanaryBytes, h->stream);
   if (e == cudaSuccess) {
@@ -729,8 +730,8 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
   io.in_tokens = nullptr; io.uniforms = uniforms; io.out_tokens = out_tokens; io.out_logits = out_logits;
   io.out_hidden = (uint16_t *)out_hidden; io.top_k = top_k; io.temperature = temperature; io.n_out = 0;
   // rows in stream-major order; a pass takes up to `pass_rows` of them (several row tiles of 128 when the
-  // tensor-core path with its bf16 pages is available, else one)
-  const int pass_rows = (h->have_tc && h->use_tc && !h->kv_fp8) ? h->prefill_pass_rows : kMaxRows;
+  // tensor-core path is available, else one)
+  const int pass_rows = (h->have_tc && h->use_tc) ? h->prefill_pass_rows : kMaxRows;
   PassParams ps;
   memset(&ps, 0, sizeof ps);
   ps.io = io;
