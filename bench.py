@@ -229,8 +229,12 @@ def run_workload(key, args, wcache, device, local, world, peaks):
         tot_ms = 0.0
         tot_tokens = tot_bytes = tot_steps = reps = 0
         while True:
+            if args.profiler_range == "all":
+                torch.cuda.profiler.start()     # the prefill call that opens the streams, then the decode steps
             ids = open_all()
             eng.sync()
+            if args.profiler_range == "decode":
+                torch.cuda.profiler.start()     # the decode steps only
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             with torch.cuda.stream(eng.stream):
                 e0.record()
@@ -238,6 +242,8 @@ def run_workload(key, args, wcache, device, local, world, peaks):
             with torch.cuda.stream(eng.stream):
                 e1.record()
             eng.sync()
+            if args.profiler_range:
+                torch.cuda.profiler.stop()
             tot_ms += e0.elapsed_time(e1)
             tot_tokens += tokens; tot_bytes += nbytes; tot_steps += steps
             reps += 1
@@ -270,11 +276,7 @@ def run_workload(key, args, wcache, device, local, world, peaks):
     l0 = eng.kernel_launches()
     barrier()
     sampler.start()
-    if args.profiler_range:
-        torch.cuda.profiler.start()
     ms, tokens, nbytes, steps_done, reps = timed(K, args.min_seconds, args.max_reps)
-    if args.profiler_range:
-        torch.cuda.profiler.stop()
     barrier()
     launches = eng.kernel_launches() - l0
     total_tokens = R.sum_over_ranks(tokens, device)     # replicas: every rank decodes its own copy of the workload
@@ -580,8 +582,9 @@ def main():
     ap.add_argument("--max-reps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dry-run", action="store_true", help="launcher and reduction check without a GPU (gloo)")
-    ap.add_argument("--profiler-range", action="store_true",
-                    help="bracket the timed region with cudaProfilerStart/Stop (for ncu --profile-from-start off)")
+    ap.add_argument("--profiler-range", nargs="?", const="decode", default=None, choices=["decode", "all"],
+                    help="bracket the timed decode steps (or, with 'all', also the prefill call in front of them) with "
+                         "cudaProfilerStart/Stop, for ncu --profile-from-start off")
     args = ap.parse_args()
     if args.workload is not None:
         args.workloads = str(args.workload)
