@@ -227,7 +227,7 @@ def run_workload(key, args, wcache, device, local, world, peaks):
         """Repeats `n_steps` steps from freshly opened streams until the summed device time reaches
         min_seconds.  Device time = CUDA events on the engine's stream around the queued steps."""
         tot_ms = 0.0
-        tot_tokens = tot_bytes = tot_steps = reps = 0
+        tot_tokens = tot_bytes = tot_steps = reps = tot_launches = 0
         while True:
             if args.profiler_range == "all":
                 torch.cuda.profiler.start()     # the prefill call that opens the streams, then the decode steps
@@ -238,7 +238,9 @@ def run_workload(key, args, wcache, device, local, world, peaks):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             with torch.cuda.stream(eng.stream):
                 e0.record()
+            l_before = eng.kernel_launches()
             tokens, nbytes, steps = decode_run(ids, n_steps)
+            tot_launches += eng.kernel_launches() - l_before     # kernels of the timed steps only
             with torch.cuda.stream(eng.stream):
                 e1.record()
             eng.sync()
@@ -250,7 +252,7 @@ def run_workload(key, args, wcache, device, local, world, peaks):
             # every rank takes the same number of repetitions: the decision is the slowest rank's
             if R.max_over_ranks(tot_ms, device) >= min_seconds * 1e3 or reps >= max_reps:
                 break
-        return tot_ms, tot_tokens, tot_bytes, tot_steps, reps
+        return tot_ms, tot_tokens, tot_bytes, tot_steps, reps, tot_launches
 
     # warm-up: open, W steps (captures the step graph of this batch size), close
     ids = open_all()
@@ -273,12 +275,10 @@ def run_workload(key, args, wcache, device, local, world, peaks):
 
     # ---- timed region: K steps x repetitions, device-resident inputs ----
     sampler = ClockSampler(local)
-    l0 = eng.kernel_launches()
     barrier()
     sampler.start()
-    ms, tokens, nbytes, steps_done, reps = timed(K, args.min_seconds, args.max_reps)
+    ms, tokens, nbytes, steps_done, reps, launches = timed(K, args.min_seconds, args.max_reps)
     barrier()
-    launches = eng.kernel_launches() - l0
     total_tokens = R.sum_over_ranks(tokens, device)     # replicas: every rank decodes its own copy of the workload
     ms = R.max_over_ranks(ms, device)
     value = total_tokens / (ms * 1e-3)
@@ -289,6 +289,14 @@ def run_workload(key, args, wcache, device, local, world, peaks):
                 "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS, "traffic": None, "peak_source": peak_kind,
                 "kernel": "whole decode step (%d kernel launches per step)" % round(launches / max(steps_done, 1)),
                 "algorithmic_bytes_per_step": nbytes / max(steps_done, 1)}
+    cap = captured_traffic(wl.name)
+    if cap is not None:
+        # DRAM bytes of one step from the committed ncu launch list of this workload (not measured in this run:
+        # a number taken under a profiler is not a bench value, so the capture is a separate, recorded run)
+        roofline["traffic"] = cap["dram_bytes_per_step"]
+        roofline["traffic_source"] = ("ncu dram__bytes_read.sum + dram__bytes_write.sum over the launches of one step, "
+                                      "profiles/decode_step_dram_traffic.json; algorithmic bytes of the captured steps: %d"
+                                      % cap["algorithmic_bytes_per_step"])
     if S <= 16:
         roofline["target_frac"] = TARGET_FRAC
         roofline["target_met"] = bool(gbs / hbm_peak >= TARGET_FRAC)
@@ -309,7 +317,7 @@ def run_workload(key, args, wcache, device, local, world, peaks):
     # ---- batch 128: the window in which every stream is still active, and the tensor-pipe fraction ----
     if S > 16:
         win = min(64, min(wl.decode_lens))
-        wms, wtok, wbytes, wsteps, wreps = timed(win, args.min_seconds / 2, args.max_reps)
+        wms, wtok, wbytes, wsteps, wreps, _ = timed(win, args.min_seconds / 2, args.max_reps)
         wms = R.max_over_ranks(wms, device)
         wg = wbytes / (wms * 1e-3) / 1e9
         entry["full_batch_window"] = {
@@ -373,6 +381,16 @@ def run_workload(key, args, wcache, device, local, world, peaks):
     del eng, prefixes
     torch.cuda.empty_cache()
     return entry, wl
+
+
+def captured_traffic(workload_name):
+    """The recorded ncu DRAM traffic of one decode step of this workload, if profiles/ holds one."""
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "profiles", "decode_step_dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(workload_name)
+    except (OSError, ValueError):
+        return None
 
 
 def tensor_roofline(eng, wl, open_all, toks, S, tc_peak, peak_kind, device):
