@@ -68,6 +68,8 @@ struct Fp8AttnArgs {
   float *partials;                // [R][H][kAttnMaxChunks][66]
   unsigned int *tickets;          // [R][H], zero between launches
   int H, pps, out_image;
+  const int *row_order;           // streaming variant: rows by descending context length, or null
+  int *err;                       // streaming variant: set when a bounded wait ran out
   unsigned long long *trace;
   int trace_slot;
 };
@@ -232,6 +234,152 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_fp8_kernel(const Fp
   }
   if (threadIdx.x == 0) a.tickets[(size_t)r * a.H + h] = 0u;  // ready for the next launch
   trace_mark(a.trace, a.trace_slot, 2);
+}
+
+// ------------------------------------------------------------------------------------------
+// Streaming variant for decode steps with enough (row, head) pairs to cover the GPU several times
+// (the same switch as the bf16 cache's streaming kernel): one CTA per pair, rows longest first,
+// warp w owns pages w, w+4, ...  A page's K and V blocks (4352 bytes each: codes, then scales) come
+// in by two bulk asynchronous copies into one of the warp's two stages; while the warp folds one
+// stage, the copy of its page after next runs into the other, so every resident warp keeps 8.7 KB
+// in flight without holding registers for outstanding loads.  The pages of a decode step are final
+// before the step starts, except the slot of the new token in the row's last page, which the
+// encoding kernel in front writes: every page but the last is requested ahead of the dependency
+// wait.
+constexpr uint32_t kFp8StageBytes = 2 * kFp8BlockBytes;   // K block | V block
+constexpr int kFp8Stages = 2;
+
+__device__ __forceinline__ void fp8_stream_issue(const Fp8AttnArgs &a, const int *pt, int h, int page, unsigned char *stage, uint64_t *bar) {
+  const int phys = pt[page];
+  const unsigned char *K = a.kv_layer + (((size_t)phys * 2 + 0) * a.H + h) * kFp8BlockBytes;
+  mbar_expect_tx(bar, kFp8StageBytes);
+  bulk_copy_g2s(stage, K, kFp8BlockBytes, bar);
+  bulk_copy_g2s(stage + kFp8BlockBytes, K + (size_t)a.H * kFp8BlockBytes, kFp8BlockBytes, bar);   // the V block of the same page and head
+}
+
+__global__ void __launch_bounds__(kAttnWarps * 32, 3) attention_fp8_stream_kernel(const Fp8AttnArgs a) {
+  extern __shared__ __align__(128) unsigned char fp8_stages[];   // [warp][stage][K block | V block]
+  __shared__ __align__(8) uint64_t bars[kAttnWarps][kFp8Stages];
+  __shared__ float sm_m[kAttnWarps], sm_l[kAttnWarps], sm_o[kAttnWarps][kHeadDim];
+  const int h = blockIdx.y, r = a.row_order ? a.row_order[blockIdx.z] : blockIdx.z;
+  trace_mark(a.trace, a.trace_slot, 0);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tg = lane >> 2, sub = lane & 3;
+  const int n_tok = min(a.row_pos[r] + 1, a.pps * kPageTokens);   // row and page tables are final before the step's first kernel starts
+  const int n_pages = (n_tok + kPageTokens - 1) / kPageTokens;
+  const int *pt = a.page_table + (size_t)a.row_stream[r] * a.pps;
+  unsigned char *stages = fp8_stages + (size_t)warp * (kFp8Stages * kFp8StageBytes);
+  // pages of this warp: warp, warp + 4, ...; iteration it uses stage it % 2
+  bool issued[kFp8Stages] = {false, false};
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kFp8Stages; ++s) mbar_init(&bars[warp][s], 1);
+#pragma unroll
+    for (int s = 0; s < kFp8Stages; ++s) {
+      const int page = warp + kAttnWarps * s;
+      if (page < n_pages - 1) { fp8_stream_issue(a, pt, h, page, stages + s * kFp8StageBytes, &bars[warp][s]); issued[s] = true; }
+    }
+  }
+  __syncwarp();
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kFp8Stages; ++s) {
+      const int page = warp + kAttnWarps * s;
+      if (!issued[s] && page < n_pages) fp8_stream_issue(a, pt, h, page, stages + s * kFp8StageBytes, &bars[warp][s]);
+    }
+  }
+  float qv[16];
+  {
+    const float qs = 0.125f * 1.4426950408889634f;   // scores in log2 units
+    const float *qp = a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim + 16 * sub;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float4 t = *reinterpret_cast<const float4 *>(qp + 4 * e);
+      qv[4 * e] = t.x * qs; qv[4 * e + 1] = t.y * qs; qv[4 * e + 2] = t.z * qs; qv[4 * e + 3] = t.w * qs;
+    }
+  }
+  float m = -INFINITY, l = 0.f, o[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) o[e] = 0.f;
+  int it = 0;
+  for (int page = warp; page < n_pages; page += kAttnWarps, ++it) {
+    const int s = it & 1;
+    uint64_t *bar = &bars[warp][s];
+    if (!mbar_wait_bounded(bar, (uint32_t)(it >> 1) & 1u, kAttnWaitNs)) {
+      if (a.err) atomicExch(a.err, 1);
+      mbar_wait_bounded(bar, (uint32_t)(it >> 1) & 1u, kAttnWaitNs);   // a last chance for the copy in flight towards this CTA
+      break;
+    }
+    const unsigned char *K = stages + s * kFp8StageBytes, *V = K + kFp8BlockBytes;
+    const int n_here = min(kPageTokens, n_tok - page * kPageTokens);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      if (32 * half >= n_here) break;                  // warp-uniform
+      uint4 kk[4], vv[4];
+      float ks[4], vs[4];
+      uint32_t vmask = 0u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = 32 * half + 8 * i + tg;
+        kk[i] = *reinterpret_cast<const uint4 *>(K + (size_t)t * kHeadDim + 16 * sub);
+        vv[i] = *reinterpret_cast<const uint4 *>(V + (size_t)t * kHeadDim + 16 * sub);
+        ks[i] = *reinterpret_cast<const float *>(K + kPageTokens * kHeadDim + 4 * t);
+        vs[i] = *reinterpret_cast<const float *>(V + kPageTokens * kHeadDim + 4 * t);
+        if (t < n_here) vmask |= 1u << i;
+      }
+      fp8_fold4(kk, vv, ks, vs, vmask, qv, m, l, o);
+    }
+    // The stage may be refilled only after every lane's reads of it have returned: the ballot needs a value
+    // that every lane computed from what it read, and the fence takes the ballot as an operand.
+    const unsigned int done = __ballot_sync(0xFFFFFFFFu, o[0] == o[0] || l >= 0.f);
+    if (page + kFp8Stages * kAttnWarps < n_pages && lane == 0) {
+      asm volatile("fence.proxy.async.shared::cta; // after %0" ::"r"(done) : "memory");
+      fp8_stream_issue(a, pt, h, page + kFp8Stages * kAttnWarps, stages + s * kFp8StageBytes, bar);
+    }
+  }
+  trace_mark(a.trace, a.trace_slot, 3);
+  // warp result: sum over the 8 token groups
+  l += __shfl_xor_sync(0xFFFFFFFFu, l, 4);
+  l += __shfl_xor_sync(0xFFFFFFFFu, l, 8);
+  l += __shfl_xor_sync(0xFFFFFFFFu, l, 16);
+#pragma unroll
+  for (int e = 0; e < 16; ++e) {
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 4);
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 8);
+    o[e] += __shfl_xor_sync(0xFFFFFFFFu, o[e], 16);
+  }
+  if (tg == 0) {
+    if (sub == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) sm_o[warp][16 * sub + e] = o[e];
+  }
+  __syncthreads();
+  const int e = threadIdx.x;
+  if (e < kHeadDim) {
+    float M = -INFINITY, L = 0.f, O = 0.f;
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) M = fmaxf(M, sm_m[w]);
+#pragma unroll
+    for (int w = 0; w < kAttnWarps; ++w) {
+      const float f = (sm_m[w] == -INFINITY) ? 0.f : exp2f(sm_m[w] - M);   // a warp without pages contributes nothing
+      L = fmaf(sm_l[w], f, L);
+      O = fmaf(sm_o[w][e], f, O);
+    }
+    uint16_t *out = a.out_image ? reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, h * kHeadDim + e, a.H * kHeadDim))
+                                : a.out + (size_t)r * a.H * kHeadDim + h * kHeadDim + e;
+    *out = float_to_bf16_bits(O / L);
+  }
+  trace_mark(a.trace, a.trace_slot, 2);
+}
+
+inline cudaError_t launch_attention_fp8_stream(const Fp8AttnArgs &a, int R, cudaStream_t st, bool pdl) {
+  static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
+  const size_t smem = (size_t)kAttnWarps * kFp8Stages * kFp8StageBytes;
+  if (attr_once.first()) cudaFuncSetAttribute(attention_fp8_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  return launch_kernel(attention_fp8_stream_kernel, dim3(1, a.H, R), dim3(kAttnWarps * 32), smem, st, pdl, a);
 }
 
 // Splits per (row, head): enough CTAs of 4 warps to cover the GPU about four times, at most kAttnMaxChunks.

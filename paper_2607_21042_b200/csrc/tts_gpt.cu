@@ -298,6 +298,12 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
     fa.q = aa.q; fa.kv_layer = kvl; fa.page_table = aa.page_table; fa.row_stream = aa.row_stream; fa.row_pos = aa.row_pos;
     fa.out = aa.out; fa.partials = h->attn_partials; fa.tickets = h->attn_tickets; fa.H = aa.H; fa.pps = aa.pps;
     fa.out_image = aa.out_image; fa.trace = aa.trace; fa.trace_slot = aa.trace_slot;
+    fa.err = h->dev_err;
+    const bool many = h->attn_stream_min_pairs > 0 ? R * aa.H >= h->attn_stream_min_pairs : attention_use_stream(R, aa.H, h->n_sm);
+    if (aa.old_pages_final && h->use_attn_stream && many) {   // decode steps with enough (row, head) pairs
+      fa.row_order = h->rt.row_order;
+      return launch_attention_fp8_stream(fa, R, st, pdl);
+    }
     return launch_attention_fp8(fa, R, attention_fp8_splits(R, aa.H, h->n_sm), st, pdl);
   }
   aa.err = h->dev_err;

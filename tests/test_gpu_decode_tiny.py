@@ -560,9 +560,11 @@ def test_poisoned_free_pages_and_canaries(tiny_models):
     eng.destroy()
 
 
-def _e4m3_run(cfg, w, model, lens, n, seed):
+def _e4m3_run(cfg, w, model, lens, n, seed, options=()):
     """Prefill the streams together, n batched greedy steps, every stream replayed by the oracle."""
     eng = B.TtsGpt(cfg, w, DEV)
+    for name, value in options:
+        eng.set_option(name, value)
     prefixes = C.make_prefixes(cfg, lens, seed=seed)
     S, V = len(lens), cfg.vocab
     t0 = torch.zeros(S, dtype=torch.int32, device=DEV)
@@ -612,6 +614,19 @@ def test_e4m3_kv_cache_matches_oracle_on_the_tensor_core_path():
     w = C.make_weights(cfg, seed=0)
     model = O.OracleModel(cfg, w)
     _e4m3_run(cfg, w, model, [20 + 9 * i for i in range(20)], 6, 33)
+
+
+@pytest.mark.parametrize("n_streams", [1, 3, 20])
+def test_e4m3_kv_cache_streaming_attention(n_streams):
+    """The bulk-copy streaming attention of the 8-bit cache (the engine takes it from about 30 streams of 20
+    heads; forced here): contexts below one page, on a page edge, of several pages per warp (two stages in
+    turn), rows in longest-first order."""
+    cfg = C.tiny_config(wfmt=C.W_BF16, kv_fmt=C.KV_FP8_E4M3, max_streams=n_streams, n_pages=n_streams * 12,
+                        max_context=768, max_pos=768)
+    w = C.make_weights(cfg, seed=0)
+    model = O.OracleModel(cfg, w)
+    lens = [[700], [63, 1, 520], [5 + 37 * i for i in range(20)]][[1, 3, 20].index(n_streams)]
+    _e4m3_run(cfg, w, model, lens, 5, 35, options=[("attn_stream_min_pairs", 1)])
 
 
 def test_e4m3_kv_cache_differs_from_the_bf16_cache_as_the_format_allows(tiny_models):
