@@ -313,6 +313,11 @@ def run_workload(key, args, wcache, device, local, world, peaks):
                     "rows_per_s": world * prefill_rows / (prefill_ms * 1e-3),
                     "note": "one prefill call over all prefixes (device resident), first token sampled; outside the timed region"},
     }
+    # the block linears' flops over the whole call (attention, LayerNorm and the heads are inside the time, not the flops)
+    pf_tf = 2.0 * linear_weight_count(cfg) * cfg.n_layer * prefill_rows / (prefill_ms * 1e-3) / 1e12
+    entry["prefill"]["roofline_tensor"] = {"bound": "tensor", "achieved": pf_tf, "peak": tc_peak, "unit": "TFLOP/s",
+                                           "frac": pf_tf / tc_peak, "peak_source": peak_kind + " (sustained bf16)",
+                                           "kernel": "whole prefill call: flops of the four block linears / time of the call"}
 
     # ---- batch 128: the window in which every stream is still active, and the tensor-pipe fraction ----
     if S > 16:

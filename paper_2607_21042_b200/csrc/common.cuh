@@ -12,7 +12,7 @@ constexpr int kHeadDim = 64;
 constexpr int kPageTokens = 64;
 constexpr int kPageElems = kPageTokens * kHeadDim;  // one (page, head, K|V) block: 4096 bf16 = 8 KB
 constexpr int kMaxRows = 128;                       // rows per decode step, and rows of one row tile of a prefill pass
-constexpr int kMaxPassRows = 512;                   // rows (streams x positions) of a prefill pass: up to 4 row tiles
+constexpr int kMaxPassRows = 1024;                  // rows (streams x positions) of a prefill pass: up to 4 row tiles
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 

@@ -88,7 +88,8 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
-  int prefill_pass_rows = kMaxPassRows;   // rows per prefill pass (option "prefill_pass_rows": 128, 256, 384 or 512)
+  int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); 768 measured best:
+                                 // FC1 then has 240 CTAs, one wave at two CTAs per SM, where 1024 rows need 320
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
   bool use_attn_mma = true;      // tensor-core attention in prefill passes (option "attn_mma")
   bool use_attn_prefill = true;  // shared-page attention in prefill passes (option "attn_prefill")
@@ -1018,7 +1019,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   if (k == "graph") h->use_graph = on && h->stream != nullptr && h->stream != cudaStreamLegacy;
   else if (k == "pdl") h->use_pdl = on;
   else if (k == "tc") h->use_tc = on;
-  else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be 128, 256, 384 or 512"); h->prefill_pass_rows = value; }
+  else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be a multiple of 128 from 128 to 1024"); h->prefill_pass_rows = value; }
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;

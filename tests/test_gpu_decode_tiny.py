@@ -646,10 +646,10 @@ def test_e4m3_kv_cache_differs_from_the_bf16_cache_as_the_format_allows(tiny_mod
 
 @pytest.mark.parametrize("wfmt", [C.W_BF16, C.W_INT8_PC, C.W_INT4_G128])
 def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
-    """Prefill passes of up to 512 rows (four row tiles of 128) run the wide tensor-core linears: a stream
-    that spans several tiles and passes, streams that end inside a tile, a pass that is exactly full, a
-    ragged last pass; then a few decode steps over the pages those passes wrote."""
-    lens = [300, 5, 207, 128, 1, 250, 133]          # 1024 rows: two full passes of 512, tile edges inside streams
+    """Prefill passes of several row tiles of 128 (768 rows by default, up to 1024) run the wide tensor-core
+    linears: a stream that spans several tiles and passes, streams that end inside a tile, passes that are
+    exactly full, a ragged last pass; then a few decode steps over the pages those passes wrote."""
+    lens = [300, 5, 207, 128, 1, 250, 133]          # 1024 rows, tile edges inside streams
     S = len(lens)
     cfg = _tiny(wfmt, max_streams=S, n_pages=S * 6, max_context=384, max_pos=512)
     w = C.make_weights(cfg, seed=5)
@@ -661,8 +661,8 @@ def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
         ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk[s][:-1])
         assert_logits_close(lg[s], ref, "multi-tile prefill, stream %d" % s)
         check_tokens(tk[s], ref, 0, 1.0, None, "multi-tile prefill, stream %d" % s)
-    # the same prefixes in passes of 128 and of 384 rows: same results up to summation order
-    for rows in (128, 384):
+    # the same prefixes in passes of 128, 512 and 1024 rows: same results up to summation order
+    for rows in (128, 512, 1024):
         eng.set_option("prefill_pass_rows", rows)
         lg2, tk2 = _run_batch(eng, prefixes, 4)
         for s in range(S):
