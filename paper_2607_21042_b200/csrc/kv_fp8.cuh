@@ -237,6 +237,44 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attention_fp8_kernel(const Fp
 }
 
 // ------------------------------------------------------------------------------------------
+// Prefill passes over the 8-bit cache.  The tensor-core prefill attention reads bf16 pages, and the rows
+// of a pass share the pages of a few streams, so those pages (a few dozen per pass) are decoded once per
+// layer into a scratch pool of bf16 pages with a page table of its own, and the bf16 kernel runs on that.
+// A decoded value is code x scale rounded to bf16: the rounding the bf16 cache applies to every value.
+// scratch page i = page `scratch_src[i]` of the pool, of which the first scratch_ntok[i] tokens exist (the
+// rest is written as zero: a stale slot may decode to NaN).  grid (scratch pages, 2 * H), 128 threads:
+// thread = (token, half of its 64 codes).
+__global__ void __launch_bounds__(128) kv_dequant_pages_kernel(const unsigned char *__restrict__ kv_layer, uint16_t *__restrict__ scratch,
+                                                               const int *__restrict__ scratch_src, const int *__restrict__ scratch_ntok, int H) {
+  pdl_launch_dependents();
+  pdl_wait();   // the pass's own rows were encoded by the kernel in front
+  const int i = blockIdx.x, which = blockIdx.y / H, head = blockIdx.y % H;
+  const int t = threadIdx.x >> 1, half = threadIdx.x & 1;
+  const unsigned char *blk = kv_layer + (((size_t)scratch_src[i] * 2 + which) * H + head) * kFp8BlockBytes;
+  uint16_t *dst = scratch + (((size_t)i * 2 + which) * H + head) * kPageElems + (size_t)t * kHeadDim + 32 * half;
+  uint4 out[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+  if (t < scratch_ntok[i]) {
+    const float sc = *reinterpret_cast<const float *>(blk + kPageTokens * kHeadDim + 4 * t);
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      float f[16];
+      e4m3x16_to_float(*reinterpret_cast<const uint4 *>(blk + (size_t)t * kHeadDim + 32 * half + 16 * q), f);
+      out[2 * q] = make_uint4(pack_bf16x2(f[0] * sc, f[1] * sc), pack_bf16x2(f[2] * sc, f[3] * sc),
+                              pack_bf16x2(f[4] * sc, f[5] * sc), pack_bf16x2(f[6] * sc, f[7] * sc));
+      out[2 * q + 1] = make_uint4(pack_bf16x2(f[8] * sc, f[9] * sc), pack_bf16x2(f[10] * sc, f[11] * sc),
+                                  pack_bf16x2(f[12] * sc, f[13] * sc), pack_bf16x2(f[14] * sc, f[15] * sc));
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) reinterpret_cast<uint4 *>(dst)[q] = out[q];
+}
+
+inline cudaError_t launch_kv_dequant_pages(const unsigned char *kv_layer, uint16_t *scratch, const int *src, const int *ntok,
+                                           int n_scratch, int H, cudaStream_t st, bool pdl) {
+  return launch_kernel(kv_dequant_pages_kernel, dim3(n_scratch, 2 * H), dim3(128), 0, st, pdl, kv_layer, scratch, src, ntok, H);
+}
+
+// ------------------------------------------------------------------------------------------
 // Streaming variant for decode steps with enough (row, head) pairs to cover the GPU several times
 // (the same switch as the bf16 cache's streaming kernel): one CTA per pair, rows longest first,
 // warp w owns pages w, w+4, ...  A page's K and V blocks (4352 bytes each: codes, then scales) come

@@ -143,6 +143,11 @@ struct PassParams {
   short out_rows[kMaxRows], out_slot[kMaxRows];
   StepIO io;
   int text_shift, text_pos0, emb_rows;   // text rows: table row = id + text_shift (clamped), position row = text_pos0 + j
+  // 8-bit cache: the pages the pass's rows attend over, decoded into scratch pages; run j owns the scratch pages
+  // run_scratch0[j] .. run_scratch0[j+1]-1 = pages 0.. of its stream (n_scratch = 0: not used)
+  int n_scratch;
+  short run_scratch0[kMaxRows + 1];
+  int *scratch_table, *scratch_src, *scratch_ntok;   // [max_streams][pps], [n_scratch], [n_scratch]
 };
 
 // Row table of one prefill pass: up to kMaxPassRows (stream, position) rows taken from the prefixes.
@@ -168,6 +173,15 @@ __global__ void __launch_bounds__(kMaxPassRows) prefill_pass_kernel(const PassPa
   }
   if (i < p.n_out) { rt.out_rows[i] = p.out_rows[i]; rt.out_slot[i] = p.out_slot[i]; }
   if (i == 0) *io = p.io;
+  if (i < p.n_scratch) {
+    int j = 0;
+    while (j + 1 < p.n_runs && p.run_scratch0[j + 1] <= i) ++j;
+    const int s = p.run_stream[j], pg = i - p.run_scratch0[j];
+    const int last_pos = p.run_pos0[j] + (p.run_row0[j + 1] - p.run_row0[j]) - 1;   // last position the run's rows reach
+    p.scratch_table[(size_t)s * ps.pps + pg] = i;
+    p.scratch_src[i] = ps.page_table[(size_t)s * ps.pps + pg];
+    p.scratch_ntok[i] = min(kPageTokens, last_pos + 1 - pg * kPageTokens);
+  }
 }
 
 // Debug aid: fills the K and V blocks of the given pages, in every layer, with bf16 NaN.  A kernel that reads

@@ -57,6 +57,9 @@ struct tts_gpt {
   size_t kv_layer_elems;      // 16-bit units of one layer's slice of the pool
   size_t kv_page_elems;       // ... of one page in one layer
   bool kv_fp8 = false;        // e4m3 pages with a scale per cached row and head
+  uint16_t *kv_scratch = nullptr;   // 8-bit cache: bf16 pages decoded for the tensor-core prefill attention [kScratchPages][2][H][64*64]
+  int *scratch_table = nullptr, *scratch_src = nullptr, *scratch_ntok = nullptr;
+  int pass_scratch = 0;             // scratch pages of the prefill pass in flight (0: the pass attends over the codes)
   uint16_t *kv_stage = nullptr;   // 8-bit cache: the pass's new K/V rows as bf16 [kMaxRows][2][d], encoded by kv_quantize_kernel
   // state
   PageState ps;
@@ -147,6 +150,7 @@ int check_config(const tts_gpt_config_t *c) {
 // rows of the embedding table: the semantic codes and specials the head predicts, then the text region if any
 inline int emb_rows_of(const tts_gpt_config_t &c) { return c.emb_rows > 0 ? c.emb_rows : c.vocab; }
 
+constexpr int kScratchPages = 256;          // decoded pages a prefill pass over the 8-bit cache may need
 constexpr size_t kCanaryBytes = 4096;      // guard region in front of and behind the KV pool
 constexpr unsigned char kCanaryByte = 0xA5;
 
@@ -232,6 +236,12 @@ size_t carve(tts_gpt *h, void *base) {
   h->hbuf = cv.take<uint16_t>((size_t)kMaxRows * F);
   h->hf = cv.take<uint16_t>((size_t)kMaxRows * d);
   h->kv_stage = h->kv_fp8 ? cv.take<uint16_t>((size_t)kMaxPassRows * 2 * d) : nullptr;
+  if (h->kv_fp8) {
+    h->kv_scratch = cv.take<uint16_t>((size_t)kScratchPages * 2 * c.n_head * kPageElems);
+    h->scratch_table = cv.take<int>((size_t)S * h->pps);
+    h->scratch_src = cv.take<int>(kScratchPages);
+    h->scratch_ntok = cv.take<int>(kScratchPages);
+  }
   const size_t attn_rows = h->kv_fp8 ? kMaxPassRows : kMaxRows;   // the 8-bit cache's attention kernel also serves prefill passes
   h->attn_partials = cv.take<float>(attn_rows * c.n_head * kAttnMaxChunks * kAttnPartialFloats);
   h->attn_tickets = cv.take<unsigned int>(attn_rows * c.n_head);
@@ -294,6 +304,14 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
     cudaError_t e = launch_kv_quantize(h->kv_stage, kvl, aa.page_table, aa.row_stream, aa.row_pos, aa.pps, aa.H, R, st, pdl);
     if (e != cudaSuccess) return e;
     h->launches += 1;
+    if (!aa.old_pages_final && h->pass_scratch > 0 && h->use_attn_mma && R >= kAttnPrefillRows) {
+      // prefill pass: decode the pages its rows attend over into bf16 scratch pages, then the tensor-core kernel
+      e = launch_kv_dequant_pages(kvl, h->kv_scratch, h->scratch_src, h->scratch_ntok, h->pass_scratch, aa.H, st, pdl);
+      if (e != cudaSuccess) return e;
+      h->launches += 1;
+      aa.kv_layer = h->kv_scratch; aa.page_table = h->scratch_table; aa.err = h->dev_err; aa.row_order = nullptr;
+      return launch_attention_prefill_mma(aa, R, st, pdl);
+    }
     Fp8AttnArgs fa;
     memset(&fa, 0, sizeof fa);
     fa.q = aa.q; fa.kv_layer = kvl; fa.page_table = aa.page_table; fa.row_stream = aa.row_stream; fa.row_pos = aa.row_pos;
@@ -743,10 +761,16 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
   memset(&ps, 0, sizeof ps);
   ps.io = io;
   ps.text_shift = text_shift; ps.text_pos0 = text_pos0; ps.emb_rows = emb_rows_of(c);
+  int scratch_pages = 0;   // 8-bit cache: pages the rows of the pass attend over
   auto flush = [&]() -> int {
     if (ps.n_rows == 0) return TTS_GPT_OK;
     ps.io.n_out = ps.n_out;
     ps.run_row0[ps.n_runs] = (short)ps.n_rows;
+    if (scratch_pages > kScratchPages || !h->kv_fp8) scratch_pages = 0;   // too many pages: the pass attends over the codes
+    ps.n_scratch = scratch_pages;
+    ps.run_scratch0[ps.n_runs] = (short)scratch_pages;
+    ps.scratch_table = h->scratch_table; ps.scratch_src = h->scratch_src; ps.scratch_ntok = h->scratch_ntok;
+    h->pass_scratch = scratch_pages;
     prefill_pass_kernel<<<1, kMaxPassRows, 0, h->stream>>>(ps, h->ps, h->rt, h->io, c.d_model);
     CUDA_TRY(h, cudaGetLastError());
     h->launches += 1;
@@ -756,6 +780,7 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
     if (r) return r;
     if (ps.n_out > 0) r = run_head(h, ps.n_out, ps.n_rows);
     ps.n_rows = 0; ps.n_out = 0; ps.n_runs = 0;
+    scratch_pages = 0; h->pass_scratch = 0;
     return r;
   };
   for (int i = 0; i < n; ++i) {
@@ -765,6 +790,8 @@ static int prefill_impl(tts_gpt_t *h, int32_t n, const void *const *emb, const i
       ps.run_stream[ps.n_runs] = (short)pp.stream_ids[i];
       ps.run_pos0[ps.n_runs] = (short)t;
       ps.run_row0[ps.n_runs] = (short)ps.n_rows;
+      ps.run_scratch0[ps.n_runs] = (short)std::min(scratch_pages, 32767);
+      scratch_pages += (t + take - 1) / kPageTokens + 1;
       ++ps.n_runs;
       ps.n_rows += take;
       t += take;
