@@ -137,13 +137,17 @@ struct LnTcArgs {
   unsigned long long *trace;  // optional timeline trace
   int trace_slot;
 };
-__global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs a) {
+// NP: elements per thread (d <= 256 * NP); the engine instantiates what its d needs.  MINB: CTAs per SM the register
+// allocation must allow: 5 for the many rows of a prefill pass (768 rows then run as 1.04 waves instead of 2.6: 7-8
+// us per launch instead of 10), 1 for decode steps, where the few spills that buys cost more than they save.
+template <int NP, int MINB>
+__global__ void __launch_bounds__(kLnThreads, MINB) layernorm_tc_kernel(const LnTcArgs a) {
   __shared__ float sm[kLnThreads / 32];
   trace_mark(a.trace, a.trace_slot, 0);
   // gamma, beta and the folded bias do not depend on the kernel in front: fetched ahead of the dependency wait
-  float gg[kLnMaxPerThread], bb[kLnMaxPerThread], bs[kLnMaxPerThread];
+  float gg[NP], bb[NP], bs[NP];
 #pragma unroll
-  for (int i = 0; i < kLnMaxPerThread; ++i) {
+  for (int i = 0; i < NP; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     gg[i] = c < a.d ? bf16_bits_to_float(a.g[c]) : 0.f;
     bb[i] = c < a.d ? bf16_bits_to_float(a.b[c]) : 0.f;
@@ -158,9 +162,9 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   // all loads of the row (x, bias and up to 4 partial sums per element) are issued before any is
   // used; the sum itself is taken in a fixed order
   constexpr int kMaxPart = 4;
-  float v[kLnMaxPerThread], pp[kLnMaxPerThread][kMaxPart];
+  float v[NP], pp[NP][kMaxPart];
 #pragma unroll
-  for (int i = 0; i < kLnMaxPerThread; ++i) {
+  for (int i = 0; i < NP; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     v[i] = 0.f;
 #pragma unroll
@@ -176,7 +180,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   }
   float s = 0.f;
 #pragma unroll
-  for (int i = 0; i < kLnMaxPerThread; ++i) {
+  for (int i = 0; i < NP; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     if (c < a.d && a.n_part > 0) {
       float t = v[i] + bs[i];
@@ -190,7 +194,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   const float mu = block_sum(s, sm) / a.d;
   float q = 0.f;
 #pragma unroll
-  for (int i = 0; i < kLnMaxPerThread; ++i) {
+  for (int i = 0; i < NP; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     const float t = c < a.d ? v[i] - mu : 0.f;
     q += t * t;
@@ -198,7 +202,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
   const float rstd = rsqrtf(block_sum(q, sm) / a.d + a.eps);
   uint16_t *hid = (a.io && a.io->out_hidden) ? a.io->out_hidden + (size_t)(a.out_slot ? a.out_slot[j] : j) * a.d : nullptr;
 #pragma unroll
-  for (int i = 0; i < kLnMaxPerThread; ++i) {
+  for (int i = 0; i < NP; ++i) {
     const int c = threadIdx.x + i * kLnThreads;
     if (c < a.d) {
       const uint16_t y = float_to_bf16_bits((v[i] - mu) * rstd * gg[i] + bb[i]);

@@ -359,7 +359,12 @@ int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int
   la.add_bias = add_bias; la.g = g; la.b = b; la.eps = h->cfg.ln_eps; la.out_img = out_img; la.out_plain = out_plain;
   la.gather = gather; la.out_slot = out_slot; la.io = io; la.write_back = write_back;
   trace_attach(h, la);
-  CUDA_TRY(h, launch_kernel(layernorm_tc_kernel, dim3(rows), dim3(kLnThreads), 0, h->stream, h->use_pdl, la));
+  const int np = (h->cfg.d_model + kLnThreads - 1) / kLnThreads;
+  const dim3 grid(rows), block(kLnThreads);
+  if (np <= 1) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<1, 1>, grid, block, 0, h->stream, h->use_pdl, la));
+  else if (np <= 5 && rows > kMaxRows) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<5, 5>, grid, block, 0, h->stream, h->use_pdl, la));
+  else if (np <= 5) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<5, 1>, grid, block, 0, h->stream, h->use_pdl, la));
+  else CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<kLnMaxPerThread, 1>, grid, block, 0, h->stream, h->use_pdl, la));
   h->launches += 1;
   return TTS_GPT_OK;
 }
