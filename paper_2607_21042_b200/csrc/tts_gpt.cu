@@ -91,8 +91,8 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
-  int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); 768 measured best:
-                                 // FC1 then has 240 CTAs, one wave at two CTAs per SM, where 1024 rows need 320
+  int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); set at creation
+                                 // to the most row tiles whose widest linear still runs as one wave of two CTAs per SM
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
   bool use_attn_mma = true;      // tensor-core attention in prefill passes (option "attn_mma")
   bool use_attn_prefill = true;  // shared-page attention in prefill passes (option "attn_prefill")
@@ -690,6 +690,15 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
     h->n_sm = sms;
+  {
+    // rows per prefill pass: the wide linears run two CTAs per SM; a pass of t row tiles gives the widest linear
+    // t x (features / 128) x k-ranges CTAs, and one CTA too many doubles its time.  Measured on 148 SMs with this
+    // model (FC1: 40 feature tiles): 88946 prefix rows in 301 / 279 / 308 ms at 6 / 7 / 8 row tiles.
+    const tts_gpt_config_t &c = h->cfg;
+    const int widest = std::max(std::max((c.d_ff + 127) / 128, (3 * c.d_model + 127) / 128), tcw_ksplit_resid(c.d_ff) * ((c.d_model + 127) / 128));
+    const int t = std::max(1, std::min(kMaxPassRows / kMaxRows, 2 * h->n_sm / std::max(1, widest)));
+    h->prefill_pass_rows = t * kMaxRows;
+  }
   *out = h;
   return TTS_GPT_OK;
 }
