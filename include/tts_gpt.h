@@ -224,7 +224,7 @@ int32_t tts_gpt_debug_check_canaries(tts_gpt_t *h, int32_t *bad_bytes);
  * step graphs.  Names: "graph", "pdl", "tc" and "tc_min_rows" (tensor-core
  * linears), "prefill_pass_rows" (rows per prefill pass: a multiple of 128 up to 1024; the default is chosen at creation
  * from the SM count and the model width, 896 for the 24-layer model on 148 SMs; passes of more than 128 rows need
- * the tensor-core path), "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
+ * the tensor-core path), "attn_tc", "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
  * "fc2_ksplit"; "poison_free_pages" (test aid standing in for a memory checker: every free page, and
  * from then on every released page, is filled with NaN in all layers, so that a kernel reading a slot no
  * token was written to poisons its result).  Unknown name or value out of range: TTS_GPT_E_ARG. */
@@ -295,6 +295,9 @@ int32_t tts_gpt_op_attention(int32_t R, int32_t n_head, const float *q, const vo
  * cluster_size -2: the prefill variant the engine uses, same requirement on the rows: 16 consecutive rows
  * per CTA, Q K^T and P V on the tensor cores (bf16 operands: Q and the softmax weights are rounded to
  * bf16, sums and accumulators stay fp32).  It has no waits.
+ * cluster_size -3: the prefill variant the engine uses for passes of more than 128 rows, same requirement on
+ * the rows: 128 consecutive rows per CTA, Q K^T and P V as tcgen05 instructions with the scores and the
+ * output in tensor memory (same roundings as -2); its waits are bounded.
  * The waits on the copies of variants 0 and -1 are bounded; this stand-alone entry does not report an
  * expired wait (the engine does, as TTS_GPT_E_TIMEOUT).  q, out and kv_layer must be 16-byte aligned. */
 int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, const void *kv_layer,

@@ -18,6 +18,7 @@
 #include "attention.cuh"
 #include "attention_prefill.cuh"
 #include "gemm_tc.cuh"
+#include "attention_prefill_tc.cuh"
 #include "elementwise.cuh"
 #include "kv_pages.cuh"
 #include "kv_fp8.cuh"
@@ -91,6 +92,7 @@ struct tts_gpt {
   int pending_parts = 0;        // k-range partial sums of the last FC2 still to be folded into x
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
+  bool use_attn_tc = true;   // prefill passes of more than 128 rows: attention on tcgen05 (option "attn_tc")
   int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); set at creation
                                  // to the most row tiles whose widest linear still runs as one wave of two CTAs per SM
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
@@ -310,6 +312,7 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
       if (e != cudaSuccess) return e;
       h->launches += 1;
       aa.kv_layer = h->kv_scratch; aa.page_table = h->scratch_table; aa.err = h->dev_err; aa.row_order = nullptr;
+      if (h->use_attn_tc && R > kMaxRows) return launch_attention_prefill_tc(aa, R, st, pdl);
       return launch_attention_prefill_mma(aa, R, st, pdl);
     }
     Fp8AttnArgs fa;
@@ -329,6 +332,8 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
   aa.row_order = aa.old_pages_final ? h->rt.row_order : nullptr;   // written by the decode step's set-up kernel
   // prefill passes: rows of one stream share their pages (one CTA per 16 rows and head on the tensor cores;
   // the CUDA-core variant with 8 rows per CTA stays selectable)
+  // (passes of several row tiles: 128 rows per CTA on tcgen05)
+  if (!aa.old_pages_final && h->use_attn_mma && h->use_attn_tc && R > kMaxRows) return launch_attention_prefill_tc(aa, R, st, pdl);
   if (!aa.old_pages_final && h->use_attn_mma && R >= kAttnPrefillRows) return launch_attention_prefill_mma(aa, R, st, pdl);
   if (!aa.old_pages_final && h->use_attn_prefill && R >= kAttnPrefillRows) return launch_attention_prefill(aa, R, st, pdl);
   const bool stream = h->attn_stream_min_pairs > 0 ? R * aa.H >= h->attn_stream_min_pairs : attention_use_stream(R, aa.H, h->n_sm);
@@ -1062,6 +1067,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "tc") h->use_tc = on;
   else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be a multiple of 128 from 128 to 1024"); h->prefill_pass_rows = value; }
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
+  else if (k == "attn_tc") h->use_attn_tc = on;
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;
   else if (k == "attn_stream") h->use_attn_stream = on;
@@ -1290,8 +1296,9 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
   if (R < 1 || R > 65535 || n_head < 1 || !q || !kv_layer || !page_table || !row_stream || !row_pos || !out ||
       pages_per_stream < 1)
     return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: bad argument");
-  if (cluster_size != -2 && cluster_size != -1 && cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
-    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be -2, -1, 0, 1, 2, 4 or 8");
+  if (cluster_size != -3 && cluster_size != -2 && cluster_size != -1 && cluster_size != 0 && cluster_size != 1 && cluster_size != 2 &&
+      cluster_size != 4 && cluster_size != 8)
+    return fail(nullptr, TTS_GPT_E_ARG, "op_attention_cluster: cluster_size must be -3, -2, -1, 0, 1, 2, 4 or 8");
   AttnArgs a;
   memset(&a, 0, sizeof a);
   a.q = q; a.kv_layer = (const uint16_t *)kv_layer; a.page_table = page_table; a.row_stream = row_stream;
@@ -1300,7 +1307,11 @@ int32_t tts_gpt_op_attention_cluster(int32_t R, int32_t n_head, const float *q, 
     CUDA_TRY(nullptr, launch_attention_stream(a, R, (cudaStream_t)cuda_stream, false));
     return TTS_GPT_OK;
   }
-  if (cluster_size == -2) {   // rows must be stream-major with ascending positions, as in a prefill pass
+  if (cluster_size == -3) {   // rows must be stream-major with ascending positions, as in a prefill pass
+    CUDA_TRY(nullptr, launch_attention_prefill_tc(a, R, (cudaStream_t)cuda_stream, false));
+    return TTS_GPT_OK;
+  }
+  if (cluster_size == -2) {   // same requirement on the rows
     CUDA_TRY(nullptr, launch_attention_prefill_mma(a, R, (cudaStream_t)cuda_stream, false));
     return TTS_GPT_OK;
   }

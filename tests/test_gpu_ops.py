@@ -204,10 +204,11 @@ def test_attention_streaming_variant_rows_of_one_stream():
         assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -8 * np.abs(ref).max() + 1e-5
 
 
-@pytest.mark.parametrize("variant", [-1, -2])
+@pytest.mark.parametrize("variant", [-1, -2, -3])
 def test_attention_prefill_variant_mixed_streams(variant):
     # rows as a prefill pass orders them: stream-major, positions ascending; runs of 5, 11, 1 and 40 rows so
-    # that CTAs of 8 (variant -1) or 16 rows (variant -2) hold one, two and three streams, starting inside a context
+    # that CTAs of 8 (variant -1), 16 (variant -2) or 128 rows (variant -3) hold one, two and more streams, starting
+    # inside a context
     rng = np.random.default_rng(79)
     H = 3
     ctxs = [70, 200, 1, 333]
@@ -225,6 +226,29 @@ def test_attention_prefill_variant_mixed_streams(variant):
     for r, (s_, p_) in enumerate(rows):
         ref = _attention_ref(q[r].astype(np.float64), Ks[s_][:p_ + 1], Vs[s_][:p_ + 1], H)
         assert np.max(np.abs(got[r] - ref)) <= tol * np.abs(ref).max() + 1e-5, (r, s_, p_)
+
+
+def test_attention_prefill_tcgen05_long_runs():
+    """The 128-row tcgen05 variant on a pass-like row list of 300 rows: a stream's tail that starts deep inside its
+    context (pages the tile's rows only read), a whole short stream, a stream of 130 rows crossing a tile edge, one
+    row at position 0, and a ragged last tile."""
+    rng = np.random.default_rng(80)
+    H = 2
+    ctxs = [900, 40, 130, 1, 160]
+    kv, pt, Ks, Vs = _attention_case(rng, H, ctxs, 24, 32)
+    rows = ([(0, p) for p in range(860, 900)] + [(1, p) for p in range(40)] + [(2, p) for p in range(130)] + [(3, 0)] +
+            [(4, p) for p in range(71, 160)])
+    R = len(rows)
+    assert R == 300
+    q = rng.standard_normal(size=(R, H * 64)).astype(np.float32)
+    out = B.op_attention_cluster(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                                 torch.tensor([s for s, _ in rows], dtype=torch.int32, device=DEV),
+                                 torch.tensor([p for _, p in rows], dtype=torch.int32, device=DEV), -3)
+    torch.cuda.synchronize()
+    got = bits_to_f64(out)
+    for r, (s_, p_) in enumerate(rows):
+        ref = _attention_ref(q[r].astype(np.float64), Ks[s_][:p_ + 1], Vs[s_][:p_ + 1], H)
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -7 * np.abs(ref).max() + 1e-5, (r, s_, p_)
 
 
 @pytest.mark.parametrize("R,d", [(1, 256), (5, 1280), (128, 1280), (3, 2048), (2, 128)])
