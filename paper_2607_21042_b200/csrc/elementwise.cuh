@@ -137,11 +137,9 @@ struct LnTcArgs {
   unsigned long long *trace;  // optional timeline trace
   int trace_slot;
 };
-// NP: elements per thread (d <= 256 * NP); the engine instantiates what its d needs.  MINB: CTAs per SM the register
-// allocation must allow: 5 for the many rows of a prefill pass (768 rows then run as 1.04 waves instead of 2.6: 7-8
-// us per launch instead of 10), 1 for decode steps, where the few spills that buys cost more than they save.
-template <int NP, int MINB>
-__global__ void __launch_bounds__(kLnThreads, MINB) layernorm_tc_kernel(const LnTcArgs a) {
+// NP: elements per thread (d <= 256 * NP); the engine instantiates what its d needs.
+template <int NP>
+__global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs a) {
   __shared__ float sm[kLnThreads / 32];
   trace_mark(a.trace, a.trace_slot, 0);
   // gamma, beta and the folded bias do not depend on the kernel in front: fetched ahead of the dependency wait
@@ -209,6 +207,127 @@ __global__ void __launch_bounds__(kLnThreads, MINB) layernorm_tc_kernel(const Ln
       if (a.out_img) *reinterpret_cast<uint16_t *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset_tiled(j, c, a.d)) = y;
       if (a.out_plain) a.out_plain[(size_t)j * a.d + c] = y;
       if (hid) hid[c] = y;
+    }
+  }
+  trace_mark(a.trace, a.trace_slot, 2);
+}
+
+// The same operation for the many rows of a large prefill pass: one warp per row, lane l owning the
+// groups of 4 consecutive columns f = l + 32 * m, so that every load instruction of the warp covers 512
+// contiguous bytes, every store of bf16 values 256, and the two reductions are warp shuffles with no block
+// barrier.  The fold into the residual stream keeps the order of layernorm_tc_kernel (x + bias + partial 0
+// + partial 1 + ...), so x comes out bit-identical.  Needs d % 8 == 0 and d <= 128 * NF.
+constexpr int kLnRowsWarps = 4;
+__device__ __forceinline__ void unpack_bf16x4(const uint2 p, float (&f)[4]) {
+  f[0] = __uint_as_float(p.x << 16); f[1] = __uint_as_float(p.x & 0xffff0000u);
+  f[2] = __uint_as_float(p.y << 16); f[3] = __uint_as_float(p.y & 0xffff0000u);
+}
+__device__ __forceinline__ void add4(float (&v)[4], const float4 q) { v[0] += q.x; v[1] += q.y; v[2] += q.z; v[3] += q.w; }
+template <int NF>
+__global__ void __launch_bounds__(kLnRowsWarps * 32) layernorm_rows_kernel(const LnTcArgs a, int rows) {
+  trace_mark(a.trace, a.trace_slot, 0);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int nf = a.d >> 2;
+  const bool fold = a.n_part > 0;
+  // gamma, beta and the folded bias do not depend on the kernel in front: fetched (packed) ahead of the wait
+  uint2 gp[NF], bp[NF], sp[NF];
+#pragma unroll
+  for (int m = 0; m < NF; ++m) {
+    const int f = lane + 32 * m;
+    gp[m] = bp[m] = sp[m] = make_uint2(0, 0);
+    if (f < nf) {
+      gp[m] = __ldg(reinterpret_cast<const uint2 *>(a.g) + f);
+      bp[m] = __ldg(reinterpret_cast<const uint2 *>(a.b) + f);
+      if (fold && a.add_bias) sp[m] = __ldg(reinterpret_cast<const uint2 *>(a.add_bias) + f);
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  trace_mark(a.trace, a.trace_slot, 1);
+  const int j = blockIdx.x * kLnRowsWarps + w;
+  if (j >= rows) return;
+  const int r = a.gather ? a.gather[j] : j;
+  float *xr = a.x + (size_t)r * a.d;
+  const float4 *pr = reinterpret_cast<const float4 *>(
+      a.partials + (((size_t)(r >> 7) * a.n_part) * kMaxRows + (r & (kMaxRows - 1))) * a.part_cols);
+  const size_t pstride = (size_t)kMaxRows * a.part_cols / 4;
+  // the row is latency-bound: the loads of x and of two partial sums at a time are all issued before
+  // the first of them is used, and nothing is stored until every load has come back
+  float v[NF][4];
+#pragma unroll
+  for (int m = 0; m < NF; ++m) {
+    const int f = lane + 32 * m;
+    const float4 x = f < nf ? __ldcg(reinterpret_cast<const float4 *>(xr) + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+    v[m][0] = x.x; v[m][1] = x.y; v[m][2] = x.z; v[m][3] = x.w;
+  }
+  if (fold) {
+    float4 q[NF][2];
+#pragma unroll
+    for (int pp = 0; pp < 4; pp += 2) {
+      if (pp < a.n_part) {
+        const bool two = pp + 1 < a.n_part;
+#pragma unroll
+        for (int m = 0; m < NF; ++m) {
+          const int f = lane + 32 * m;
+          q[m][0] = q[m][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (f < nf) {
+            q[m][0] = __ldcg(pr + pp * pstride + f);
+            if (two) q[m][1] = __ldcg(pr + (pp + 1) * pstride + f);
+          }
+        }
+        if (pp == 0) {
+#pragma unroll
+          for (int m = 0; m < NF; ++m) {
+            float bs[4];
+            unpack_bf16x4(sp[m], bs);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[m][k] += bs[k];
+          }
+        }
+#pragma unroll
+        for (int m = 0; m < NF; ++m) { add4(v[m], q[m][0]); add4(v[m], q[m][1]); }
+      }
+    }
+    if (a.write_back) {
+#pragma unroll
+      for (int m = 0; m < NF; ++m) {
+        const int f = lane + 32 * m;
+        if (f < nf) reinterpret_cast<float4 *>(xr)[f] = make_float4(v[m][0], v[m][1], v[m][2], v[m][3]);
+      }
+    }
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int m = 0; m < NF; ++m) s += (v[m][0] + v[m][1]) + (v[m][2] + v[m][3]);
+  const float mu = warp_sum(s) / a.d;
+  float qq = 0.f;
+#pragma unroll
+  for (int m = 0; m < NF; ++m) {
+    if (lane + 32 * m < nf) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { const float t = v[m][k] - mu; qq += t * t; }
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(qq) / a.d + a.eps);
+  uint16_t *hid = (a.io && a.io->out_hidden) ? a.io->out_hidden + (size_t)(a.out_slot ? a.out_slot[j] : j) * a.d : nullptr;
+#pragma unroll
+  for (int m = 0; m < NF; ++m) {
+    const int f = lane + 32 * m;
+    if (f < nf) {
+      float gg[4], bb[4];
+      unpack_bf16x4(gp[m], gg);
+      unpack_bf16x4(bp[m], bb);
+      uint32_t y[2];
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const uint32_t lo = float_to_bf16_bits((v[m][2 * k] - mu) * rstd * gg[2 * k] + bb[2 * k]);
+        const uint32_t hi = float_to_bf16_bits((v[m][2 * k + 1] - mu) * rstd * gg[2 * k + 1] + bb[2 * k + 1]);
+        y[k] = lo | (hi << 16);
+      }
+      const uint2 yy = make_uint2(y[0], y[1]);
+      if (a.out_img) *reinterpret_cast<uint2 *>(reinterpret_cast<unsigned char *>(a.out_img) + act_image_offset_tiled(j, f * 4, a.d)) = yy;
+      if (a.out_plain) *reinterpret_cast<uint2 *>(a.out_plain + (size_t)j * a.d + f * 4) = yy;
+      if (hid) *reinterpret_cast<uint2 *>(hid + f * 4) = yy;
     }
   }
   trace_mark(a.trace, a.trace_slot, 2);

@@ -366,10 +366,15 @@ int launch_ln_tc(tts_gpt *h, int rows, const uint16_t *g, const uint16_t *b, int
   trace_attach(h, la);
   const int np = (h->cfg.d_model + kLnThreads - 1) / kLnThreads;
   const dim3 grid(rows), block(kLnThreads);
-  if (np <= 1) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<1, 1>, grid, block, 0, h->stream, h->use_pdl, la));
-  else if (np <= 5 && rows > kMaxRows) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<5, 5>, grid, block, 0, h->stream, h->use_pdl, la));
-  else if (np <= 5) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<5, 1>, grid, block, 0, h->stream, h->use_pdl, la));
-  else CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<kLnMaxPerThread, 1>, grid, block, 0, h->stream, h->use_pdl, la));
+  if (rows > kMaxRows && h->cfg.d_model % 8 == 0) {
+    // the many rows of a large prefill pass: one warp per row
+    const dim3 rgrid((rows + kLnRowsWarps - 1) / kLnRowsWarps), rblock(kLnRowsWarps * 32);
+    if (np <= 1) CUDA_TRY(h, launch_kernel(layernorm_rows_kernel<2>, rgrid, rblock, 0, h->stream, h->use_pdl, la, rows));
+    else if (np <= 5) CUDA_TRY(h, launch_kernel(layernorm_rows_kernel<10>, rgrid, rblock, 0, h->stream, h->use_pdl, la, rows));
+    else CUDA_TRY(h, launch_kernel(layernorm_rows_kernel<2 * kLnMaxPerThread>, rgrid, rblock, 0, h->stream, h->use_pdl, la, rows));
+  } else if (np <= 1) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<1>, grid, block, 0, h->stream, h->use_pdl, la));
+  else if (np <= 5) CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<5>, grid, block, 0, h->stream, h->use_pdl, la));
+  else CUDA_TRY(h, launch_kernel(layernorm_tc_kernel<kLnMaxPerThread>, grid, block, 0, h->stream, h->use_pdl, la));
   h->launches += 1;
   return TTS_GPT_OK;
 }
