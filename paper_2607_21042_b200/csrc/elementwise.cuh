@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kLnThreads) layernorm_tc_kernel(const LnTcArgs
 // contiguous bytes, every store of bf16 values 256, and the two reductions are warp shuffles with no block
 // barrier.  The fold into the residual stream keeps the order of layernorm_tc_kernel (x + bias + partial 0
 // + partial 1 + ...), so x comes out bit-identical.  Needs d % 8 == 0 and d <= 128 * NF.
-constexpr int kLnRowsWarps = 4;
+constexpr int kLnRowsWarps = 2;
 __device__ __forceinline__ void unpack_bf16x4(const uint2 p, float (&f)[4]) {
   f[0] = __uint_as_float(p.x << 16); f[1] = __uint_as_float(p.x & 0xffff0000u);
   f[2] = __uint_as_float(p.y << 16); f[3] = __uint_as_float(p.y & 0xffff0000u);
