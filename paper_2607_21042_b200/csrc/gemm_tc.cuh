@@ -113,6 +113,46 @@ __global__ void pack_weight_image_int4_kernel(const uint32_t *__restrict__ w, in
   dst[unit] = v;
 }
 
+// int4 weights for prefill passes of several row tiles: the images of a layer's four linears (integer
+// codes) times the group scales, rounded once to bf16, into a scratch image of the same layout, so that
+// the pass runs the ungrouped kernel.  One thread per 16-byte unit; a unit lies in one row and one
+// 128-column group.  The codes and scales do not depend on the kernels in front and are fetched ahead
+// of the dependency wait; the stores come after it (the previous layer's linears read the scratch).
+struct DequantImgArgs {
+  const uint4 *src[4];
+  uint4 *dst[4];
+  const uint16_t *scales[4];   // tiled scales [N/8][K/128][8]
+  int N[4], K[4];
+  unsigned long long unit_end[4];   // running totals of 16-byte units
+};
+__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t codes, float sc) {
+  return pack_bf16x2(__uint_as_float(codes << 16) * sc, __uint_as_float(codes & 0xffff0000u) * sc);
+}
+__global__ void __launch_bounds__(256) dequant_weight_images_kernel(const DequantImgArgs a) {
+  const unsigned long long unit = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  int s = 0;
+  while (s < 3 && unit >= a.unit_end[s]) ++s;
+  const bool live = unit < a.unit_end[3];
+  uint4 v = make_uint4(0, 0, 0, 0);
+  float sc = 0.f;
+  size_t local = 0;
+  if (live) {
+    local = (size_t)(unit - (s ? a.unit_end[s - 1] : 0ull));
+    const int KC = a.K[s] / 64;
+    const int within = (int)(local % (kTcABytes / 16));
+    const size_t blk = local / (kTcABytes / 16);
+    const int kc = (int)(blk % KC), nt = (int)(blk / KC);
+    const int n = nt * 128 + (within >> 3);
+    if (n < a.N[s]) {
+      v = __ldg(a.src[s] + local);
+      sc = bf16_bits_to_float(__ldg(a.scales[s] + ((size_t)(n >> 3) * (a.K[s] / 128) + (kc >> 1)) * 8 + (n & 7)));
+    }
+  }
+  pdl_launch_dependents();
+  pdl_wait();
+  if (live) a.dst[s][local] = make_uint4(scale_bf16x2(v.x, sc), scale_bf16x2(v.y, sc), scale_bf16x2(v.z, sc), scale_bf16x2(v.w, sc));
+}
+
 inline cudaError_t launch_pack_image(int wf, int N, int K, const void *w, void *img, cudaStream_t st) {
   const size_t units = weight_image_bytes(N, K) / 16;
   const unsigned blocks = (unsigned)((units + 255) / 256);
@@ -211,6 +251,8 @@ struct GemmTcArgs {
   int out_stride;
   void *out_img;            // EPI_GELU: activation image of the next linear (row length N)
   int gelu_tanh;
+  int w_written_in_stream;  // wide kernel: w_img is written by an earlier kernel of the stream (dequantized scratch
+                            // image), so no weight copy may start ahead of the dependency wait
   uint16_t *kv_layer;
   uint16_t *kv_stage;       // if set, K/V rows go here as bf16 [B][2][d] instead of into their page slots (8-bit KV cache)
   const int *page_table, *row_stream, *row_pos;
@@ -575,7 +617,7 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   const unsigned char *gX = reinterpret_cast<const unsigned char *>(a.act_img) + ((size_t)blockIdx.z * KC + kc0) * (kMaxRows * 128);
 
   const int pre = min(n_it, n_stage);
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && !a.w_written_in_stream) {
     for (int i = 0; i < pre; ++i) {   // weights do not depend on the previous kernel
       mbar_expect_tx(full + i, kTwStageBytes);
       bulk_copy_g2s(ring + (size_t)i * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + i);
@@ -586,6 +628,12 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   trace_mark(a.trace, a.trace_slot, 1);
   if (warp == 0) {
     if (lane == 0) {
+      if (a.w_written_in_stream) {   // a weight image that a kernel earlier in the stream wrote: only after the wait
+        for (int i = 0; i < pre; ++i) {
+          mbar_expect_tx(full + i, kTwStageBytes);
+          bulk_copy_g2s(ring + (size_t)i * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + i);
+        }
+      }
       for (int i = 0; i < pre; ++i)
         bulk_copy_g2s(ring + (size_t)i * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + i);
       for (int i = pre; i < n_it; ++i) {

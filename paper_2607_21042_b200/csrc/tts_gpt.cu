@@ -93,6 +93,8 @@ struct tts_gpt {
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
   bool use_attn_tc = true;   // prefill passes of more than 128 rows: attention on tcgen05 (option "attn_tc")
+  bool use_w4_dequant = true;   // int4 weights, prefill passes of more than 128 rows: the layer's weights dequantized to bf16 once per pass (option "w4_prefill_dequant")
+  char *wq_scratch[4] = {nullptr, nullptr, nullptr, nullptr};   // int4: bf16 images of one layer's QKV / O / FC1 / FC2 weights
   int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); set at creation
                                  // to the most row tiles whose widest linear still runs as one wave of two CTAs per SM
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
@@ -256,6 +258,10 @@ size_t carve(tts_gpt *h, void *base) {
     h->hf_img = cv.take<char>(act_image_bytes(d));
     h->partials_floats = (size_t)kTiles * std::max(kTcKSplit, kTwMaxPartials) * kMaxRows * d;   // [row tile][k-range][128][d]
     h->partials = cv.take<float>(h->partials_floats);
+    if (c.wfmt == WF_INT4) {
+      const int NK[4][2] = {{3 * d, d}, {d, d}, {F, d}, {d, F}};
+      for (int i = 0; i < 4; ++i) h->wq_scratch[i] = NK[i][1] % 128 == 0 ? cv.take<char>(weight_image_bytes(NK[i][0], NK[i][1])) : nullptr;
+    }
   }
   return cv.off;
 }
@@ -396,14 +402,39 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
   const int o_ks = wide ? tcw_ksplit_resid(d) : kTcKSplit;
   const int f2_ks = wide ? tcw_ksplit_resid(c.d_ff) : kTcKSplit;
   const int o_parts = o_ks > 1 ? o_ks : 0, f2_parts = f2_ks > 1 ? f2_ks : 0;   // 0: the linear added into x itself
+  // int4 weights in a pass of several row tiles: the layer's four weight images are dequantized (code x group
+  // scale, one rounding to bf16) into scratch images and the linears run ungrouped; the kernel with per-group
+  // accumulators needs twice the registers and runs one CTA per SM
+  const bool deq = wide && c.wfmt == WF_INT4 && h->use_w4_dequant && h->wq_scratch[0] && h->wq_scratch[1] &&
+                   h->wq_scratch[2] && h->wq_scratch[3];
+  auto dequantized = [&](GemmTcArgs &a, int which) {
+    if (!deq) return;
+    a.w_img = h->wq_scratch[which]; a.wfmt = WF_BF16; a.scales = nullptr; a.w_written_in_stream = 1;
+  };
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
+    int rc;
+    if (deq) {
+      const PackedLinear *pl[4] = {&L.qkv, &L.o, &L.fc1, &L.fc2};
+      DequantImgArgs da;
+      memset(&da, 0, sizeof da);
+      unsigned long long end = 0;
+      for (int i = 0; i < 4; ++i) {
+        da.src[i] = (const uint4 *)pl[i]->w_img; da.dst[i] = (uint4 *)h->wq_scratch[i]; da.scales[i] = pl[i]->s;
+        da.N[i] = pl[i]->N; da.K[i] = pl[i]->K;
+        end += weight_image_bytes(pl[i]->N, pl[i]->K) / 16;
+        da.unit_end[i] = end;
+      }
+      CUDA_TRY(h, launch_kernel(dequant_weight_images_kernel, dim3((unsigned)((end + 255) / 256)), dim3(256), 0, st, pdl, da));
+      h->launches += 1;
+    }
     // fold the previous layer's FC2 partial sums into x, then LN1 -> image
-    int rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : f2_parts, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
-                          h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
+    rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : f2_parts, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
+                      h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
+    dequantized(qa, 0);
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
     qa.kv_stage = h->kv_stage;
@@ -417,16 +448,19 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     trace_attach(h, aa);
     CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, o_ks);
+    dequantized(oa, 1);
     oa.out_f32 = o_parts ? h->partials : h->x; oa.out_stride = d;
     trace_attach(h, oa);
     if ((rc = launch_gemm(h, oa, wide, st, pdl))) return rc;
     rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, o_parts, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs f1 = gemm_args(h, L.fc1, h->a_img, R, EPI_GELU, 1);
+    dequantized(f1, 2);
     f1.out_img = h->h_img; f1.gelu_tanh = c.gelu_tanh;
     trace_attach(h, f1);
     if ((rc = launch_gemm(h, f1, wide, st, pdl))) return rc;
     GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, f2_ks);
+    dequantized(f2, 3);
     f2.out_f32 = f2_parts ? h->partials : h->x; f2.out_stride = d;
     trace_attach(h, f2);
     if ((rc = launch_gemm(h, f2, wide, st, pdl))) return rc;
@@ -1073,6 +1107,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be a multiple of 128 from 128 to 1024"); h->prefill_pass_rows = value; }
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
   else if (k == "attn_tc") h->use_attn_tc = on;
+  else if (k == "w4_prefill_dequant") h->use_w4_dequant = on;
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;
   else if (k == "attn_stream") h->use_attn_stream = on;

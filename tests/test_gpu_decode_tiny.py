@@ -669,6 +669,15 @@ def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
             assert_same_up_to_ties(tk[s], lg[s], tk2[s], lg2[s], "passes of %d rows, stream %d" % (rows, s))
     with pytest.raises(B.TtsGptError):
         eng.set_option("prefill_pass_rows", 200)
+    if wfmt == C.W_INT4_G128:
+        # large passes dequantize a layer's int4 weights to bf16 images by default (one rounding per weight);
+        # switched off, the kernel with per-group accumulators applies the scales to fp32 group sums
+        eng.set_option("w4_prefill_dequant", 0)
+        lg3, tk3 = _run_batch(eng, prefixes, 4)
+        for s in range(S):
+            ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk3[s][:-1])
+            assert_logits_close(lg3[s], ref, "multi-tile prefill with group accumulators, stream %d" % s)
+            assert_same_up_to_ties(tk[s], lg[s], tk3[s], lg3[s], "group accumulators, stream %d" % s)
     eng.destroy()
 
 
