@@ -113,21 +113,21 @@ __global__ void pack_weight_image_int4_kernel(const uint32_t *__restrict__ w, in
   dst[unit] = v;
 }
 
-// int4 weights for prefill passes of several row tiles: the images of a layer's four linears (integer
-// codes) times the group scales, rounded once to bf16, into a scratch image of the same layout, so that
-// the pass runs the ungrouped kernel.  One thread per 16-byte unit; a unit lies in one row and one
-// 128-column group.  The codes and scales do not depend on the kernels in front and are fetched ahead
-// of the dependency wait; the stores come after it (the previous layer's linears read the scratch).
+// int4 weights for prefill passes of several row tiles: a layer's four linears are dequantized (code x
+// group scale, rounded once to bf16) from the packed streaming layout of linear.cuh (half a byte per
+// weight) into scratch operand images, so that the pass runs the ungrouped kernel.  One thread per
+// 16-byte unit of the source = 32 columns of one row inside one 128-column group = four 16-byte units
+// of one k-chunk of the image.  The codes and scales do not depend on the kernels in front and are
+// fetched ahead of the dependency wait; the stores come after it (the previous layer's linears read
+// the scratch).  Image rows past the last 8-row tile of the source are never written: they are zeroed
+// when the engine is created.
 struct DequantImgArgs {
-  const uint4 *src[4];
-  uint4 *dst[4];
+  const uint4 *src[4];         // packed int4 tiles [row tile of 8][K/128][32 lanes]
+  uint4 *dst[4];               // operand images
   const uint16_t *scales[4];   // tiled scales [N/8][K/128][8]
-  int N[4], K[4];
-  unsigned long long unit_end[4];   // running totals of 16-byte units
+  int K[4];
+  unsigned long long unit_end[4];   // running totals of source units
 };
-__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t codes, float sc) {
-  return pack_bf16x2(__uint_as_float(codes << 16) * sc, __uint_as_float(codes & 0xffff0000u) * sc);
-}
 __global__ void __launch_bounds__(256) dequant_weight_images_kernel(const DequantImgArgs a) {
   const unsigned long long unit = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   int s = 0;
@@ -135,22 +135,36 @@ __global__ void __launch_bounds__(256) dequant_weight_images_kernel(const Dequan
   const bool live = unit < a.unit_end[3];
   uint4 v = make_uint4(0, 0, 0, 0);
   float sc = 0.f;
-  size_t local = 0;
+  uint4 *out = nullptr;
   if (live) {
-    local = (size_t)(unit - (s ? a.unit_end[s - 1] : 0ull));
-    const int KC = a.K[s] / 64;
-    const int within = (int)(local % (kTcABytes / 16));
-    const size_t blk = local / (kTcABytes / 16);
-    const int kc = (int)(blk % KC), nt = (int)(blk / KC);
-    const int n = nt * 128 + (within >> 3);
-    if (n < a.N[s]) {
-      v = __ldg(a.src[s] + local);
-      sc = bf16_bits_to_float(__ldg(a.scales[s] + ((size_t)(n >> 3) * (a.K[s] / 128) + (kc >> 1)) * 8 + (n & 7)));
-    }
+    const size_t local = (size_t)(unit - (s ? a.unit_end[s - 1] : 0ull));
+    const int KB = a.K[s] / 128, KC = a.K[s] / 64;
+    const int lane = (int)(local & 31);
+    const size_t tile = local >> 5;
+    const int kb = (int)(tile % KB), rt = (int)(tile / KB);
+    const int row = rt * 8 + (lane >> 2), k = kb * 128 + 32 * (lane & 3);
+    v = __ldg(a.src[s] + local);
+    sc = bf16_bits_to_float(__ldg(a.scales[s] + ((size_t)rt * KB + kb) * 8 + (row & 7)));
+    // units (k % 64) / 8 .. + 3 of image row `row`, k-chunk k / 64; logical unit u sits at u ^ (row % 8)
+    out = a.dst[s] + ((size_t)(row >> 7) * KC + (k >> 6)) * (kTcABytes / 16) + (size_t)(row & 127) * 8;
   }
   pdl_launch_dependents();
   pdl_wait();
-  if (live) a.dst[s][local] = make_uint4(scale_bf16x2(v.x, sc), scale_bf16x2(v.y, sc), scale_bf16x2(v.z, sc), scale_bf16x2(v.w, sc));
+  if (live) {
+    const int lane = (int)(unit & 31);   // unit_end values are multiples of 32
+    const int row7 = (lane >> 2) & 7, u0 = ((32 * (lane & 3)) & 63) >> 3;
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t y[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t pair = (w[q] >> (4 * e)) & 0x000F000Fu;   // columns 2e, 2e+1 of the word, stored as code + 8
+        y[e] = pack_bf16x2((float)((int)(pair & 0xffffu) - 8) * sc, (float)((int)(pair >> 16) - 8) * sc);
+      }
+      out[(u0 + q) ^ row7] = make_uint4(y[0], y[1], y[2], y[3]);
+    }
+  }
 }
 
 inline cudaError_t launch_pack_image(int wf, int N, int K, const void *w, void *img, cudaStream_t st) {

@@ -421,9 +421,9 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
       memset(&da, 0, sizeof da);
       unsigned long long end = 0;
       for (int i = 0; i < 4; ++i) {
-        da.src[i] = (const uint4 *)pl[i]->w_img; da.dst[i] = (uint4 *)h->wq_scratch[i]; da.scales[i] = pl[i]->s;
-        da.N[i] = pl[i]->N; da.K[i] = pl[i]->K;
-        end += weight_image_bytes(pl[i]->N, pl[i]->K) / 16;
+        da.src[i] = (const uint4 *)pl[i]->w; da.dst[i] = (uint4 *)h->wq_scratch[i]; da.scales[i] = pl[i]->s;
+        da.K[i] = pl[i]->K;
+        end += packed_weight_bytes(WF_INT4, pl[i]->N, pl[i]->K) / 16;
         da.unit_end[i] = end;
       }
       CUDA_TRY(h, launch_kernel(dequant_weight_images_kernel, dim3((unsigned)((end + 255) / 256)), dim3(256), 0, st, pdl, da));
@@ -707,6 +707,11 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)(h->kv_fp8 ? kMaxPassRows : kMaxRows) * c.n_head * sizeof(unsigned int), h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_lo, kCanaryByte, kCanaryBytes, h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_hi, kCanaryByte, kCanaryBytes, h->stream);
+  {   // image rows past a matrix's last 8-row tile are never written by the per-pass dequantization
+    const int NK[4][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}};
+    for (int i = 0; i < 4; ++i)
+      if (e == cudaSuccess && h->wq_scratch[i]) e = cudaMemsetAsync(h->wq_scratch[i], 0, weight_image_bytes(NK[i][0], NK[i][1]), h->stream);
+  }
   if (e == cudaSuccess) {
     void *hp = nullptr, *dp = nullptr;
     e = cudaHostAlloc(&hp, sizeof(int), cudaHostAllocMapped);
