@@ -530,7 +530,7 @@ def mid_context(wl):
     return int(np.mean(wl.prefix_lens)) + int(np.mean(wl.decode_lens)) // 2
 
 
-def cpu_baseline(wl, wcache, steps=24):
+def cpu_baseline(wl, wcache, steps=36):
     w = wcache.get(wl.cfg, wl.seed)
     ctx = mid_context(wl)
     all_rate, all_dt = oracle_decode_rate(wl, w, steps, ctx, None)
