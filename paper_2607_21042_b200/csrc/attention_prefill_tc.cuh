@@ -10,9 +10,10 @@
 //     O += P V      M=128 x N=64 (dimensions) x K=64 (tokens), 4 instructions; V is read as stored (token-major =
 //                   MN-major for this product); O stays in tensor memory and is rescaled there when a row's
 //                   maximum moves
-// Warps 0-3 are the softmax threads, warp 4 stages pages (16-byte asynchronous copies into three slots, with the
-// 128-byte swizzle the tensor core expects) and issues the instructions.  The Q K^T of page j+1 and the P V of
-// page j-1 run while page j goes through the softmax.  Every wait is bounded.
+// Warps 0-3 and 4-7 are two softmax groups that take alternate pages, each with its own S, P and O (the two
+// partial results meet at the end); one thread of warp 8 issues the instructions, with Q K^T a page ahead of the
+// groups; warps 9 and 10 stage the K and V halves of the pages (16-byte asynchronous copies into six slots, with
+// the 128-byte swizzle the tensor core expects).  Every wait is bounded.
 #pragma once
 #include "attention_prefill.cuh"
 #include "gemm_tc.cuh"
@@ -20,8 +21,9 @@
 namespace ttsgpt {
 
 constexpr int kPtRows = 128;
-constexpr int kPtThreads = 160;
-constexpr int kPtSlots = 3;
+constexpr int kPtThreads = 352;
+constexpr int kPtSlots = 6;
+constexpr int kPtMergePitch = 65;   // floats per row of the merge buffer: lane = row, conflict-free
 constexpr int kPtMaxJobs = 256;   // two partial long streams + streams of at most 128 rows
 
 __device__ __forceinline__ void pt_cp16(void *smem, const void *gmem, bool real) {
@@ -62,14 +64,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) 
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
-// one page (64 tokens x 128 bytes, K then V) into a slot, chunk j of token row t at chunk j ^ (t & 7)
-__device__ __forceinline__ void pt_stage(unsigned char *slot, const uint16_t *K, const uint16_t *V, int n_here, int lane) {
+// half a page (K or V of one head: 64 tokens x 128 bytes) into its half of a slot, chunk j of token row t at
+// chunk j ^ (t & 7)
+__device__ __forceinline__ void pt_stage(unsigned char *dst, const uint16_t *src, int n_here, int lane) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     const int idx = lane + 32 * i, t = idx >> 3, j = idx & 7;
-    const int off = t * 128 + ((j ^ (t & 7)) << 4);
-    pt_cp16(slot + off, K + (size_t)t * kHeadDim + 8 * j, t < n_here);
-    pt_cp16(slot + kPageElems * 2 + off, V + (size_t)t * kHeadDim + 8 * j, t < n_here);
+    pt_cp16(dst + t * 128 + ((j ^ (t & 7)) << 4), src + (size_t)t * kHeadDim + 8 * j, t < n_here);
   }
   pt_commit();
 }
@@ -78,16 +79,20 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
   extern __shared__ __align__(16) unsigned char pt_smem_raw[];
   unsigned char *base = pt_smem_raw + ((1024u - (smem_u32(pt_smem_raw) & 1023u)) & 1023u);
   unsigned char *Qs = base;                   // 128 rows x 64 dimensions bf16, K-major, 128-byte swizzle
-  unsigned char *Ps = base + 16384;           // 128 rows x 64 tokens bf16, same layout
-  unsigned char *slots = base + 32768;        // [3][K 64 tokens x 128 B | V 64 tokens x 128 B]
-  uint64_t *q_full = reinterpret_cast<uint64_t *>(slots + kPtSlots * 16384);
-  uint64_t *s_full = q_full + 1, *s_free = q_full + 2, *p_full = q_full + 3, *pv_done = q_full + 4;
-  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 5);
+  unsigned char *Ps = base + 16384;           // [2 groups] 128 rows x 64 tokens bf16, same layout
+  unsigned char *slots = base + 49152;        // [6][K 64 tokens x 128 B | V 64 tokens x 128 B]
+  float *Ms = reinterpret_cast<float *>(slots + kPtSlots * 16384);   // [128][65] group 1's O for the merge
+  uint64_t *q_full = reinterpret_cast<uint64_t *>(Ms + kPtRows * kPtMergePitch);
+  uint64_t *s_full = q_full + 1, *s_free = q_full + 3, *p_full = q_full + 5, *pv_done = q_full + 7;   // [2] each, by group
+  uint64_t *page_full = q_full + 9;   // [kPtSlots] K and V of the slot's page have landed
+  uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_full + 9 + kPtSlots);
   volatile int *failed = reinterpret_cast<volatile int *>(tmem_slot + 1);
   __shared__ int row_s[kPtRows], row_p[kPtRows];
   __shared__ int seg_stream[kPtRows], seg_i0[kPtRows], seg_i1[kPtRows], seg_last[kPtRows];
   __shared__ unsigned short jobs[kPtMaxJobs];   // (run << 8) | page, in run order
   __shared__ int n_job_s;
+  __shared__ int job_ph[kPtMaxJobs];            // physical page of each job
+  __shared__ float ref1_s[kPtRows], l1_s[kPtRows];   // group 1's reference score and sum per row
 
   const int h = blockIdx.y, r0 = blockIdx.z * kPtRows;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,10 +103,12 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
     row_p[threadIdx.x] = r < R ? a.row_pos[r] : -1;
   }
   if (threadIdx.x == 0) {
-    mbar_init(q_full, kPtRows); mbar_init(s_full, 1); mbar_init(s_free, kPtRows); mbar_init(p_full, kPtRows); mbar_init(pv_done, 1);
+    mbar_init(q_full, kPtRows);
+    for (int sl = 0; sl < kPtSlots; ++sl) mbar_init(page_full + sl, 2);
+    for (int g = 0; g < 2; ++g) { mbar_init(s_full + g, 1); mbar_init(s_free + g, kPtRows); mbar_init(p_full + g, kPtRows); mbar_init(pv_done + g, 1); }
     *failed = 0;
   }
-  if (warp == 4) tmem_alloc(tmem_slot, 128);   // S: columns 0-63, O: columns 64-127
+  if (warp == 8) tmem_alloc(tmem_slot, 256);   // S of group g: columns 64 g .. + 63, O of group g: columns 128 + 64 g .. + 63
   __syncthreads();
   if (threadIdx.x == 0) {
     const int n_rows = min(R - r0, kPtRows);
@@ -123,66 +130,89 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   const int n_job = n_job_s;
+  // the physical pages of all jobs up front (the page table is final before the pass's first kernel starts): a
+  // page-table read in front of every page's copies would put an L2 round trip into each turn of the producer's loop
+  for (int j = threadIdx.x; j < n_job; j += kPtThreads)
+    job_ph[j] = a.page_table[(size_t)seg_stream[jobs[j] >> 8] * a.pps + (jobs[j] & 255)];
+  __syncthreads();
   pdl_launch_dependents();
   pdl_wait();     // Q and the K/V rows of this pass were written by the QKV kernel in front
   trace_mark(a.trace, a.trace_slot, 1);
 
-  if (warp == 4) {
-    // ---- pages into the slots, instructions to the tensor core ----
+  if (warp >= 9) {
+    // ---- copy warps: warp 9 brings the K half of every page into its slot, warp 10 the V half ----
+    const int part = warp - 9;
     auto stage = [&](int j) {
       if (j < n_job) {
         const int sg = jobs[j] >> 8, pg = jobs[j] & 255;
         const int n_here = min(kPageTokens, seg_last[sg] + 1 - pg * kPageTokens);
-        const int ph = a.page_table[(size_t)seg_stream[sg] * a.pps + pg];
-        const uint16_t *K = a.kv_layer + (((size_t)ph * 2 + 0) * a.H + h) * kPageElems;
-        pt_stage(slots + (size_t)(j % kPtSlots) * 16384, K, K + (size_t)a.H * kPageElems, n_here, lane);
+        const uint16_t *src = a.kv_layer + (((size_t)job_ph[j] * 2 + part) * a.H + h) * kPageElems;
+        pt_stage(slots + (size_t)(j % kPtSlots) * 16384 + part * (kPageElems * 2), src, n_here, lane);
       } else {
         pt_commit();   // an empty group keeps the count of groups per job uniform
       }
     };
     stage(0); stage(1); stage(2);
-    if (lane == 0) tc_wait(q_full, 0, failed, a.err);
-    const uint32_t idesc_qk = tc_instr_desc(kPtRows, 64);
-    const uint32_t idesc_pv = tc_instr_desc(kPtRows, 64) | (1u << 16);   // B (= V) is MN-major: token rows of 64 dimensions
-    auto pv = [&](int j) {   // O (+)= P V for job j
-      tc_wait(p_full, (uint32_t)j & 1u, failed, a.err);
-      tc_fence_after_sync();
-      const uint64_t dp = tc_smem_desc(Ps), dv = tc_smem_desc(slots + (size_t)(j % kPtSlots) * 16384 + kPageElems * 2);
-#pragma unroll
-      for (int k = 0; k < 4; ++k)   // 16 tokens per instruction: 32 bytes along a P row, two 8-row groups (2048 bytes) down V
-        tc_mma(tmem + 64u, dp + 2 * k, dv + 128 * k, idesc_pv, (j == 0 && k == 0) ? 0u : 1u);
-      tc_commit(pv_done);
-    };
-    for (int j = 0; j < n_job; ++j) {
-      // page j + 1 goes into the slot page j - 2 used, free once P V of job j - 2 has completed
-      if (j + 1 >= kPtSlots) {
-        if (lane == 0) tc_wait(pv_done, (uint32_t)(j - 2) & 1u, failed, a.err);
+    pt_wait_but<2>();            // page 0 has landed
+    fence_proxy_async_smem();    // the tensor core reads the slots through the async proxy
+    __syncwarp();
+    if (lane == 0 && n_job > 0) mbar_arrive(page_full);
+    for (int i = 0; i < n_job; ++i) {
+      // page i + 3 goes into the slot page i - 3 used, free once P V of job i - 3 has completed
+      if (i >= 3) {
+        if (lane == 0) tc_wait(pv_done + ((i - 3) & 1), (uint32_t)((i - 3) >> 1) & 1u, failed, a.err);
         __syncwarp();
-        stage(j + 1);
-      } else {
-        pt_commit();
       }
-      pt_wait_but<1>();            // everything but the group just committed: page j has landed
-      fence_proxy_async_smem();    // the tensor core reads the slot through the async proxy
+      stage(i + 3);
+      pt_wait_but<2>();            // everything but the two groups just committed: page i + 1 has landed
+      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        if (j > 0) tc_wait(s_free, (uint32_t)(j - 1) & 1u, failed, a.err);   // the softmax threads hold S of job j - 1 in registers
+      if (lane == 0 && i + 1 < n_job) mbar_arrive(page_full + (i + 1) % kPtSlots);
+    }
+  } else if (warp == 8) {
+    // ---- one thread issues the instructions to the tensor core ----
+    if (lane == 0) {
+      const uint32_t idesc_qk = tc_instr_desc(kPtRows, 64);
+      const uint32_t idesc_pv = tc_instr_desc(kPtRows, 64) | (1u << 16);   // B (= V) is MN-major: token rows of 64 dimensions
+      auto qk = [&](int j) {   // S of group j % 2 = Q K^T for job j; that group holds S of its job before in registers
+        const int g = j & 1, k = j >> 1;
+        tc_wait(page_full + j % kPtSlots, (uint32_t)(j / kPtSlots) & 1u, failed, a.err);
+        if (k > 0) tc_wait(s_free + g, (uint32_t)(k - 1) & 1u, failed, a.err);
         tc_fence_after_sync();
         const uint64_t dq = tc_smem_desc(Qs), dk = tc_smem_desc(slots + (size_t)(j % kPtSlots) * 16384);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) tc_mma(tmem, dq + 2 * k, dk + 2 * k, idesc_qk, k == 0 ? 0u : 1u);   // 16 dimensions per instruction
-        tc_commit(s_full);
-        if (j > 0) pv(j - 1);
+        for (int q = 0; q < 4; ++q) tc_mma(tmem + 64u * g, dq + 2 * q, dk + 2 * q, idesc_qk, q == 0 ? 0u : 1u);   // 16 dimensions per instruction
+        tc_commit(s_full + g);
+      };
+      auto pv = [&](int j) {   // O of group j % 2 (+)= P V for job j
+        const int g = j & 1, k = j >> 1;
+        tc_wait(p_full + g, (uint32_t)k & 1u, failed, a.err);
+        tc_fence_after_sync();
+        const uint64_t dp = tc_smem_desc(Ps + g * 16384), dv = tc_smem_desc(slots + (size_t)(j % kPtSlots) * 16384 + kPageElems * 2);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)   // 16 tokens per instruction: 32 bytes along a P row, two 8-row groups (2048 bytes) down V
+          tc_mma(tmem + 128u + 64u * g, dp + 2 * q, dv + 128 * q, idesc_pv, (k == 0 && q == 0) ? 0u : 1u);
+        tc_commit(pv_done + g);
+      };
+      tc_wait(q_full, 0, failed, a.err);
+      if (n_job > 0) qk(0);
+      for (int i = 0; i < n_job; ++i) {
+        // Q K^T runs a job ahead of the softmax groups: S of job i + 1 is under way before this thread blocks on P of
+        // job i - 1, so a group finds its next S complete when it has handed over its P
+        if (i + 1 < n_job) qk(i + 1);
+        if (i > 0) pv(i - 1);
       }
-      __syncwarp();
+      if (n_job > 0) pv(n_job - 1);
     }
-    if (lane == 0 && n_job > 0) pv(n_job - 1);
     __syncwarp();
   } else {
-    // ---- softmax: thread t owns row t of the tile = accumulator lane t ----
-    const int t = threadIdx.x, r = r0 + t;
-    const uint32_t t_lane = tmem + ((uint32_t)(32 * warp) << 16);
-    {
+    // ---- softmax: group g = warps 4 g .. 4 g + 3 takes jobs g, g + 2, ...; thread t of a group owns row t = accumulator
+    //      lane t, with the group's own S, P and O; the two partial results meet at the end ----
+    const int g = warp >> 2, t = threadIdx.x & (kPtRows - 1), r = r0 + t;
+    const uint32_t t_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    const uint32_t t_S = t_lane + 64u * g, t_O = t_lane + 128u + 64u * g;
+    unsigned char *Pg = Ps + g * 16384;
+    if (g == 0) {
       // Q row of this head as bf16 into the swizzled tile (a row beyond the pass is zero)
       const float *qp = a.q + (size_t)r * a.H * kHeadDim + h * kHeadDim;
 #pragma unroll
@@ -198,19 +228,20 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
     const float qs = 0.125f * 1.4426950408889634f;   // scores in log2 units: 1/sqrt(64) * log2(e)
     const int pos = row_p[t];
     float m = -INFINITY, l = 0.f;
-    for (int j = 0; j < n_job; ++j) {
-      pt_warp_wait(s_full, (uint32_t)j & 1u, failed, a.err, lane);
+    int k = 0;
+    for (int j = g; j < n_job; j += 2, ++k) {
+      pt_warp_wait(s_full + g, (uint32_t)k & 1u, failed, a.err, lane);
       tc_fence_after_sync();
       float s[64];
       {
         float lo[32], hi[32];
-        tmem_ld32(t_lane, lo);
-        tmem_ld32(t_lane + 32u, hi);
+        tmem_ld32(t_S, lo);
+        tmem_ld32(t_S + 32u, hi);
 #pragma unroll
         for (int c = 0; c < 32; ++c) { s[c] = lo[c]; s[32 + c] = hi[c]; }
       }
       tc_fence_before_sync();
-      mbar_arrive(s_free);
+      mbar_arrive(s_free + g);
       const int sg = jobs[j] >> 8, pg = jobs[j] & 255;
       const bool act = r >= seg_i0[sg] && r < seg_i1[sg];
       const int see = act ? min(kPageTokens, pos + 1 - pg * kPageTokens) : 0;   // tokens of the page this row sees
@@ -229,42 +260,67 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
       for (int c = 0; c < 64; ++c) { s[c] = pt_exp2(s[c] - ref); sum4[c & 3] += s[c]; }
       const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l = l * sc + sum;
-      // P and O belong to the tensor core until P V of the job before has completed
-      if (j > 0) { pt_warp_wait(pv_done, (uint32_t)(j - 1) & 1u, failed, a.err, lane); tc_fence_after_sync(); }
+      // the group's P and O belong to the tensor core until P V of the group's job before has completed
+      if (k > 0) { pt_warp_wait(pv_done + g, (uint32_t)(k - 1) & 1u, failed, a.err, lane); tc_fence_after_sync(); }
 #pragma unroll
       for (int c8 = 0; c8 < 8; ++c8)
-        *reinterpret_cast<uint4 *>(Ps + t * 128 + ((c8 ^ (t & 7)) << 4)) =
+        *reinterpret_cast<uint4 *>(Pg + t * 128 + ((c8 ^ (t & 7)) << 4)) =
             make_uint4(pack_bf16x2(s[8 * c8], s[8 * c8 + 1]), pack_bf16x2(s[8 * c8 + 2], s[8 * c8 + 3]),
                        pack_bf16x2(s[8 * c8 + 4], s[8 * c8 + 5]), pack_bf16x2(s[8 * c8 + 6], s[8 * c8 + 7]));
       __syncwarp();
-      if (j > 0 && !__all_sync(0xFFFFFFFFu, sc == 1.0f)) {   // some row's maximum moved: rescale the warp's rows of O
+      if (k > 0 && !__all_sync(0xFFFFFFFFu, sc == 1.0f)) {   // some row's maximum moved: rescale the warp's rows of O
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
           float o[32];
-          tmem_ld32(t_lane + 64u + 32u * hh, o);
+          tmem_ld32(t_O + 32u * hh, o);
 #pragma unroll
           for (int c = 0; c < 32; ++c) o[c] *= sc;
-          tmem_st32(t_lane + 64u + 32u * hh, o);
+          tmem_st32(t_O + 32u * hh, o);
         }
       }
       fence_proxy_async_smem();
       tc_fence_before_sync();
-      mbar_arrive(p_full);
+      mbar_arrive(p_full + g);
     }
     trace_mark(a.trace, a.trace_slot, 3);
-    if (n_job > 0) {
-      pt_warp_wait(pv_done, (uint32_t)(n_job - 1) & 1u, failed, a.err, lane);
-      tc_fence_after_sync();
-      const float inv = l > 0.f ? 1.0f / l : 0.f;
+    // ---- the two groups' partial results: O = (O0 2^(m0 - M) + O1 2^(m1 - M)) / (l0 2^(m0 - M) + l1 2^(m1 - M)) ----
+    if (k > 0) { pt_warp_wait(pv_done + g, (uint32_t)(k - 1) & 1u, failed, a.err, lane); tc_fence_after_sync(); }
+    if (g == 1) {
+      ref1_s[t] = m; l1_s[t] = l;   // without a job of its own: m = -inf, l = 0, and Ms is not read
+      if (k > 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          float o[32];
+          tmem_ld32(t_O + 32u * hh, o);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) Ms[t * kPtMergePitch + 32 * hh + c] = o[c];
+        }
+      }
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(2 * kPtRows) : "memory");   // every softmax thread, once
+    if (g == 0 && n_job > 0) {
+      const float m1 = ref1_s[t], l1 = l1_s[t];
+      const float M = fmaxf(m, m1);
+      const float a0 = (m == -INFINITY) ? 0.f : pt_exp2(m - M), a1 = (m1 == -INFINITY) ? 0.f : pt_exp2(m1 - M);
+      const float lt = l * a0 + l1 * a1;
+      const float inv = lt > 0.f ? 1.0f / lt : 0.f;
+      const float w0 = a0 * inv, w1 = a1 * inv;
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
         float o[32];
-        tmem_ld32(t_lane + 64u + 32u * hh, o);
+        tmem_ld32(t_O + 32u * hh, o);
+        if (a1 != 0.f) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = o[c] * w0 + Ms[t * kPtMergePitch + 32 * hh + c] * w1;
+        } else {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] *= w0;
+        }
         if (r < R && !*failed) {
 #pragma unroll
           for (int c8 = 0; c8 < 4; ++c8) {
-            const uint4 y = make_uint4(pack_bf16x2(o[8 * c8] * inv, o[8 * c8 + 1] * inv), pack_bf16x2(o[8 * c8 + 2] * inv, o[8 * c8 + 3] * inv),
-                                       pack_bf16x2(o[8 * c8 + 4] * inv, o[8 * c8 + 5] * inv), pack_bf16x2(o[8 * c8 + 6] * inv, o[8 * c8 + 7] * inv));
+            const uint4 y = make_uint4(pack_bf16x2(o[8 * c8], o[8 * c8 + 1]), pack_bf16x2(o[8 * c8 + 2], o[8 * c8 + 3]),
+                                       pack_bf16x2(o[8 * c8 + 4], o[8 * c8 + 5]), pack_bf16x2(o[8 * c8 + 6], o[8 * c8 + 7]));
             const int col = h * kHeadDim + 32 * hh + 8 * c8;
             if (a.out_image) *reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(a.out) + act_image_offset_tiled(r, col, a.H * kHeadDim)) = y;
             else *reinterpret_cast<uint4 *>(a.out + (size_t)r * a.H * kHeadDim + col) = y;
@@ -276,10 +332,10 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
   tc_fence_before_sync();
   __syncthreads();
   trace_mark(a.trace, a.trace_slot, 2);
-  if (warp == 4) tmem_dealloc(tmem, 128);
+  if (warp == 8) tmem_dealloc(tmem, 256);
 }
 
-inline size_t attention_prefill_tc_smem_bytes() { return 32768 + (size_t)kPtSlots * 16384 + 1024 + 256; }
+inline size_t attention_prefill_tc_smem_bytes() { return 49152 + (size_t)kPtSlots * 16384 + (size_t)kPtRows * kPtMergePitch * 4 + 1024 + 256; }
 
 inline cudaError_t launch_attention_prefill_tc(const AttnArgs &a, int R, cudaStream_t st, bool pdl) {
   static PerDeviceOnce attr_once;   // per device: opt-in to more than 48 KB of dynamic shared memory
