@@ -245,19 +245,25 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
       const int sg = jobs[j] >> 8, pg = jobs[j] & 255;
       const bool act = r >= seg_i0[sg] && r < seg_i1[sg];
       const int see = act ? min(kPageTokens, pos + 1 - pg * kPageTokens) : 0;   // tokens of the page this row sees
+      // all but the last page of a row's own stream are seen whole by every row of the warp: no masks there
+      if (!__all_sync(0xFFFFFFFFu, see == kPageTokens)) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) s[c] = c < see ? s[c] : -INFINITY;
+      }
       // four independent chains for the maximum and for the sum: one chain of 64 dependent operations per row and
-      // page was the longest thing in the loop
+      // page was the longest thing in the loop.  The scale (positive) is applied to the maximum and inside the
+      // exponential's argument: one multiply-add per score.
       float pm4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 64; ++c) { s[c] = c < see ? s[c] * qs : -INFINITY; pm4[c & 3] = fmaxf(pm4[c & 3], s[c]); }
-      const float pm = fmaxf(fmaxf(pm4[0], pm4[1]), fmaxf(pm4[2], pm4[3]));
+      for (int c = 0; c < 64; ++c) pm4[c & 3] = fmaxf(pm4[c & 3], s[c]);
+      const float pm = fmaxf(fmaxf(pm4[0], pm4[1]), fmaxf(pm4[2], pm4[3])) * qs;
       const float m_new = fmaxf(m, pm);
       const float ref = (m_new == -INFINITY) ? 0.f : m_new;   // a row that has seen nothing yet keeps m = -inf
       const float sc = pt_exp2(m - ref);
       m = m_new;
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < 64; ++c) { s[c] = pt_exp2(s[c] - ref); sum4[c & 3] += s[c]; }
+      for (int c = 0; c < 64; ++c) { s[c] = pt_exp2(fmaf(s[c], qs, -ref)); sum4[c & 3] += s[c]; }
       const float sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       l = l * sc + sum;
       // the group's P and O belong to the tensor core until P V of the group's job before has completed
