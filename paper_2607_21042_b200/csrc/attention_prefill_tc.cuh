@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
   __shared__ int seg_stream[kPtRows], seg_i0[kPtRows], seg_i1[kPtRows], seg_last[kPtRows];
   __shared__ unsigned short jobs[kPtMaxJobs];   // (run << 8) | page, in run order
   __shared__ int n_job_s;
+  __shared__ unsigned run_open[kPtRows / 32];   // bit l of word w: row 32 w + l opens a run
   __shared__ int job_ph[kPtMaxJobs];            // physical page of each job
   __shared__ float ref1_s[kPtRows], l1_s[kPtRows];   // group 1's reference score and sum per row
 
@@ -110,16 +111,28 @@ __global__ void __launch_bounds__(kPtThreads) attention_prefill_tc_kernel(const 
   }
   if (warp == 8) tmem_alloc(tmem_slot, 256);   // S of group g: columns 64 g .. + 63, O of group g: columns 128 + 64 g .. + 63
   __syncthreads();
-  if (threadIdx.x == 0) {
-    const int n_rows = min(R - r0, kPtRows);
-    int n = 0, i0 = 0;
-    while (i0 < n_rows) {   // runs of rows of one stream
-      const int s = row_s[i0];
-      int i1 = i0 + 1;
-      while (i1 < n_rows && row_s[i1] == s) ++i1;
-      seg_stream[n] = s; seg_i0[n] = r0 + i0; seg_i1[n] = r0 + i1; seg_last[n] = row_p[i1 - 1];
-      ++n; i0 = i1;
+  // runs of rows of one stream, found by all rows at once: a row that differs from the one before opens a run, the
+  // number of openings up to a row is its run's index (this set-up is not hidden behind the kernel in front)
+  const int n_rows = min(R - r0, kPtRows);
+  if (threadIdx.x < kPtRows) {
+    const int t = threadIdx.x;
+    const bool first = t < n_rows && (t == 0 || row_s[t] != row_s[t - 1]);
+    const unsigned b = __ballot_sync(0xFFFFFFFFu, first);
+    if (lane == 0) run_open[warp] = b;
+  }
+  __syncthreads();
+  if (threadIdx.x < kPtRows) {
+    const int t = threadIdx.x;
+    int idx = __popc(run_open[warp] & (0xFFFFFFFFu >> (31 - lane))) - 1;
+    for (int w = 0; w < warp; ++w) idx += __popc(run_open[w]);
+    if (t < n_rows) {
+      if (t == 0 || row_s[t] != row_s[t - 1]) { seg_stream[idx] = row_s[t]; seg_i0[idx] = r0 + t; }
+      if (t == n_rows - 1 || row_s[t + 1] != row_s[t]) { seg_i1[idx] = r0 + t + 1; seg_last[idx] = row_p[t]; }
     }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int n = __popc(run_open[0]) + __popc(run_open[1]) + __popc(run_open[2]) + __popc(run_open[3]);
     int nj = 0;
     for (int sg = 0; sg < n; ++sg)
       for (int pg = 0; pg <= seg_last[sg] / kPageTokens && nj < kPtMaxJobs; ++pg) jobs[nj++] = (unsigned short)((sg << 8) | pg);
