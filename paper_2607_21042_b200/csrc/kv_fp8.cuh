@@ -60,6 +60,43 @@ __global__ void __launch_bounds__(64) kv_quantize_kernel(const uint16_t *__restr
   if (lane == 0) *reinterpret_cast<float *>(blk + kPageTokens * kHeadDim + 4 * (pos & 63)) = s;
 }
 
+// The same encoding for the many rows of a large prefill pass: one CTA of 8 warps per row; a warp takes the
+// (K|V, head) slices w, w + 8, ... of the row, five at a time with their loads in flight together (a grid of
+// one 64-thread CTA per row and head is 18 000 CTAs for a 896-row pass and takes 22 us).  Bit-identical codes.
+constexpr int kQrWarps = 8, kQrBatch = 5;
+__global__ void __launch_bounds__(kQrWarps * 32) kv_quantize_rows_kernel(const uint16_t *__restrict__ stage, unsigned char *__restrict__ kv_layer,
+                                                                         const int *__restrict__ page_table, const int *__restrict__ row_stream,
+                                                                         const int *__restrict__ row_pos, int pps, int H) {
+  const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int pos = row_pos[r];   // the row table is final before the pass's first kernel starts
+  const int page = page_table[(size_t)row_stream[r] * pps + (pos >> 6)];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int d = H * kHeadDim, n_items = 2 * H;
+  for (int it0 = warp; it0 < n_items; it0 += kQrWarps * kQrBatch) {
+    uint32_t pair[kQrBatch];
+#pragma unroll
+    for (int b = 0; b < kQrBatch; ++b) {
+      const int it = it0 + b * kQrWarps;   // item = which * H + head: the staged row is [K of all heads | V of all heads]
+      pair[b] = it < n_items ? *reinterpret_cast<const uint32_t *>(stage + (size_t)r * 2 * d + (size_t)it * kHeadDim + 2 * lane) : 0u;
+    }
+#pragma unroll
+    for (int b = 0; b < kQrBatch; ++b) {
+      const int it = it0 + b * kQrWarps;
+      if (it < n_items) {   // uniform in the warp
+        const int which = it / H, h = it - which * H;
+        const float x0 = bf16_lo(pair[b]), x1 = bf16_hi(pair[b]);
+        const float amax = warp_max(fmaxf(fabsf(x0), fabsf(x1)));
+        const float sc = amax > 0.f ? amax / kE4m3Max : 1.0f;
+        const __nv_fp8x2_storage_t codes = __nv_cvt_float2_to_fp8x2(make_float2(__fdiv_rn(x0, sc), __fdiv_rn(x1, sc)), __NV_SATFINITE, __NV_E4M3);
+        unsigned char *blk = kv_layer + (((size_t)page * 2 + which) * H + h) * kFp8BlockBytes;
+        *reinterpret_cast<uint16_t *>(blk + (size_t)(pos & 63) * kHeadDim + 2 * lane) = (uint16_t)codes;
+        if (lane == 0) *reinterpret_cast<float *>(blk + kPageTokens * kHeadDim + 4 * (pos & 63)) = sc;
+      }
+    }
+  }
+}
+
 struct Fp8AttnArgs {
   const float *q;                 // [R][H*64]
   const unsigned char *kv_layer;  // this layer's slice of the e4m3 pool
@@ -429,6 +466,8 @@ inline int attention_fp8_splits(int R, int H, int n_sm) {
 
 inline cudaError_t launch_kv_quantize(const uint16_t *stage, unsigned char *kv_layer, const int *page_table, const int *row_stream,
                                       const int *row_pos, int pps, int H, int R, cudaStream_t st, bool pdl) {
+  if (R > kMaxRows)   // a prefill pass of several row tiles
+    return launch_kernel(kv_quantize_rows_kernel, dim3(R), dim3(kQrWarps * 32), 0, st, pdl, stage, kv_layer, page_table, row_stream, row_pos, pps, H);
   return launch_kernel(kv_quantize_kernel, dim3(H, R), dim3(64), 0, st, pdl, stage, kv_layer, page_table, row_stream, row_pos, pps, H);
 }
 
