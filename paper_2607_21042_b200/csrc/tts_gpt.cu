@@ -94,7 +94,10 @@ struct tts_gpt {
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
   bool use_attn_tc = true;   // prefill passes of more than 128 rows: attention on tcgen05 (option "attn_tc")
   bool use_w4_dequant = true;   // int4 weights, prefill passes of more than 128 rows: the layer's weights dequantized to bf16 once per pass (option "w4_prefill_dequant")
-  char *wq_scratch[4] = {nullptr, nullptr, nullptr, nullptr};   // int4: bf16 images of one layer's QKV / O / FC1 / FC2 weights
+  char *wq_scratch[2][4] = {};   // int4: bf16 images of a layer's QKV / O / FC1 / FC2 weights, for even and odd layers
+  // int4: the dequantization of layer l + 1 runs on a stream of its own while layer l computes
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_deq[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
   int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); set at creation
                                  // to the most row tiles whose widest linear still runs as one wave of two CTAs per SM
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
@@ -260,7 +263,8 @@ size_t carve(tts_gpt *h, void *base) {
     h->partials = cv.take<float>(h->partials_floats);
     if (c.wfmt == WF_INT4) {
       const int NK[4][2] = {{3 * d, d}, {d, d}, {F, d}, {d, F}};
-      for (int i = 0; i < 4; ++i) h->wq_scratch[i] = NK[i][1] % 128 == 0 ? cv.take<char>(weight_image_bytes(NK[i][0], NK[i][1])) : nullptr;
+      for (int b = 0; b < 2; ++b)
+        for (int i = 0; i < 4; ++i) h->wq_scratch[b][i] = NK[i][1] % 128 == 0 ? cv.take<char>(weight_image_bytes(NK[i][0], NK[i][1])) : nullptr;
     }
   }
   return cv.off;
@@ -405,34 +409,57 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
   // int4 weights in a pass of several row tiles: the layer's four weight images are dequantized (code x group
   // scale, one rounding to bf16) into scratch images and the linears run ungrouped; the kernel with per-group
   // accumulators needs twice the registers and runs one CTA per SM
-  const bool deq = wide && c.wfmt == WF_INT4 && h->use_w4_dequant && h->wq_scratch[0] && h->wq_scratch[1] &&
-                   h->wq_scratch[2] && h->wq_scratch[3];
+  const bool deq = wide && c.wfmt == WF_INT4 && h->use_w4_dequant && h->wq_scratch[0][0] && h->wq_scratch[0][1] &&
+                   h->wq_scratch[0][2] && h->wq_scratch[0][3];
+  // With a second stream the images of layer l + 1 are written (into the other pair of scratch images) while layer l
+  // computes, and layer l's linears are launched behind an event; without one the dequantization sits in the pass's
+  // own stream in front of the layer, and the linears may not fetch weights ahead of their dependency wait.
+  const bool aside = deq && h->side != nullptr;
+  auto dequantize = [&](int l, cudaStream_t on, bool with_pdl) -> cudaError_t {
+    LayerW &L = h->layers[l];
+    const PackedLinear *pl[4] = {&L.qkv, &L.o, &L.fc1, &L.fc2};
+    DequantImgArgs da;
+    memset(&da, 0, sizeof da);
+    unsigned long long end = 0;
+    for (int i = 0; i < 4; ++i) {
+      da.src[i] = (const uint4 *)pl[i]->w; da.dst[i] = (uint4 *)h->wq_scratch[aside ? (l & 1) : 0][i]; da.scales[i] = pl[i]->s;
+      da.K[i] = pl[i]->K;
+      end += packed_weight_bytes(WF_INT4, pl[i]->N, pl[i]->K) / 16;
+      da.unit_end[i] = end;
+    }
+    h->launches += 1;
+    return launch_kernel(dequant_weight_images_kernel, dim3((unsigned)((end + 255) / 256)), dim3(256), 0, on, with_pdl, da);
+  };
+  int cur = 0;   // which pair of scratch images the current layer reads
   auto dequantized = [&](GemmTcArgs &a, int which) {
     if (!deq) return;
-    a.w_img = h->wq_scratch[which]; a.wfmt = WF_BF16; a.scales = nullptr; a.w_written_in_stream = 1;
+    a.w_img = h->wq_scratch[cur][which]; a.wfmt = WF_BF16; a.scales = nullptr; a.w_written_in_stream = aside ? 0 : 1;
   };
+  if (aside) {   // everything queued so far (the pass before read both pairs) precedes the first write
+    CUDA_TRY(h, cudaEventRecord(h->ev_start, st));
+    CUDA_TRY(h, cudaStreamWaitEvent(h->side, h->ev_start, 0));
+    CUDA_TRY(h, dequantize(0, h->side, false));
+    CUDA_TRY(h, cudaEventRecord(h->ev_deq[0], h->side));
+  }
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
     int rc;
-    if (deq) {
-      const PackedLinear *pl[4] = {&L.qkv, &L.o, &L.fc1, &L.fc2};
-      DequantImgArgs da;
-      memset(&da, 0, sizeof da);
-      unsigned long long end = 0;
-      for (int i = 0; i < 4; ++i) {
-        da.src[i] = (const uint4 *)pl[i]->w; da.dst[i] = (uint4 *)h->wq_scratch[i]; da.scales[i] = pl[i]->s;
-        da.K[i] = pl[i]->K;
-        end += packed_weight_bytes(WF_INT4, pl[i]->N, pl[i]->K) / 16;
-        da.unit_end[i] = end;
+    cur = aside ? (l & 1) : 0;
+    if (aside) {
+      if (l + 1 < c.n_layer) {   // the next layer's images, once the layer before this one has let go of that pair
+        if (l >= 1) CUDA_TRY(h, cudaStreamWaitEvent(h->side, h->ev_free[(l + 1) & 1], 0));
+        CUDA_TRY(h, dequantize(l + 1, h->side, false));
+        CUDA_TRY(h, cudaEventRecord(h->ev_deq[(l + 1) & 1], h->side));
       }
-      CUDA_TRY(h, launch_kernel(dequant_weight_images_kernel, dim3((unsigned)((end + 255) / 256)), dim3(256), 0, st, pdl, da));
-      h->launches += 1;
+    } else if (deq) {
+      CUDA_TRY(h, dequantize(l, st, pdl));
     }
     // fold the previous layer's FC2 partial sums into x, then LN1 -> image
     rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : f2_parts, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
                       h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
+    if (aside) CUDA_TRY(h, cudaStreamWaitEvent(st, h->ev_deq[cur], 0));   // this layer's images are complete
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
     dequantized(qa, 0);
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
@@ -464,6 +491,7 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     f2.out_f32 = f2_parts ? h->partials : h->x; f2.out_stride = d;
     trace_attach(h, f2);
     if ((rc = launch_gemm(h, f2, wide, st, pdl))) return rc;
+    if (aside) CUDA_TRY(h, cudaEventRecord(h->ev_free[cur], st));
     h->launches += 5;
   }
   h->tc_tail_parts = f2_parts;
@@ -710,7 +738,8 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
   {   // image rows past a matrix's last 8-row tile are never written by the per-pass dequantization
     const int NK[4][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}};
     for (int i = 0; i < 4; ++i)
-      if (e == cudaSuccess && h->wq_scratch[i]) e = cudaMemsetAsync(h->wq_scratch[i], 0, weight_image_bytes(NK[i][0], NK[i][1]), h->stream);
+      for (int b = 0; b < 2; ++b)
+        if (e == cudaSuccess && h->wq_scratch[b][i]) e = cudaMemsetAsync(h->wq_scratch[b][i], 0, weight_image_bytes(NK[i][0], NK[i][1]), h->stream);
   }
   if (e == cudaSuccess) {
     void *hp = nullptr, *dp = nullptr;
@@ -722,10 +751,24 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
       h->dev_err = (int *)dp;
     }
   }
+  if (e == cudaSuccess && c.wfmt == WF_INT4 && h->wq_scratch[1][0]) {
+    // the stream and events of the per-pass weight dequantization; without them it runs in the engine's stream
+    bool ok = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) == cudaSuccess;
+    cudaEvent_t *evs[5] = {&h->ev_start, &h->ev_deq[0], &h->ev_deq[1], &h->ev_free[0], &h->ev_free[1]};
+    for (cudaEvent_t *ev : evs) ok = ok && cudaEventCreateWithFlags(ev, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      if (h->side) cudaStreamDestroy(h->side);
+      h->side = nullptr;
+      for (cudaEvent_t *ev : evs) { if (*ev) cudaEventDestroy(*ev); *ev = nullptr; }
+      cudaGetLastError();
+    }
+  }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
   if (e != cudaSuccess) {
     if (h->host_err) cudaFreeHost((void *)h->host_err);
+    if (h->side) cudaStreamDestroy(h->side);
+    for (cudaEvent_t ev : {h->ev_start, h->ev_deq[0], h->ev_deq[1], h->ev_free[0], h->ev_free[1]}) if (ev) cudaEventDestroy(ev);
     delete h;
     return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(e));
   }
@@ -1046,6 +1089,8 @@ int32_t tts_gpt_sync(tts_gpt_t *h) {
 int32_t tts_gpt_destroy(tts_gpt_t *h) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   cudaStreamSynchronize(h->stream);
+  if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
+  for (cudaEvent_t e : {h->ev_start, h->ev_deq[0], h->ev_deq[1], h->ev_free[0], h->ev_free[1]}) if (e) cudaEventDestroy(e);
   for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second);
   if (h->host_err) cudaFreeHost((void *)h->host_err);
   delete h;
@@ -1113,6 +1158,7 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
   else if (k == "attn_tc") h->use_attn_tc = on;
   else if (k == "w4_prefill_dequant") h->use_w4_dequant = on;
+  else if (k == "w4_dequant_side_stream") { if (!on && h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); h->side = nullptr; } }
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;
   else if (k == "attn_stream") h->use_attn_stream = on;

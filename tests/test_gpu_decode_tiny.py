@@ -670,7 +670,13 @@ def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
     with pytest.raises(B.TtsGptError):
         eng.set_option("prefill_pass_rows", 200)
     if wfmt == C.W_INT4_G128:
-        # large passes dequantize a layer's int4 weights to bf16 images by default (one rounding per weight);
+        # large passes dequantize a layer's int4 weights to bf16 images by default (one rounding per weight), the
+        # next layer's on a second stream; without that stream the same kernel runs in front of each layer
+        eng.set_option("prefill_pass_rows", 512)
+        eng.set_option("w4_dequant_side_stream", 0)
+        lg4, tk4 = _run_batch(eng, prefixes, 4)
+        for s in range(S):
+            assert_same_up_to_ties(tk[s], lg[s], tk4[s], lg4[s], "dequantization in the engine's stream, stream %d" % s)
         # switched off, the kernel with per-group accumulators applies the scales to fp32 group sums
         eng.set_option("w4_prefill_dequant", 0)
         lg3, tk3 = _run_batch(eng, prefixes, 4)
