@@ -835,7 +835,7 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
 inline size_t gemm_tcw_smem_bytes(int stages) { return (size_t)stages * kTwStageBytes + 1024 + 2304; }
 
 // k-ranges of a residual linear in the wide kernel: at least 4 k-chunks per CTA, at most what LayerNorm folds
-inline int tcw_ksplit_resid(int K) { return std::max(1, std::min(kTwMaxPartials, (K / 64) / 4)); }
+inline int tcw_ksplit_resid(int K) { return std::max(1, std::min(kTwMaxPartials, (K / 64) / 8)); }
 
 // n_sm: SMs of the device; a grid that fits at one CTA per SM gets the deep ring
 inline cudaError_t launch_gemm_tcw(const GemmTcArgs &a0, int n_sm, cudaStream_t st, bool pdl) {
