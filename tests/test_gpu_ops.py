@@ -251,6 +251,29 @@ def test_attention_prefill_tcgen05_long_runs():
         assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -7 * np.abs(ref).max() + 1e-5, (r, s_, p_)
 
 
+def test_attention_prefill_tcgen05_many_short_streams():
+    """The 128-row tcgen05 variant where a tile holds many runs: 100 streams of one or two rows each (a run opens
+    on almost every row, runs cross warp boundaries, every job is a single page and alternate jobs go to the two
+    softmax groups), then a tile with one single-page stream only (the second group gets no job at all)."""
+    rng = np.random.default_rng(81)
+    H = 2
+    ctxs = [1 + (i % 2) for i in range(100)] + [50]
+    kv, pt, Ks, Vs = _attention_case(rng, H, ctxs, 110, 2)
+    short = [(s, p) for s in range(100) for p in range(ctxs[s])]
+    assert len(short) == 150
+    rows = short[:128] + [(100, p) for p in range(50)]   # tile 0: 86 short streams; tile 1: one stream, one page
+    R = len(rows)
+    q = rng.standard_normal(size=(R, H * 64)).astype(np.float32)
+    out = B.op_attention_cluster(torch.from_numpy(q).to(DEV), bits_dev(kv), torch.from_numpy(pt).to(DEV),
+                                 torch.tensor([s for s, _ in rows], dtype=torch.int32, device=DEV),
+                                 torch.tensor([p for _, p in rows], dtype=torch.int32, device=DEV), -3)
+    torch.cuda.synchronize()
+    got = bits_to_f64(out)
+    for r, (s_, p_) in enumerate(rows):
+        ref = _attention_ref(q[r].astype(np.float64), Ks[s_][:p_ + 1], Vs[s_][:p_ + 1], H)
+        assert np.max(np.abs(got[r] - ref)) <= 2.0 ** -7 * np.abs(ref).max() + 1e-5, (r, s_, p_)
+
+
 @pytest.mark.parametrize("R,d", [(1, 256), (5, 1280), (128, 1280), (3, 2048), (2, 128)])
 def test_layernorm_matches_oracle(R, d):
     rng = np.random.default_rng(R + d)
