@@ -224,9 +224,9 @@ int32_t tts_gpt_debug_check_canaries(tts_gpt_t *h, int32_t *bad_bytes);
  * step graphs.  Names: "graph", "pdl", "tc" and "tc_min_rows" (tensor-core
  * linears), "prefill_pass_rows" (rows per prefill pass: a multiple of 128 up to 1024; the default is chosen at creation
  * from the SM count and the model width, 896 for the 24-layer model on 148 SMs; passes of more than 128 rows need
- * the tensor-core path), "w4_prefill_dequant" (int4 weights: passes of more than 128 rows multiply by the layer's weights
- * dequantized to bf16, code x group scale rounded once, instead of scaling fp32 group sums; on by default), "w4_dequant_side_stream" (0: that dequantization runs in
- * the engine's own stream in front of each layer instead of a layer ahead on a second stream), "attn_tc", "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
+ * the tensor-core path), "w4_tc_exact" (int4 weights only: by default the operand images of the tensor-core path, used for more than 16 rows,
+ * hold code x group scale rounded once to bf16; 1 rewrites them as integer codes and the kernels scale fp32 sums per
+ * 128-column group, 0 writes the default back), "attn_tc", "attn_mma", "attn_prefill", "attn_stream", "attn_stream_min_pairs", "attn_cluster_fill",
  * "fc2_ksplit"; "poison_free_pages" (test aid standing in for a memory checker: every free page, and
  * from then on every released page, is filled with NaN in all layers, so that a kernel reading a slot no
  * token was written to poisons its result).  Unknown name or value out of range: TTS_GPT_E_ARG. */

@@ -113,22 +113,21 @@ __global__ void pack_weight_image_int4_kernel(const uint32_t *__restrict__ w, in
   dst[unit] = v;
 }
 
-// int4 weights for prefill passes of several row tiles: a layer's four linears are dequantized (code x
-// group scale, rounded once to bf16) from the packed streaming layout of linear.cuh (half a byte per
-// weight) into scratch operand images, so that the pass runs the ungrouped kernel.  One thread per
-// 16-byte unit of the source = 32 columns of one row inside one 128-column group = four 16-byte units
-// of one k-chunk of the image.  The codes and scales do not depend on the kernels in front and are
-// fetched ahead of the dependency wait; the stores come after it (the previous layer's linears read
-// the scratch).  Image rows past the last 8-row tile of the source are never written: they are zeroed
-// when the engine is created.
-struct DequantImgArgs {
+// int4 weights: the operand images of a layer's four linears written from the packed streaming layout of
+// linear.cuh (half a byte per weight), either dequantized (code x group scale, rounded once to bf16: the
+// linears then run as plain bf16 contractions) or as the integer codes (raw: the grouped kernels scale fp32
+// group sums).  One thread per 16-byte unit of the source = 32 columns of one row inside one 128-column
+// group = four 16-byte units of one k-chunk of the image.  Image rows past the last 8-row tile of the
+// source are never written: the caller zeroes the image first.
+struct Int4ImageArgs {
   const uint4 *src[4];         // packed int4 tiles [row tile of 8][K/128][32 lanes]
   uint4 *dst[4];               // operand images
   const uint16_t *scales[4];   // tiled scales [N/8][K/128][8]
   int K[4];
+  int raw;                     // 1: integer codes, 0: code x scale
   unsigned long long unit_end[4];   // running totals of source units
 };
-__global__ void __launch_bounds__(256) dequant_weight_images_kernel(const DequantImgArgs a) {
+__global__ void __launch_bounds__(256) int4_weight_images_kernel(const Int4ImageArgs a) {
   const unsigned long long unit = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   int s = 0;
   while (s < 3 && unit >= a.unit_end[s]) ++s;
@@ -144,12 +143,10 @@ __global__ void __launch_bounds__(256) dequant_weight_images_kernel(const Dequan
     const int kb = (int)(tile % KB), rt = (int)(tile / KB);
     const int row = rt * 8 + (lane >> 2), k = kb * 128 + 32 * (lane & 3);
     v = __ldg(a.src[s] + local);
-    sc = bf16_bits_to_float(__ldg(a.scales[s] + ((size_t)rt * KB + kb) * 8 + (row & 7)));
+    sc = a.raw ? 1.0f : bf16_bits_to_float(__ldg(a.scales[s] + ((size_t)rt * KB + kb) * 8 + (row & 7)));
     // units (k % 64) / 8 .. + 3 of image row `row`, k-chunk k / 64; logical unit u sits at u ^ (row % 8)
     out = a.dst[s] + ((size_t)(row >> 7) * KC + (k >> 6)) * (kTcABytes / 16) + (size_t)(row & 127) * 8;
   }
-  pdl_launch_dependents();
-  pdl_wait();
   if (live) {
     const int lane = (int)(unit & 31);   // unit_end values are multiples of 32
     const int row7 = (lane >> 2) & 7, u0 = ((32 * (lane & 3)) & 63) >> 3;
@@ -265,8 +262,6 @@ struct GemmTcArgs {
   int out_stride;
   void *out_img;            // EPI_GELU: activation image of the next linear (row length N)
   int gelu_tanh;
-  int w_written_in_stream;  // wide kernel: w_img is written by an earlier kernel of the stream (dequantized scratch
-                            // image), so no weight copy may start ahead of the dependency wait
   uint16_t *kv_layer;
   uint16_t *kv_stage;       // if set, K/V rows go here as bf16 [B][2][d] instead of into their page slots (8-bit KV cache)
   const int *page_table, *row_stream, *row_pos;
@@ -631,7 +626,7 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   const unsigned char *gX = reinterpret_cast<const unsigned char *>(a.act_img) + ((size_t)blockIdx.z * KC + kc0) * (kMaxRows * 128);
 
   const int pre = min(n_it, n_stage);
-  if (threadIdx.x == 0 && !a.w_written_in_stream) {
+  if (threadIdx.x == 0) {
     for (int i = 0; i < pre; ++i) {   // weights do not depend on the previous kernel
       mbar_expect_tx(full + i, kTwStageBytes);
       bulk_copy_g2s(ring + (size_t)i * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + i);
@@ -642,12 +637,6 @@ __global__ void __launch_bounds__(kTwThreads) gemm_tcw_kernel(const GemmTcArgs a
   trace_mark(a.trace, a.trace_slot, 1);
   if (warp == 0) {
     if (lane == 0) {
-      if (a.w_written_in_stream) {   // a weight image that a kernel earlier in the stream wrote: only after the wait
-        for (int i = 0; i < pre; ++i) {
-          mbar_expect_tx(full + i, kTwStageBytes);
-          bulk_copy_g2s(ring + (size_t)i * kTwStageBytes + 16384, gW + (size_t)i * kTcABytes, 16384, full + i);
-        }
-      }
       for (int i = 0; i < pre; ++i)
         bulk_copy_g2s(ring + (size_t)i * kTwStageBytes, gX + (size_t)i * (kMaxRows * 128), 16384, full + i);
       for (int i = pre; i < n_it; ++i) {

@@ -93,11 +93,7 @@ struct tts_gpt {
   size_t partials_floats = 0;
   bool use_tc = true;   // tensor-core path for more than 16 rows (option "tc")
   bool use_attn_tc = true;   // prefill passes of more than 128 rows: attention on tcgen05 (option "attn_tc")
-  bool use_w4_dequant = true;   // int4 weights, prefill passes of more than 128 rows: the layer's weights dequantized to bf16 once per pass (option "w4_prefill_dequant")
-  char *wq_scratch[2][4] = {};   // int4: bf16 images of a layer's QKV / O / FC1 / FC2 weights, for even and odd layers
-  // int4: the dequantization of layer l + 1 runs on a stream of its own while layer l computes
-  cudaStream_t side = nullptr;
-  cudaEvent_t ev_start = nullptr, ev_deq[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
+  bool w4_exact = false;   // int4 weights on the tensor-core path: images hold the integer codes and the kernels scale fp32 group sums (option "w4_tc_exact"); default: images hold code x group scale rounded to bf16
   int prefill_pass_rows = 768;   // rows per prefill pass (option "prefill_pass_rows": a multiple of 128 up to 1024); set at creation
                                  // to the most row tiles whose widest linear still runs as one wave of two CTAs per SM
   int tc_tail_parts = 0;  // partial sums the last FC2 of the tensor-core path left for the final LayerNorm
@@ -261,11 +257,6 @@ size_t carve(tts_gpt *h, void *base) {
     h->hf_img = cv.take<char>(act_image_bytes(d));
     h->partials_floats = (size_t)kTiles * std::max(kTcKSplit, kTwMaxPartials) * kMaxRows * d;   // [row tile][k-range][128][d]
     h->partials = cv.take<float>(h->partials_floats);
-    if (c.wfmt == WF_INT4) {
-      const int NK[4][2] = {{3 * d, d}, {d, d}, {F, d}, {d, F}};
-      for (int b = 0; b < 2; ++b)
-        for (int i = 0; i < 4; ++i) h->wq_scratch[b][i] = NK[i][1] % 128 == 0 ? cv.take<char>(weight_image_bytes(NK[i][0], NK[i][1])) : nullptr;
-    }
   }
   return cv.off;
 }
@@ -276,10 +267,35 @@ int copy_bf16(tts_gpt *h, uint16_t *dst, const void *src, size_t n, const char *
   return TTS_GPT_OK;
 }
 
+// int4 weights: the operand images of the tensor-core path, written from the packed streaming layout.  Default: code x
+// group scale rounded once to bf16, so that the linears of more than 16 rows run as plain bf16 contractions; with
+// w4_exact: the integer codes, and the kernels scale the fp32 sums of each 128-column group.
+int write_int4_images(tts_gpt *h) {
+  for (int l = 0; l < h->cfg.n_layer; ++l) {
+    LayerW &L = h->layers[l];
+    const PackedLinear *pl[4] = {&L.qkv, &L.o, &L.fc1, &L.fc2};
+    Int4ImageArgs da;
+    memset(&da, 0, sizeof da);
+    da.raw = h->w4_exact ? 1 : 0;
+    unsigned long long end = 0;
+    for (int i = 0; i < 4; ++i) {
+      if (!pl[i]->w_img) return TTS_GPT_OK;   // no tensor-core path for this shape
+      da.src[i] = (const uint4 *)pl[i]->w; da.dst[i] = (uint4 *)pl[i]->w_img; da.scales[i] = pl[i]->s;
+      da.K[i] = pl[i]->K;
+      end += packed_weight_bytes(WF_INT4, pl[i]->N, pl[i]->K) / 16;
+      da.unit_end[i] = end;
+    }
+    int4_weight_images_kernel<<<(unsigned)((end + 255) / 256), 256, 0, h->stream>>>(da);
+    CUDA_TRY(h, cudaGetLastError());
+  }
+  return TTS_GPT_OK;
+}
+
 int load_linear(tts_gpt *h, PackedLinear &pl, int wf, const void *w, const void *s, const void *b, const char *what) {
   if (!w || !b || (wf != WF_BF16 && !s)) return fail(h, TTS_GPT_E_ARG, "weights: %s has a null tensor", what);
   CUDA_TRY(h, launch_pack(wf, pl.N, pl.K, w, s, pl.w, pl.s, h->stream));
-  if (pl.w_img) CUDA_TRY(h, launch_pack_image(wf, pl.N, pl.K, w, pl.w_img, h->stream));
+  if (pl.w_img && wf == WF_INT4) CUDA_TRY(h, cudaMemsetAsync(pl.w_img, 0, weight_image_bytes(pl.N, pl.K), h->stream));   // written by write_int4_images; rows past the last 8-row tile stay zero
+  else if (pl.w_img) CUDA_TRY(h, launch_pack_image(wf, pl.N, pl.K, w, pl.w_img, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(pl.bias, b, (size_t)pl.N * 2, cudaMemcpyDeviceToDevice, h->stream));
   return TTS_GPT_OK;
 }
@@ -358,8 +374,10 @@ cudaError_t run_attention(tts_gpt *h, AttnArgs &aa, int R, cudaStream_t st, bool
 GemmTcArgs gemm_args(tts_gpt *h, const PackedLinear &pl, const void *act_img, int B, int mode, int ksplit) {
   GemmTcArgs a;
   memset(&a, 0, sizeof a);
-  a.wfmt = pl.s ? h->cfg.wfmt : WF_BF16;   // the LM head has no scales: bf16 in every format
-  a.scales = pl.s;
+  // the LM head has no scales: bf16 in every format; int4 images hold dequantized weights unless the exact form is on
+  const bool plain = !pl.s || (h->cfg.wfmt == WF_INT4 && !h->w4_exact);
+  a.wfmt = plain ? WF_BF16 : h->cfg.wfmt;
+  a.scales = plain ? nullptr : pl.s;
   a.w_img = pl.w_img; a.act_img = act_img; a.bias = pl.bias; a.N = pl.N; a.K = pl.K; a.B = B; a.mode = mode;
   a.ksplit = ksplit; a.err = h->dev_err;
   return a;
@@ -406,62 +424,15 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
   const int o_ks = wide ? tcw_ksplit_resid(d) : kTcKSplit;
   const int f2_ks = wide ? tcw_ksplit_resid(c.d_ff) : kTcKSplit;
   const int o_parts = o_ks > 1 ? o_ks : 0, f2_parts = f2_ks > 1 ? f2_ks : 0;   // 0: the linear added into x itself
-  // int4 weights in a pass of several row tiles: the layer's four weight images are dequantized (code x group
-  // scale, one rounding to bf16) into scratch images and the linears run ungrouped; the kernel with per-group
-  // accumulators needs twice the registers and runs one CTA per SM
-  const bool deq = wide && c.wfmt == WF_INT4 && h->use_w4_dequant && h->wq_scratch[0][0] && h->wq_scratch[0][1] &&
-                   h->wq_scratch[0][2] && h->wq_scratch[0][3];
-  // With a second stream the images of layer l + 1 are written (into the other pair of scratch images) while layer l
-  // computes, and layer l's linears are launched behind an event; without one the dequantization sits in the pass's
-  // own stream in front of the layer, and the linears may not fetch weights ahead of their dependency wait.
-  const bool aside = deq && h->side != nullptr;
-  auto dequantize = [&](int l, cudaStream_t on, bool with_pdl) -> cudaError_t {
-    LayerW &L = h->layers[l];
-    const PackedLinear *pl[4] = {&L.qkv, &L.o, &L.fc1, &L.fc2};
-    DequantImgArgs da;
-    memset(&da, 0, sizeof da);
-    unsigned long long end = 0;
-    for (int i = 0; i < 4; ++i) {
-      da.src[i] = (const uint4 *)pl[i]->w; da.dst[i] = (uint4 *)h->wq_scratch[aside ? (l & 1) : 0][i]; da.scales[i] = pl[i]->s;
-      da.K[i] = pl[i]->K;
-      end += packed_weight_bytes(WF_INT4, pl[i]->N, pl[i]->K) / 16;
-      da.unit_end[i] = end;
-    }
-    h->launches += 1;
-    return launch_kernel(dequant_weight_images_kernel, dim3((unsigned)((end + 255) / 256)), dim3(256), 0, on, with_pdl, da);
-  };
-  int cur = 0;   // which pair of scratch images the current layer reads
-  auto dequantized = [&](GemmTcArgs &a, int which) {
-    if (!deq) return;
-    a.w_img = h->wq_scratch[cur][which]; a.wfmt = WF_BF16; a.scales = nullptr; a.w_written_in_stream = aside ? 0 : 1;
-  };
-  if (aside) {   // everything queued so far (the pass before read both pairs) precedes the first write
-    CUDA_TRY(h, cudaEventRecord(h->ev_start, st));
-    CUDA_TRY(h, cudaStreamWaitEvent(h->side, h->ev_start, 0));
-    CUDA_TRY(h, dequantize(0, h->side, false));
-    CUDA_TRY(h, cudaEventRecord(h->ev_deq[0], h->side));
-  }
   for (int l = 0; l < c.n_layer; ++l) {
     LayerW &L = h->layers[l];
     uint16_t *kvl = h->kv + h->kv_layer_elems * l;
     int rc;
-    cur = aside ? (l & 1) : 0;
-    if (aside) {
-      if (l + 1 < c.n_layer) {   // the next layer's images, once the layer before this one has let go of that pair
-        if (l >= 1) CUDA_TRY(h, cudaStreamWaitEvent(h->side, h->ev_free[(l + 1) & 1], 0));
-        CUDA_TRY(h, dequantize(l + 1, h->side, false));
-        CUDA_TRY(h, cudaEventRecord(h->ev_deq[(l + 1) & 1], h->side));
-      }
-    } else if (deq) {
-      CUDA_TRY(h, dequantize(l, st, pdl));
-    }
     // fold the previous layer's FC2 partial sums into x, then LN1 -> image
     rc = launch_ln_tc(h, R, L.ln1_g, L.ln1_b, l == 0 ? 0 : f2_parts, l == 0 ? nullptr : h->layers[l - 1].fc2.bias,
                       h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
-    if (aside) CUDA_TRY(h, cudaStreamWaitEvent(st, h->ev_deq[cur], 0));   // this layer's images are complete
     GemmTcArgs qa = gemm_args(h, L.qkv, h->a_img, R, EPI_QKV, 1);
-    dequantized(qa, 0);
     qa.out_f32 = h->q; qa.out_stride = d; qa.kv_layer = kvl; qa.page_table = h->ps.page_table;
     qa.row_stream = h->rt.row_stream; qa.row_pos = h->rt.row_pos; qa.pps = h->pps; qa.d = d; qa.H = c.n_head;
     qa.kv_stage = h->kv_stage;
@@ -475,23 +446,19 @@ int run_layers_tc(tts_gpt *h, int R, bool decode) {
     trace_attach(h, aa);
     CUDA_TRY(h, run_attention(h, aa, R, st, pdl));
     GemmTcArgs oa = gemm_args(h, L.o, h->o_img, R, EPI_RESID, o_ks);
-    dequantized(oa, 1);
     oa.out_f32 = o_parts ? h->partials : h->x; oa.out_stride = d;
     trace_attach(h, oa);
     if ((rc = launch_gemm(h, oa, wide, st, pdl))) return rc;
     rc = launch_ln_tc(h, R, L.ln2_g, L.ln2_b, o_parts, L.o.bias, h->a_img, nullptr, nullptr, nullptr, nullptr, 1);
     if (rc) return rc;
     GemmTcArgs f1 = gemm_args(h, L.fc1, h->a_img, R, EPI_GELU, 1);
-    dequantized(f1, 2);
     f1.out_img = h->h_img; f1.gelu_tanh = c.gelu_tanh;
     trace_attach(h, f1);
     if ((rc = launch_gemm(h, f1, wide, st, pdl))) return rc;
     GemmTcArgs f2 = gemm_args(h, L.fc2, h->h_img, R, EPI_RESID, f2_ks);
-    dequantized(f2, 3);
     f2.out_f32 = f2_parts ? h->partials : h->x; f2.out_stride = d;
     trace_attach(h, f2);
     if ((rc = launch_gemm(h, f2, wide, st, pdl))) return rc;
-    if (aside) CUDA_TRY(h, cudaEventRecord(h->ev_free[cur], st));
     h->launches += 5;
   }
   h->tc_tail_parts = f2_parts;
@@ -729,18 +696,13 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
     TRY_(load_linear(h, L.fc1, c.wfmt, w->fc1_w[l], qz ? w->fc1_s[l] : nullptr, w->fc1_b[l], "fc1"));
     TRY_(load_linear(h, L.fc2, c.wfmt, w->fc2_w[l], qz ? w->fc2_s[l] : nullptr, w->fc2_b[l], "fc2"));
   }
+  if (c.wfmt == WF_INT4) TRY_(write_int4_images(h));
 #undef TRY_
   const int init_n = std::max(std::max(c.n_pages, c.max_streams * h->pps), c.max_streams);
   init_pages_kernel<<<(init_n + 255) / 256, 256, 0, h->stream>>>(h->ps);
   cudaError_t e = cudaMemsetAsync(h->attn_tickets, 0, (size_t)(h->kv_fp8 ? kMaxPassRows : kMaxRows) * c.n_head * sizeof(unsigned int), h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_lo, kCanaryByte, kCanaryBytes, h->stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(h->canary_hi, kCanaryByte, kCanaryBytes, h->stream);
-  {   // image rows past a matrix's last 8-row tile are never written by the per-pass dequantization
-    const int NK[4][2] = {{3 * c.d_model, c.d_model}, {c.d_model, c.d_model}, {c.d_ff, c.d_model}, {c.d_model, c.d_ff}};
-    for (int i = 0; i < 4; ++i)
-      for (int b = 0; b < 2; ++b)
-        if (e == cudaSuccess && h->wq_scratch[b][i]) e = cudaMemsetAsync(h->wq_scratch[b][i], 0, weight_image_bytes(NK[i][0], NK[i][1]), h->stream);
-  }
   if (e == cudaSuccess) {
     void *hp = nullptr, *dp = nullptr;
     e = cudaHostAlloc(&hp, sizeof(int), cudaHostAllocMapped);
@@ -751,24 +713,10 @@ int32_t tts_gpt_create(const tts_gpt_config_t *cfg, const tts_gpt_weights_t *w, 
       h->dev_err = (int *)dp;
     }
   }
-  if (e == cudaSuccess && c.wfmt == WF_INT4 && h->wq_scratch[1][0]) {
-    // the stream and events of the per-pass weight dequantization; without them it runs in the engine's stream
-    bool ok = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) == cudaSuccess;
-    cudaEvent_t *evs[5] = {&h->ev_start, &h->ev_deq[0], &h->ev_deq[1], &h->ev_free[0], &h->ev_free[1]};
-    for (cudaEvent_t *ev : evs) ok = ok && cudaEventCreateWithFlags(ev, cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) {
-      if (h->side) cudaStreamDestroy(h->side);
-      h->side = nullptr;
-      for (cudaEvent_t *ev : evs) { if (*ev) cudaEventDestroy(*ev); *ev = nullptr; }
-      cudaGetLastError();
-    }
-  }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
   if (e != cudaSuccess) {
     if (h->host_err) cudaFreeHost((void *)h->host_err);
-    if (h->side) cudaStreamDestroy(h->side);
-    for (cudaEvent_t ev : {h->ev_start, h->ev_deq[0], h->ev_deq[1], h->ev_free[0], h->ev_free[1]}) if (ev) cudaEventDestroy(ev);
     delete h;
     return fail(nullptr, TTS_GPT_E_CUDA, "create: %s", cudaGetErrorString(e));
   }
@@ -1089,8 +1037,6 @@ int32_t tts_gpt_sync(tts_gpt_t *h) {
 int32_t tts_gpt_destroy(tts_gpt_t *h) {
   if (!h) return fail(nullptr, TTS_GPT_E_ARG, "null handle");
   cudaStreamSynchronize(h->stream);
-  if (h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); }
-  for (cudaEvent_t e : {h->ev_start, h->ev_deq[0], h->ev_deq[1], h->ev_free[0], h->ev_free[1]}) if (e) cudaEventDestroy(e);
   for (auto &kv : h->graphs) cudaGraphExecDestroy(kv.second);
   if (h->host_err) cudaFreeHost((void *)h->host_err);
   delete h;
@@ -1157,8 +1103,13 @@ int32_t tts_gpt_debug_set_option(tts_gpt_t *h, const char *name, int32_t value) 
   else if (k == "prefill_pass_rows") { if (value < kMaxRows || value > kMaxPassRows || value % kMaxRows) return fail(h, TTS_GPT_E_ARG, "prefill_pass_rows must be a multiple of 128 from 128 to 1024"); h->prefill_pass_rows = value; }
   else if (k == "tc_min_rows") { if (value < 1 || value > kMaxRows) return fail(h, TTS_GPT_E_ARG, "tc_min_rows must be in 1..%d", kMaxRows); h->tc_min_rows = value; }
   else if (k == "attn_tc") h->use_attn_tc = on;
-  else if (k == "w4_prefill_dequant") h->use_w4_dequant = on;
-  else if (k == "w4_dequant_side_stream") { if (!on && h->side) { cudaStreamSynchronize(h->side); cudaStreamDestroy(h->side); h->side = nullptr; } }
+  else if (k == "w4_tc_exact") {
+    if (h->cfg.wfmt != WF_INT4) return fail(h, TTS_GPT_E_ARG, "w4_tc_exact needs int4 weights");
+    h->w4_exact = on;
+    int rc = write_int4_images(h);   // the images change their meaning with the option
+    if (rc) return rc;
+    CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  }
   else if (k == "attn_mma") h->use_attn_mma = on;
   else if (k == "attn_prefill") h->use_attn_prefill = on;
   else if (k == "attn_stream") h->use_attn_stream = on;

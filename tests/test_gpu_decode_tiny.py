@@ -140,6 +140,19 @@ def test_medium_batches_match_oracle(wfmt, S):
         ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk[s][:-1])
         assert_logits_close(lg[s], ref, "batch of %d, stream %d" % (S, s))
         check_tokens(tk[s], ref, 0, 1.0, None, "batch of %d, stream %d" % (S, s))
+    if wfmt == C.W_INT4_G128 and S == 40:
+        # the tensor-core path multiplies by int4 weights dequantized to bf16 (one rounding per weight) by default;
+        # with w4_tc_exact its images hold the integer codes and the kernels scale fp32 sums per 128-column group
+        eng.set_option("w4_tc_exact", 1)
+        lg2, tk2 = _run_batch(eng, prefixes, n)
+        for s in range(0, S, max(1, S // 6)):
+            ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk2[s][:-1])
+            assert_logits_close(lg2[s], ref, "batch of %d with group sums, stream %d" % (S, s))
+            assert_same_up_to_ties(tk[s], lg[s], tk2[s], lg2[s], "group sums, stream %d" % s)
+        eng.set_option("w4_tc_exact", 0)
+        lg3, tk3 = _run_batch(eng, prefixes, n)
+        for s in range(S):
+            assert np.array_equal(tk3[s], tk[s]) and np.array_equal(lg3[s], lg[s]), "images restored, stream %d" % s
     eng.destroy()
 
 
@@ -670,20 +683,17 @@ def test_prefill_passes_of_several_row_tiles_match_oracle(wfmt):
     with pytest.raises(B.TtsGptError):
         eng.set_option("prefill_pass_rows", 200)
     if wfmt == C.W_INT4_G128:
-        # large passes dequantize a layer's int4 weights to bf16 images by default (one rounding per weight), the
-        # next layer's on a second stream; without that stream the same kernel runs in front of each layer
+        # with w4_tc_exact the wide kernel with per-group accumulators applies the scales to fp32 group sums
         eng.set_option("prefill_pass_rows", 512)
-        eng.set_option("w4_dequant_side_stream", 0)
-        lg4, tk4 = _run_batch(eng, prefixes, 4)
-        for s in range(S):
-            assert_same_up_to_ties(tk[s], lg[s], tk4[s], lg4[s], "dequantization in the engine's stream, stream %d" % s)
-        # switched off, the kernel with per-group accumulators applies the scales to fp32 group sums
-        eng.set_option("w4_prefill_dequant", 0)
+        eng.set_option("w4_tc_exact", 1)
         lg3, tk3 = _run_batch(eng, prefixes, 4)
         for s in range(S):
             ref, _ = O.replay_full(model, O.bf16_to_f64(prefixes[s]), tk3[s][:-1])
             assert_logits_close(lg3[s], ref, "multi-tile prefill with group accumulators, stream %d" % s)
             assert_same_up_to_ties(tk[s], lg[s], tk3[s], lg3[s], "group accumulators, stream %d" % s)
+    else:
+        with pytest.raises(B.TtsGptError):   # the option belongs to int4 weights
+            eng.set_option("w4_tc_exact", 1)
     eng.destroy()
 
 
